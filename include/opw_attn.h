@@ -1,0 +1,188 @@
+/*
+ * opw_attn.h -- C ABI of the decode-time core-attention stage (sm_100a).
+ *
+ * The stage is the operator that core-attention disaggregation (CAD) places on its own
+ * device group: per decode step a (micro)batch of one-token queries arrives together
+ * with the step's new key/value rows, the rows are appended to a paged KV cache that
+ * stays resident on the stage, grouped-query attention (full or sliding-window) runs
+ * over each sequence's pages, and the attention output goes back to the next stage
+ * (paper: Section 3.4 "From Bounds to Plans: CAD and Its Limits"; Section 4, the CAD
+ * template "isolates only the core attention kernels"; Section 6, first paragraph:
+ * slots, shapes and buffers are static and bound once while token, position and
+ * KV-cache metadata change between iterations).
+ *
+ * Conventions that hold for every entry point:
+ *   - Plain C: no C++ types, no exceptions cross this boundary.  Every call returns an
+ *     opw_status_t; nothing aborts, traps or waits without a bound.
+ *   - "DEVICE" pointers are CUDA device addresses on the stage's device; "HOST"
+ *     pointers are ordinary host addresses.  The library never allocates or frees
+ *     device memory: pools, workspace, inputs and outputs are caller-owned and must
+ *     stay valid until the work enqueued on the stream has finished.
+ *   - Step calls only enqueue work on the given stream (a cudaStream_t passed as
+ *     void*, NULL = default stream) and return; they never synchronise and never read
+ *     device metadata on the host, so launch shapes depend only on create-time
+ *     constants and on the `batch` argument.
+ *   - One handle is used from one host thread at a time.
+ *
+ * KV pool layout (per layer, part of this ABI).  bf16 elements.  Element
+ * (page p, kv head g, kv in {K = 0, V = 1}, slot t in [0, page_size), dim d) is at
+ *     ((((p*Hkv + g)*2 + kv)*page_size + t)*D) + (((d/8) ^ (t & 7))*8) + (d % 8).
+ * So each (page, head) owns one contiguous K tile followed by one V tile, each
+ * page_size rows of D elements; inside a row the eight-element (16-byte) groups are
+ * permuted by XOR with the low three bits of the slot (this makes a tile that is
+ * copied linearly into shared memory conflict-free for matrix loads).
+ * opw_kv_pool_index() evaluates the formula on the host.
+ */
+#ifndef OPW_ATTN_H_
+#define OPW_ATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct opw_attn_stage opw_attn_stage_t; /* opaque handle (host memory only) */
+
+typedef enum {
+  OPW_OK = 0,
+  OPW_ERR_INVALID_ARG = 1, /* NULL pointer, index out of range, misaligned pointer, bad struct_size */
+  OPW_ERR_UNSUPPORTED = 2, /* head_dim / page_size / group size the kernels do not cover */
+  OPW_ERR_CAPACITY = 3,    /* batch > max_batch, workspace too small */
+  OPW_ERR_CUDA = 4,        /* a CUDA runtime call or launch failed (no device, bad stream ...) */
+  OPW_ERR_BAD_PAGE = 5,    /* device side: a page id outside [0, num_pages) or a position beyond the table */
+  OPW_ERR_TIMEOUT = 6      /* device side: a bounded wait on a shared-memory copy ran out */
+} opw_status_t;
+
+#define OPW_FLAG_NONE 0u
+
+typedef struct {
+  uint32_t struct_size;           /* sizeof(opw_attn_stage_config_t); checked at create */
+  int32_t device;                 /* CUDA ordinal the stage lives on */
+  int32_t num_layers;             /* layers this stage owns (>= 1) */
+  int32_t num_q_heads;            /* Hq */
+  int32_t num_kv_heads;           /* Hkv; Hq % Hkv == 0 and Hq / Hkv <= 16 */
+  int32_t head_dim;               /* D: 64 or 128 */
+  int32_t page_size;              /* 16 */
+  int32_t max_batch;              /* static slot count; every call has batch <= max_batch */
+  int32_t max_pages_per_seq;      /* row stride (entries) of every page table */
+  const int32_t *layer_window;    /* HOST [num_layers]; 0 = full attention, W > 0 = the last W keys
+                                     including the current token (Section 3.4: efficient layers
+                                     "access a bounded window") */
+  const int64_t *layer_num_pages; /* HOST [num_layers]; physical pages in each layer's pool */
+  void *const *layer_kv_pool;     /* HOST [num_layers] of DEVICE pointers, 128-byte aligned, each at
+                                     least opw_kv_pool_bytes() long; caller-owned */
+  void *workspace;                /* DEVICE, 256-byte aligned, caller-owned scratch */
+  size_t workspace_bytes;         /* >= opw_attn_stage_workspace_bytes(cfg) */
+  float softmax_scale;            /* 0 -> 1/sqrt(head_dim) */
+  uint32_t flags;                 /* OPW_FLAG_* */
+  int32_t tune_warps;             /* 0 = default; warps per thread block (1..8) */
+  int32_t tune_stages;            /* 0 = default; shared-memory ring depth per warp (2..16) */
+  int32_t tune_ctas_per_sm;       /* 0 = default; resident thread blocks per SM (1..4) */
+  int32_t reserved;               /* must be 0 */
+} opw_attn_stage_config_t;
+
+/* Host helper: the pool layout formula above.  No device needed. */
+int64_t opw_kv_pool_index(int64_t num_kv_heads, int64_t page_size, int64_t head_dim, int64_t page,
+                          int64_t kv_head, int64_t kv, int64_t slot, int64_t dim);
+
+/* Host helper: bytes of one layer's pool holding num_pages pages (0 on invalid arguments). */
+size_t opw_kv_pool_bytes(int32_t num_kv_heads, int32_t page_size, int32_t head_dim, int64_t num_pages);
+
+/*
+ * Host helper: scratch bytes the stage needs (status word, split-KV bookkeeping and
+ * partial results, staging buffers of the host-buffer step).  Depends only on the
+ * shape fields and the tune_* fields; device pointers in cfg are ignored.  Returns 0
+ * if cfg is NULL or its shape fields are invalid.  Needs a CUDA device only to read
+ * the SM count; without one it assumes 148 SMs.
+ */
+size_t opw_attn_stage_workspace_bytes(const opw_attn_stage_config_t *cfg);
+
+/*
+ * Binds the static part of the stage (Section 6: shapes, slots and buffers are bound
+ * once).  Validates cfg on the host first (returning INVALID_ARG / UNSUPPORTED /
+ * CAPACITY without touching CUDA), then selects the device, reads its SM count, raises
+ * the kernels' shared-memory limit and clears the status word in the workspace
+ * (synchronously, on the default stream).  Copies layer_window, layer_num_pages and
+ * the pool pointers; those host arrays need not outlive the call.  *out is written
+ * only on OPW_OK.
+ */
+opw_status_t opw_attn_stage_create(const opw_attn_stage_config_t *cfg, opw_attn_stage_t **out);
+
+/*
+ * KV append (Section 6: KV-cache contents and metadata change every iteration).  For
+ * every b < batch with positions[b] >= 0, copies k_new[b] and v_new[b] bit for bit into
+ * slot positions[b] % page_size of page page_table[b][positions[b] / page_size] of the
+ * layer's pool.  positions[b] < 0 marks an inactive slot (nothing written).
+ *   k_new, v_new : DEVICE bf16 [batch, Hkv, D], 16-byte aligned
+ *   positions    : DEVICE int32 [batch]; the pre-append length of each sequence
+ *   page_table   : DEVICE int32 [batch, max_pages_per_seq]
+ * Two rows of one call must not target the same (page, slot).  A page id outside
+ * [0, num_pages) or a position beyond the table is skipped and recorded as
+ * OPW_ERR_BAD_PAGE in the status word (see opw_attn_stage_poll_error).
+ */
+opw_status_t opw_kv_append(opw_attn_stage_t *stage, int32_t layer, int32_t batch, const void *k_new,
+                           const void *v_new, const int32_t *positions, const int32_t *page_table,
+                           void *cuda_stream);
+
+/*
+ * Decode attention (Section 3.1 and Appendix A: memory-bound, latency = KV bytes over
+ * bandwidth; Section 3.4: full layers read the whole context, window layers a bounded
+ * window).  For every b < batch with n = kv_lens[b] > 0 and every query head h:
+ *     out[b,h,:] = sum_j softmax_j(scale * <q[b,h,:], K_j[h/G,:]>) V_j[h/G,:],
+ *     lse[b,h]   = log sum_j exp(scale * <q[b,h,:], K_j[h/G,:]>)
+ * over the keys j in [lo, n), lo = 0 for a full layer and max(0, n - W) for a window
+ * layer; G = Hq/Hkv; keys are read through page_table[b][j / page_size].  Rows with
+ * kv_lens[b] <= 0 are inactive: out = 0, lse = -inf.  bf16 inputs, fp32 accumulation,
+ * bf16 output rounded to nearest even.
+ *   q       : DEVICE bf16 [batch, Hq, D], 16-byte aligned
+ *   kv_lens : DEVICE int32 [batch]; keys visible after this step's append
+ *   page_table : DEVICE int32 [batch, max_pages_per_seq]; entries outside the visible
+ *             range (after the last page, or wholly before the window) are never read
+ *   out     : DEVICE bf16 [batch, Hq, D], 16-byte aligned
+ *   lse     : DEVICE float [batch, Hq] or NULL
+ * Enqueues two kernels (split-KV partial attention, then the log-sum-exp combine).
+ * The split of each sequence depends only on kv_lens and the window, never on the
+ * page ids, so permuting physical pages leaves the output bitwise unchanged.  Bad page
+ * ids are masked out and recorded as OPW_ERR_BAD_PAGE.
+ */
+opw_status_t opw_decode_attention(opw_attn_stage_t *stage, int32_t layer, int32_t batch, const void *q,
+                                  const int32_t *kv_lens, const int32_t *page_table, void *out, float *lse,
+                                  void *cuda_stream);
+
+/*
+ * One whole stage step from HOST buffers (Section 4: the stage's activation interface
+ * is the per-request q/k/v in and attention output back): copies q, k_new, v_new,
+ * positions and (if not NULL) page_table to staging areas in the workspace, runs the
+ * append and the attention with kv_lens = positions + 1, and copies out (and lse if
+ * not NULL) back to the host, all enqueued on the stream.  Host buffers should be
+ * pinned for the copies to be asynchronous; they must stay valid and unmodified until
+ * the stream has passed the step.  page_table_host == NULL reuses the table staged by
+ * the previous call for this layer's slot (tables rarely change between steps).
+ */
+opw_status_t opw_decode_step_host(opw_attn_stage_t *stage, int32_t layer, int32_t batch, const void *q_host,
+                                  const void *k_new_host, const void *v_new_host, const int32_t *positions_host,
+                                  const int32_t *page_table_host, void *out_host, float *lse_host,
+                                  void *cuda_stream);
+
+/*
+ * Synchronises the stream, then returns and clears the device status word: OPW_OK, or
+ * the first of OPW_ERR_BAD_PAGE / OPW_ERR_TIMEOUT recorded by a kernel since the last
+ * poll.  The only entry point that blocks.
+ */
+opw_status_t opw_attn_stage_poll_error(opw_attn_stage_t *stage, void *cuda_stream);
+
+/* Kernels launched through this handle since create (the library's own count). */
+int64_t opw_attn_stage_launch_count(const opw_attn_stage_t *stage);
+
+/* Frees the host-side handle.  Does not touch device memory.  NULL is accepted. */
+opw_status_t opw_attn_stage_destroy(opw_attn_stage_t *stage);
+
+/* Static string for a status code. */
+const char *opw_status_string(opw_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* OPW_ATTN_H_ */

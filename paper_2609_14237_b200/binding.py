@@ -1,0 +1,282 @@
+"""ctypes binding of the C-ABI library (argument marshalling only).
+
+Every function here has the name and the meaning of the entry point it wraps (see
+``include/opw_attn.h``).  Tensors are passed as raw device (or host) addresses; torch is
+used by callers for memory and streams only.  There is no fallback: if the shared
+library is missing, or was built without the kernels, importing ``lib()`` raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from typing import Optional, Sequence
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_ROOT = os.path.dirname(_HERE)
+LIB_PATH = os.path.join(_HERE, "libopw_attn.so")
+SOURCES = [os.path.join(_HERE, "csrc", "opw_attn.cu")]
+HEADERS = [os.path.join(_HERE, "csrc", "opw_kernels.cuh"), os.path.join(_ROOT, "include", "opw_attn.h")]
+
+OPW_OK, OPW_ERR_INVALID_ARG, OPW_ERR_UNSUPPORTED, OPW_ERR_CAPACITY, OPW_ERR_CUDA, OPW_ERR_BAD_PAGE, OPW_ERR_TIMEOUT = range(7)
+
+EXPORTS = [
+    "opw_kv_pool_index", "opw_kv_pool_bytes", "opw_attn_stage_workspace_bytes", "opw_attn_stage_create",
+    "opw_kv_append", "opw_decode_attention", "opw_decode_step_host", "opw_attn_stage_poll_error",
+    "opw_attn_stage_launch_count", "opw_attn_stage_destroy", "opw_status_string",
+]
+
+
+class StageConfig(ctypes.Structure):
+    _fields_ = [
+        ("struct_size", ctypes.c_uint32),
+        ("device", ctypes.c_int32),
+        ("num_layers", ctypes.c_int32),
+        ("num_q_heads", ctypes.c_int32),
+        ("num_kv_heads", ctypes.c_int32),
+        ("head_dim", ctypes.c_int32),
+        ("page_size", ctypes.c_int32),
+        ("max_batch", ctypes.c_int32),
+        ("max_pages_per_seq", ctypes.c_int32),
+        ("layer_window", ctypes.POINTER(ctypes.c_int32)),
+        ("layer_num_pages", ctypes.POINTER(ctypes.c_int64)),
+        ("layer_kv_pool", ctypes.POINTER(ctypes.c_void_p)),
+        ("workspace", ctypes.c_void_p),
+        ("workspace_bytes", ctypes.c_size_t),
+        ("softmax_scale", ctypes.c_float),
+        ("flags", ctypes.c_uint32),
+        ("tune_warps", ctypes.c_int32),
+        ("tune_stages", ctypes.c_int32),
+        ("tune_ctas_per_sm", ctypes.c_int32),
+        ("reserved", ctypes.c_int32),
+    ]
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    """Compile the library in-tree for sm_100a with nvcc (cross-compiles without a GPU)."""
+    srcs = [s for s in SOURCES if os.path.exists(s)]
+    deps = srcs + HEADERS
+    if not force and os.path.exists(LIB_PATH) and all(os.path.getmtime(LIB_PATH) >= os.path.getmtime(d) for d in deps):
+        return LIB_PATH
+    tmp = LIB_PATH + f".tmp{os.getpid()}"
+    cmd = [
+        "nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+        "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(_ROOT, "include"), "-o", tmp, *srcs,
+    ]
+    if verbose:
+        cmd.insert(1, "-Xptxas=-v")
+    subprocess.check_call(cmd)
+    os.replace(tmp, LIB_PATH)
+    return LIB_PATH
+
+
+class OpwError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load the C-ABI library; raises if it has not been built (no CPU fallback exists)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: run `python -c 'import __graft_entry__ as g; g.build()'` first")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, i64 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64
+    L.opw_kv_pool_index.restype = i64
+    L.opw_kv_pool_index.argtypes = [i64] * 8
+    L.opw_kv_pool_bytes.restype = ctypes.c_size_t
+    L.opw_kv_pool_bytes.argtypes = [i32, i32, i32, i64]
+    L.opw_attn_stage_workspace_bytes.restype = ctypes.c_size_t
+    L.opw_attn_stage_workspace_bytes.argtypes = [ctypes.POINTER(StageConfig)]
+    L.opw_attn_stage_create.restype = ctypes.c_int
+    L.opw_attn_stage_create.argtypes = [ctypes.POINTER(StageConfig), ctypes.POINTER(vp)]
+    L.opw_kv_append.restype = ctypes.c_int
+    L.opw_kv_append.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
+    L.opw_decode_attention.restype = ctypes.c_int
+    L.opw_decode_attention.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
+    L.opw_decode_step_host.restype = ctypes.c_int
+    L.opw_decode_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.opw_attn_stage_poll_error.restype = ctypes.c_int
+    L.opw_attn_stage_poll_error.argtypes = [vp, vp]
+    L.opw_attn_stage_launch_count.restype = i64
+    L.opw_attn_stage_launch_count.argtypes = [vp]
+    L.opw_attn_stage_destroy.restype = ctypes.c_int
+    L.opw_attn_stage_destroy.argtypes = [vp]
+    L.opw_status_string.restype = ctypes.c_char_p
+    L.opw_status_string.argtypes = [ctypes.c_int]
+    _lib = L
+    return L
+
+
+def status_string(status: int) -> str:
+    return lib().opw_status_string(int(status)).decode()
+
+
+def opw_kv_pool_index(Hkv: int, P: int, D: int, page: int, g: int, kv: int, t: int, d: int) -> int:
+    return int(lib().opw_kv_pool_index(Hkv, P, D, page, g, kv, t, d))
+
+
+def opw_kv_pool_bytes(Hkv: int, P: int, D: int, num_pages: int) -> int:
+    return int(lib().opw_kv_pool_bytes(Hkv, P, D, num_pages))
+
+
+def make_config(*, device: int, num_q_heads: int, num_kv_heads: int, head_dim: int, max_batch: int,
+                max_pages_per_seq: int, layer_window: Sequence[int], layer_num_pages: Sequence[int],
+                layer_kv_pool: Sequence[int], workspace: int = 0, workspace_bytes: int = 0, page_size: int = 16,
+                softmax_scale: float = 0.0, flags: int = 0, tune_warps: int = 0, tune_stages: int = 0,
+                tune_ctas_per_sm: int = 0):
+    """Fill a StageConfig; returns (cfg, keepalive) -- keep `keepalive` until create returns."""
+    L = len(layer_window)
+    win = (ctypes.c_int32 * L)(*[int(w) for w in layer_window])
+    npg = (ctypes.c_int64 * L)(*[int(n) for n in layer_num_pages])
+    pools = (ctypes.c_void_p * L)(*[int(p) for p in layer_kv_pool])
+    cfg = StageConfig()
+    cfg.struct_size = ctypes.sizeof(StageConfig)
+    cfg.device = device
+    cfg.num_layers = L
+    cfg.num_q_heads = num_q_heads
+    cfg.num_kv_heads = num_kv_heads
+    cfg.head_dim = head_dim
+    cfg.page_size = page_size
+    cfg.max_batch = max_batch
+    cfg.max_pages_per_seq = max_pages_per_seq
+    cfg.layer_window = ctypes.cast(win, ctypes.POINTER(ctypes.c_int32))
+    cfg.layer_num_pages = ctypes.cast(npg, ctypes.POINTER(ctypes.c_int64))
+    cfg.layer_kv_pool = ctypes.cast(pools, ctypes.POINTER(ctypes.c_void_p))
+    cfg.workspace = workspace
+    cfg.workspace_bytes = workspace_bytes
+    cfg.softmax_scale = softmax_scale
+    cfg.flags = flags
+    cfg.tune_warps = tune_warps
+    cfg.tune_stages = tune_stages
+    cfg.tune_ctas_per_sm = tune_ctas_per_sm
+    cfg.reserved = 0
+    return cfg, (win, npg, pools)
+
+
+def opw_attn_stage_workspace_bytes(cfg: StageConfig) -> int:
+    return int(lib().opw_attn_stage_workspace_bytes(ctypes.byref(cfg)))
+
+
+def opw_attn_stage_create(cfg: StageConfig) -> int:
+    """Returns the opaque handle (an integer address); raises OpwError on failure."""
+    h = ctypes.c_void_p()
+    rc = lib().opw_attn_stage_create(ctypes.byref(cfg), ctypes.byref(h))
+    if rc != OPW_OK:
+        raise OpwError(rc, "opw_attn_stage_create")
+    return h.value
+
+
+def _check(rc: int, where: str) -> None:
+    if rc != OPW_OK:
+        raise OpwError(rc, where)
+
+
+def opw_kv_append(stage: int, layer: int, batch: int, k_new: int, v_new: int, positions: int, page_table: int,
+                  stream: Optional[int] = None) -> None:
+    _check(lib().opw_kv_append(stage, layer, batch, k_new, v_new, positions, page_table, stream), "opw_kv_append")
+
+
+def opw_decode_attention(stage: int, layer: int, batch: int, q: int, kv_lens: int, page_table: int, out: int,
+                         lse: Optional[int] = None, stream: Optional[int] = None) -> None:
+    _check(lib().opw_decode_attention(stage, layer, batch, q, kv_lens, page_table, out, lse, stream),
+           "opw_decode_attention")
+
+
+def opw_decode_step_host(stage: int, layer: int, batch: int, q_host: int, k_new_host: int, v_new_host: int,
+                         positions_host: int, page_table_host: Optional[int], out_host: int,
+                         lse_host: Optional[int] = None, stream: Optional[int] = None) -> None:
+    _check(lib().opw_decode_step_host(stage, layer, batch, q_host, k_new_host, v_new_host, positions_host,
+                                      page_table_host, out_host, lse_host, stream), "opw_decode_step_host")
+
+
+def opw_attn_stage_poll_error(stage: int, stream: Optional[int] = None) -> int:
+    return int(lib().opw_attn_stage_poll_error(stage, stream))
+
+
+def opw_attn_stage_launch_count(stage: int) -> int:
+    return int(lib().opw_attn_stage_launch_count(stage))
+
+
+def opw_attn_stage_destroy(stage: Optional[int]) -> None:
+    _check(lib().opw_attn_stage_destroy(stage), "opw_attn_stage_destroy")
+
+
+class Stage:
+    """Convenience owner of one stage handle over caller-provided torch tensors.
+
+    Holds references to the pools and the workspace so they outlive the handle.  All
+    methods forward to the C entry points of the same name.
+    """
+
+    def __init__(self, *, pools, layer_window, num_q_heads, num_kv_heads, head_dim, max_batch, max_pages_per_seq,
+                 layer_num_pages=None, device=None, softmax_scale=0.0, tune_warps=0, tune_stages=0,
+                 tune_ctas_per_sm=0):
+        import torch
+
+        dev = pools[0].device if device is None else torch.device(device)
+        if dev.type != "cuda":
+            raise RuntimeError("the attention stage runs on a CUDA device only")
+        self.device = dev
+        self.pools = list(pools)
+        page_elems = num_kv_heads * 2 * 16 * head_dim
+        if layer_num_pages is None:
+            layer_num_pages = [p.numel() // page_elems for p in pools]
+        kw = dict(device=dev.index or 0, num_q_heads=num_q_heads, num_kv_heads=num_kv_heads, head_dim=head_dim,
+                  max_batch=max_batch, max_pages_per_seq=max_pages_per_seq, layer_window=layer_window,
+                  layer_num_pages=layer_num_pages, layer_kv_pool=[p.data_ptr() for p in pools],
+                  softmax_scale=softmax_scale, tune_warps=tune_warps, tune_stages=tune_stages,
+                  tune_ctas_per_sm=tune_ctas_per_sm)
+        cfg, _keep = make_config(**kw)
+        nbytes = opw_attn_stage_workspace_bytes(cfg)
+        if nbytes == 0:
+            raise OpwError(OPW_ERR_INVALID_ARG, "opw_attn_stage_workspace_bytes")
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=dev)
+        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        cfg.workspace = base
+        cfg.workspace_bytes = nbytes
+        self.num_q_heads, self.num_kv_heads, self.head_dim = num_q_heads, num_kv_heads, head_dim
+        self.handle = opw_attn_stage_create(cfg)
+
+    @staticmethod
+    def _stream():
+        import torch
+
+        return torch.cuda.current_stream().cuda_stream
+
+    def kv_append(self, layer, k_new, v_new, positions, page_table):
+        opw_kv_append(self.handle, layer, positions.shape[0], k_new.data_ptr(), v_new.data_ptr(),
+                      positions.data_ptr(), page_table.data_ptr(), self._stream())
+
+    def decode_attention(self, layer, q, kv_lens, page_table, out, lse=None):
+        opw_decode_attention(self.handle, layer, kv_lens.shape[0], q.data_ptr(), kv_lens.data_ptr(),
+                             page_table.data_ptr(), out.data_ptr(), None if lse is None else lse.data_ptr(),
+                             self._stream())
+
+    def decode_step_host(self, layer, q, k_new, v_new, positions, page_table, out, lse=None):
+        opw_decode_step_host(self.handle, layer, positions.shape[0], q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(),
+                             positions.data_ptr(), None if page_table is None else page_table.data_ptr(),
+                             out.data_ptr(), None if lse is None else lse.data_ptr(), self._stream())
+
+    def poll_error(self) -> int:
+        return opw_attn_stage_poll_error(self.handle, self._stream())
+
+    def launch_count(self) -> int:
+        return opw_attn_stage_launch_count(self.handle)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            opw_attn_stage_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,365 @@
+// Host side of the C ABI declared in include/opw_attn.h: argument checks, workspace
+// carving, launches.  The library allocates no device memory and never synchronises
+// except in opw_attn_stage_poll_error and (once) in opw_attn_stage_create.
+#include "opw_attn.h"
+
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "opw_kernels.cuh"
+
+namespace {
+
+constexpr int kDefaultSMs = 148;
+constexpr int kDefaultWarps = 8;
+constexpr int kDefaultStages = 3;
+constexpr int kDefaultCtasPerSm = 1;
+constexpr size_t kSmemLimit = 227 * 1024;
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct Shape {
+  int warps, stages, ctas_per_sm;
+};
+
+struct Layout {          // byte offsets into the caller's workspace
+  size_t status, cum, partials, st_q, st_k, st_v, st_pos, st_lens, st_out, st_lse, st_table, total;
+};
+
+bool shape_ok(const opw_attn_stage_config_t* c) {
+  return c->num_layers >= 1 && c->num_q_heads >= 1 && c->num_kv_heads >= 1 && c->max_batch >= 1 &&
+         c->max_pages_per_seq >= 1 && c->num_q_heads % c->num_kv_heads == 0;
+}
+
+opw_status_t resolve_shape(const opw_attn_stage_config_t* c, Shape* s) {
+  s->warps = c->tune_warps ? c->tune_warps : kDefaultWarps;
+  s->stages = c->tune_stages ? c->tune_stages : kDefaultStages;
+  s->ctas_per_sm = c->tune_ctas_per_sm ? c->tune_ctas_per_sm : kDefaultCtasPerSm;
+  if (s->warps < 1 || s->warps > opw::kMaxWarps || s->stages < 2 || s->stages > 16 || s->ctas_per_sm < 1 ||
+      s->ctas_per_sm > 4)
+    return OPW_ERR_INVALID_ARG;
+  return OPW_OK;
+}
+
+size_t attn_smem_bytes(int D, const Shape& s, int batch) {
+  return D == 64 ? opw::AttnSmem<64>::bytes(s.warps, s.stages, batch) : opw::AttnSmem<128>::bytes(s.warps, s.stages, batch);
+}
+
+Layout carve(const opw_attn_stage_config_t* c, const Shape& s, int sms) {
+  Layout L;
+  const size_t B = c->max_batch, Hq = c->num_q_heads, Hkv = c->num_kv_heads, D = c->head_dim;
+  const size_t G = Hq / Hkv;
+  const size_t workers = (size_t)sms * s.ctas_per_sm * s.warps;
+  size_t off = 0;
+  L.status = off;  off += 256;
+  L.cum = off;     off += align_up((B + 2) * 4, 256);
+  L.partials = off; off += align_up(workers * 2 * G * (D + 2) * 4, 256);
+  L.st_q = off;    off += align_up(B * Hq * D * 2, 256);
+  L.st_k = off;    off += align_up(B * Hkv * D * 2, 256);
+  L.st_v = off;    off += align_up(B * Hkv * D * 2, 256);
+  L.st_pos = off;  off += align_up(B * 4, 256);
+  L.st_lens = off; off += align_up(B * 4, 256);
+  L.st_out = off;  off += align_up(B * Hq * D * 2, 256);
+  L.st_lse = off;  off += align_up(B * Hq * 4, 256);
+  L.st_table = off; off += align_up((size_t)c->num_layers * B * c->max_pages_per_seq * 4, 256);
+  L.total = off;
+  return L;
+}
+
+int query_sms(int device) {
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms <= 0) {
+    (void)cudaGetLastError();
+    return kDefaultSMs;
+  }
+  return sms;
+}
+
+}  // namespace
+
+struct opw_attn_stage {
+  opw_attn_stage_config_t cfg;
+  std::vector<int32_t> window;
+  std::vector<int64_t> num_pages;
+  std::vector<void*> pool;
+  Shape shape;
+  Layout lay;
+  int sms;
+  int grid;
+  size_t smem;
+  float scale_log2e;
+  int64_t launches;
+  unsigned char* ws;
+};
+
+extern "C" {
+
+const char* opw_status_string(opw_status_t s) {
+  switch (s) {
+    case OPW_OK: return "ok";
+    case OPW_ERR_INVALID_ARG: return "invalid argument";
+    case OPW_ERR_UNSUPPORTED: return "unsupported configuration";
+    case OPW_ERR_CAPACITY: return "capacity exceeded";
+    case OPW_ERR_CUDA: return "CUDA error";
+    case OPW_ERR_BAD_PAGE: return "page id or position out of range (device)";
+    case OPW_ERR_TIMEOUT: return "bounded device wait ran out";
+  }
+  return "unknown status";
+}
+
+int64_t opw_kv_pool_index(int64_t Hkv, int64_t P, int64_t D, int64_t page, int64_t g, int64_t kv, int64_t t,
+                          int64_t d) {
+  const int64_t tile = (page * Hkv + g) * 2 + kv;
+  return (tile * P + t) * D + ((((d >> 3) ^ (t & 7)) << 3) | (d & 7));
+}
+
+size_t opw_kv_pool_bytes(int32_t Hkv, int32_t P, int32_t D, int64_t num_pages) {
+  if (Hkv < 1 || P < 1 || D < 1 || num_pages < 0) return 0;
+  return (size_t)num_pages * Hkv * 2 * P * D * 2;
+}
+
+size_t opw_attn_stage_workspace_bytes(const opw_attn_stage_config_t* cfg) {
+  if (!cfg || cfg->struct_size != sizeof(opw_attn_stage_config_t) || !shape_ok(cfg)) return 0;
+  Shape s;
+  if (resolve_shape(cfg, &s) != OPW_OK) return 0;
+  return carve(cfg, s, query_sms(cfg->device)).total;
+}
+
+opw_status_t opw_attn_stage_create(const opw_attn_stage_config_t* cfg, opw_attn_stage_t** out) {
+  if (!cfg || !out) return OPW_ERR_INVALID_ARG;
+  if (cfg->struct_size != sizeof(opw_attn_stage_config_t) || cfg->reserved != 0) return OPW_ERR_INVALID_ARG;
+  if (!shape_ok(cfg) || cfg->device < 0) return OPW_ERR_INVALID_ARG;
+  if (!cfg->layer_window || !cfg->layer_num_pages || !cfg->layer_kv_pool || !cfg->workspace) return OPW_ERR_INVALID_ARG;
+  if (cfg->head_dim != 64 && cfg->head_dim != 128) return OPW_ERR_UNSUPPORTED;
+  if (cfg->page_size != opw::kPage) return OPW_ERR_UNSUPPORTED;
+  const int G = cfg->num_q_heads / cfg->num_kv_heads;
+  if (G > 16) return OPW_ERR_UNSUPPORTED;
+  if (cfg->max_batch > 32768) return OPW_ERR_UNSUPPORTED;
+  if ((int64_t)cfg->max_pages_per_seq * opw::kPage > INT32_MAX) return OPW_ERR_UNSUPPORTED;
+  if (!(cfg->softmax_scale >= 0.f) || !std::isfinite(cfg->softmax_scale)) return OPW_ERR_INVALID_ARG;
+  Shape s;
+  if (resolve_shape(cfg, &s) != OPW_OK) return OPW_ERR_INVALID_ARG;
+  if ((uintptr_t)cfg->workspace % 256) return OPW_ERR_INVALID_ARG;
+  for (int l = 0; l < cfg->num_layers; ++l) {
+    if (cfg->layer_window[l] < 0 || cfg->layer_num_pages[l] < 1) return OPW_ERR_INVALID_ARG;
+    if (!cfg->layer_kv_pool[l] || (uintptr_t)cfg->layer_kv_pool[l] % 128) return OPW_ERR_INVALID_ARG;
+    if (cfg->layer_num_pages[l] * (int64_t)cfg->num_kv_heads > INT32_MAX) return OPW_ERR_UNSUPPORTED;
+  }
+  const size_t smem = attn_smem_bytes(cfg->head_dim, s, cfg->max_batch);
+  if ((smem + 1024) * s.ctas_per_sm > kSmemLimit + 1024) return OPW_ERR_CAPACITY;   // ring does not fit an SM
+
+  // ---- CUDA from here on ----
+  if (cudaSetDevice(cfg->device) != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess || sms <= 0) {
+    (void)cudaGetLastError();
+    return OPW_ERR_CUDA;
+  }
+  const Layout lay = carve(cfg, s, sms);
+  if (cfg->workspace_bytes < lay.total) return OPW_ERR_CAPACITY;
+
+  cudaError_t e = cudaSuccess;
+  const int smem_i = (int)smem;
+  if (cfg->head_dim == 64) {
+    e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_i);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_i);
+  } else {
+    e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_i);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_i);
+  }
+  if (e != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
+  if (cudaMemset(cfg->workspace, 0, 256) != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
+  if (cudaDeviceSynchronize() != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
+
+  opw_attn_stage* st = new (std::nothrow) opw_attn_stage();
+  if (!st) return OPW_ERR_INVALID_ARG;
+  st->cfg = *cfg;
+  st->window.assign(cfg->layer_window, cfg->layer_window + cfg->num_layers);
+  st->num_pages.assign(cfg->layer_num_pages, cfg->layer_num_pages + cfg->num_layers);
+  st->pool.assign(cfg->layer_kv_pool, cfg->layer_kv_pool + cfg->num_layers);
+  st->cfg.layer_window = nullptr;
+  st->cfg.layer_num_pages = nullptr;
+  st->cfg.layer_kv_pool = nullptr;
+  st->shape = s;
+  st->lay = lay;
+  st->sms = sms;
+  st->grid = sms * s.ctas_per_sm;
+  st->smem = smem;
+  const double scale = cfg->softmax_scale > 0.f ? (double)cfg->softmax_scale : 1.0 / std::sqrt((double)cfg->head_dim);
+  st->scale_log2e = (float)(scale * 1.4426950408889634);
+  st->launches = 0;
+  st->ws = static_cast<unsigned char*>(cfg->workspace);
+  *out = st;
+  return OPW_OK;
+}
+
+opw_status_t opw_attn_stage_destroy(opw_attn_stage_t* st) {
+  delete st;
+  return OPW_OK;
+}
+
+int64_t opw_attn_stage_launch_count(const opw_attn_stage_t* st) { return st ? st->launches : 0; }
+
+static opw_status_t check_step(opw_attn_stage_t* st, int32_t layer, int32_t batch) {
+  if (!st) return OPW_ERR_INVALID_ARG;
+  if (layer < 0 || layer >= st->cfg.num_layers || batch < 0) return OPW_ERR_INVALID_ARG;
+  if (batch > st->cfg.max_batch) return OPW_ERR_CAPACITY;
+  return OPW_OK;
+}
+
+opw_status_t opw_kv_append(opw_attn_stage_t* st, int32_t layer, int32_t batch, const void* k_new, const void* v_new,
+                           const int32_t* positions, const int32_t* page_table, void* cuda_stream) {
+  opw_status_t rc = check_step(st, layer, batch);
+  if (rc != OPW_OK) return rc;
+  if (!k_new || !v_new || !positions || !page_table) return OPW_ERR_INVALID_ARG;
+  if (((uintptr_t)k_new | (uintptr_t)v_new) % 16 || (uintptr_t)positions % 4 || (uintptr_t)page_table % 4)
+    return OPW_ERR_INVALID_ARG;
+  if (batch == 0) return OPW_OK;
+  opw::AppendParams p;
+  p.pool = static_cast<__nv_bfloat16*>(st->pool[layer]);
+  p.k_new = static_cast<const __nv_bfloat16*>(k_new);
+  p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+  p.positions = positions;
+  p.page_table = page_table;
+  p.status = reinterpret_cast<uint32_t*>(st->ws + st->lay.status);
+  p.num_pages = st->num_pages[layer];
+  p.batch = batch;
+  p.Hkv = st->cfg.num_kv_heads;
+  p.D = st->cfg.head_dim;
+  p.max_pages = st->cfg.max_pages_per_seq;
+  const int groups = p.Hkv * 2 * (p.D / 8);
+  const int threads = groups < 256 ? ((groups + 31) / 32 * 32) : 256;
+  opw::kv_append_kernel<<<batch, threads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(p);
+  if (cudaGetLastError() != cudaSuccess) return OPW_ERR_CUDA;
+  st->launches += 1;
+  return OPW_OK;
+}
+
+opw_status_t opw_decode_attention(opw_attn_stage_t* st, int32_t layer, int32_t batch, const void* q,
+                                  const int32_t* kv_lens, const int32_t* page_table, void* out, float* lse,
+                                  void* cuda_stream) {
+  opw_status_t rc = check_step(st, layer, batch);
+  if (rc != OPW_OK) return rc;
+  if (!q || !kv_lens || !page_table || !out) return OPW_ERR_INVALID_ARG;
+  if (((uintptr_t)q | (uintptr_t)out) % 16 || (uintptr_t)kv_lens % 4 || (uintptr_t)page_table % 4 || (uintptr_t)lse % 4)
+    return OPW_ERR_INVALID_ARG;
+  if (batch == 0) return OPW_OK;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const int D = st->cfg.head_dim, Hq = st->cfg.num_q_heads, Hkv = st->cfg.num_kv_heads, G = Hq / Hkv;
+
+  opw::AttnParams p;
+  p.pool = static_cast<const __nv_bfloat16*>(st->pool[layer]);
+  p.q = static_cast<const __nv_bfloat16*>(q);
+  p.kv_lens = kv_lens;
+  p.page_table = page_table;
+  p.out = static_cast<__nv_bfloat16*>(out);
+  p.lse = lse;
+  p.partials = reinterpret_cast<float*>(st->ws + st->lay.partials);
+  p.cum = reinterpret_cast<int32_t*>(st->ws + st->lay.cum);
+  p.status = reinterpret_cast<uint32_t*>(st->ws + st->lay.status);
+  p.num_pages = st->num_pages[layer];
+  p.batch = batch;
+  p.Hq = Hq;
+  p.Hkv = Hkv;
+  p.G = G;
+  p.max_pages = st->cfg.max_pages_per_seq;
+  p.window = st->window[layer];
+  p.stages = st->shape.stages;
+  p.scale_log2e = st->scale_log2e;
+
+  const dim3 grid(st->grid), block(st->shape.warps * 32);
+  const size_t smem = attn_smem_bytes(D, st->shape, batch);
+  if (D == 64) {
+    if (G > 8) opw::attn_splitkv_kernel<64, true><<<grid, block, smem, stream>>>(p);
+    else opw::attn_splitkv_kernel<64, false><<<grid, block, smem, stream>>>(p);
+  } else {
+    if (G > 8) opw::attn_splitkv_kernel<128, true><<<grid, block, smem, stream>>>(p);
+    else opw::attn_splitkv_kernel<128, false><<<grid, block, smem, stream>>>(p);
+  }
+  if (cudaGetLastError() != cudaSuccess) return OPW_ERR_CUDA;
+  st->launches += 1;
+
+  opw::CombineParams c;
+  c.partials = p.partials;
+  c.cum = p.cum;
+  c.kv_lens = kv_lens;
+  c.out = p.out;
+  c.lse = lse;
+  c.batch = batch;
+  c.Hq = Hq;
+  c.Hkv = Hkv;
+  c.G = G;
+  c.D = D;
+  c.max_pages = p.max_pages;
+  c.window = p.window;
+  c.num_workers = st->grid * st->shape.warps;
+  opw::combine_kernel<<<batch * Hkv, 128, 0, stream>>>(c);
+  if (cudaGetLastError() != cudaSuccess) return OPW_ERR_CUDA;
+  st->launches += 1;
+  return OPW_OK;
+}
+
+opw_status_t opw_decode_step_host(opw_attn_stage_t* st, int32_t layer, int32_t batch, const void* q_host,
+                                  const void* k_new_host, const void* v_new_host, const int32_t* positions_host,
+                                  const int32_t* page_table_host, void* out_host, float* lse_host, void* cuda_stream) {
+  opw_status_t rc = check_step(st, layer, batch);
+  if (rc != OPW_OK) return rc;
+  if (!q_host || !k_new_host || !v_new_host || !positions_host || !out_host) return OPW_ERR_INVALID_ARG;
+  if (batch == 0) return OPW_OK;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const size_t B = batch, Hq = st->cfg.num_q_heads, Hkv = st->cfg.num_kv_heads, D = st->cfg.head_dim;
+  unsigned char* ws = st->ws;
+  void* d_q = ws + st->lay.st_q;
+  void* d_k = ws + st->lay.st_k;
+  void* d_v = ws + st->lay.st_v;
+  int32_t* d_pos = reinterpret_cast<int32_t*>(ws + st->lay.st_pos);
+  int32_t* d_lens = reinterpret_cast<int32_t*>(ws + st->lay.st_lens);
+  void* d_out = ws + st->lay.st_out;
+  float* d_lse = reinterpret_cast<float*>(ws + st->lay.st_lse);
+  const size_t table_elems = (size_t)st->cfg.max_batch * st->cfg.max_pages_per_seq;
+  int32_t* d_table = reinterpret_cast<int32_t*>(ws + st->lay.st_table) + (size_t)layer * table_elems;
+
+  bool ok = true;
+  ok &= cudaMemcpyAsync(d_q, q_host, B * Hq * D * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  ok &= cudaMemcpyAsync(d_k, k_new_host, B * Hkv * D * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  ok &= cudaMemcpyAsync(d_v, v_new_host, B * Hkv * D * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  ok &= cudaMemcpyAsync(d_pos, positions_host, B * 4, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  if (page_table_host)
+    ok &= cudaMemcpyAsync(d_table, page_table_host, B * st->cfg.max_pages_per_seq * 4, cudaMemcpyHostToDevice,
+                          stream) == cudaSuccess;
+  if (!ok) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
+  // kv_lens = positions + 1 on the device (inactive rows become 0)
+  opw::lens_from_positions_kernel<<<(batch + 255) / 256, 256, 0, stream>>>(d_pos, d_lens, batch);
+  if (cudaGetLastError() != cudaSuccess) return OPW_ERR_CUDA;
+  st->launches += 1;
+  rc = opw_kv_append(st, layer, batch, d_k, d_v, d_pos, d_table, cuda_stream);
+  if (rc != OPW_OK) return rc;
+  rc = opw_decode_attention(st, layer, batch, d_q, d_lens, d_table, d_out, lse_host ? d_lse : nullptr, cuda_stream);
+  if (rc != OPW_OK) return rc;
+  ok &= cudaMemcpyAsync(out_host, d_out, B * Hq * D * 2, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+  if (lse_host) ok &= cudaMemcpyAsync(lse_host, d_lse, B * Hq * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+  if (!ok) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
+  return OPW_OK;
+}
+
+opw_status_t opw_attn_stage_poll_error(opw_attn_stage_t* st, void* cuda_stream) {
+  if (!st) return OPW_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  uint32_t word = 0;
+  uint32_t* d = reinterpret_cast<uint32_t*>(st->ws + st->lay.status);
+  if (cudaMemcpyAsync(&word, d, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaMemsetAsync(d, 0, 4, stream) != cudaSuccess || cudaStreamSynchronize(stream) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return OPW_ERR_CUDA;
+  }
+  if (word & opw::kErrBadPage) return OPW_ERR_BAD_PAGE;
+  if (word & opw::kErrTimeout) return OPW_ERR_TIMEOUT;
+  return OPW_OK;
+}
+
+}  // extern "C"

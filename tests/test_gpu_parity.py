@@ -1,0 +1,388 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the
+same seeded inputs.  Append and page indexing must be bit-exact; attention output must
+satisfy max |err| <= 1e-2 and mean |err| <= 1e-3 (bf16 in, fp32 accumulate, bf16 out),
+plus the tighter checks below (error relative to the output's rms, log-sum-exp)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import P, bits, make_case, rand_bits
+from paper_2609_14237_b200 import binding as B
+from paper_2609_14237_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+MAX_ABS, MEAN_ABS = 1e-2, 1e-3          # the stated tolerance
+REL_RMS = 2.0 ** -6                     # max |err| / rms(out): catches dropped chunks on long contexts
+LSE_TOL = 2e-3
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    B.build()
+    assert torch.cuda.is_available()
+
+
+def dev(a, dtype=None):
+    t = torch.from_numpy(np.ascontiguousarray(a))
+    if dtype is torch.bfloat16:
+        t = t.view(torch.int16).view(torch.bfloat16)
+    return t.cuda()
+
+
+def out_to_f64(t):
+    return oracle.bf16_bits_to_f64(t.cpu().view(torch.int16).numpy().view(np.uint16))
+
+
+def check_close(got, ref, lse_got=None, lse_ref=None, rows=None):
+    if rows is not None:
+        got, ref = got[rows], ref[rows]
+        if lse_got is not None:
+            lse_got, lse_ref = lse_got[rows], lse_ref[rows]
+    err = np.abs(got - ref)
+    rms = float(np.sqrt(np.mean(ref ** 2)))
+    assert np.isfinite(got).all()
+    assert err.max() <= MAX_ABS, err.max()
+    assert err.mean() <= MEAN_ABS, err.mean()
+    # per (sequence, head) relative check: error against that row's own rms (+ bf16 half-ulp slack)
+    row_rms = np.sqrt(np.mean(ref ** 2, axis=-1, keepdims=True))
+    assert (err <= REL_RMS * row_rms + 2.0 ** -8 * np.abs(ref) + 1e-6).all(), float((err / (row_rms + 1e-30)).max())
+    if lse_got is not None:
+        fin = np.isfinite(lse_ref)
+        assert (np.isneginf(lse_got) == np.isneginf(lse_ref)).all()
+        assert np.abs(lse_got[fin] - lse_ref[fin]).max() <= LSE_TOL
+    return float(err.max()), float(err.mean()), rms
+
+
+def gpu_attention(pool_np, tab, q_bits, lens, Hq, Hkv, D, window=0, scale=0.0, want_lse=True, **tune):
+    pool = dev(pool_np, torch.bfloat16)
+    st = B.Stage(pools=[pool], layer_window=[window], num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D,
+                 max_batch=len(lens), max_pages_per_seq=tab.shape[1], softmax_scale=scale, **tune)
+    q = dev(q_bits, torch.bfloat16)
+    kv = dev(np.asarray(lens, np.int32))
+    tb = dev(tab.astype(np.int32))
+    out = torch.full((len(lens), Hq, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((len(lens), Hq), float("nan"), dtype=torch.float32, device="cuda") if want_lse else None
+    st.decode_attention(0, q, kv, tb, out, lse)
+    rc = st.poll_error()
+    launches = st.launch_count()
+    st.close()
+    return out, (lse.cpu().numpy().astype(np.float64) if want_lse else None), rc, launches
+
+
+# ------------------------------------------------------------------ append ---
+
+def test_append_is_bit_exact_over_the_whole_pool():
+    rng = np.random.default_rng(31)
+    Hkv, D = 2, 64
+    lens = [0, 15, 16, 255, 100, 17, 64]
+    pool_np, tab, _, _, _ = make_case(rng, [n + 1 for n in lens], 8, Hkv, D)
+    k_new, v_new = rand_bits(rng, (len(lens), Hkv, D)), rand_bits(rng, (len(lens), Hkv, D))
+    pos = np.array(lens, np.int32)
+    pos[5] = -1                                                        # an inactive slot
+    pool = dev(pool_np, torch.bfloat16)
+    st = B.Stage(pools=[pool], layer_window=[0], num_q_heads=8, num_kv_heads=Hkv, head_dim=D,
+                 max_batch=len(lens), max_pages_per_seq=tab.shape[1])
+    st.kv_append(0, dev(k_new, torch.bfloat16), dev(v_new, torch.bfloat16), dev(pos), dev(tab))
+    assert st.poll_error() == B.OPW_OK and st.launch_count() == 1
+    ref = pool_np.copy()
+    assert oracle.kv_append(ref, Hkv, D, P, k_new, v_new, pos, tab) == 0
+    got = pool.cpu().view(torch.int16).numpy().view(np.uint16)
+    assert (got == ref).all()
+    assert (got != pool_np).sum() > 0
+    st.close()
+
+
+def test_append_reports_bad_pages_without_writing():
+    rng = np.random.default_rng(32)
+    Hkv, D = 8, 128
+    pool_np, tab, _, _, _ = make_case(rng, [20, 20, 20], 32, Hkv, D)
+    bad = tab.copy()
+    bad[0, 1] = -1
+    bad[1, 1] = 1 << 20
+    k_new, v_new = rand_bits(rng, (3, Hkv, D)), rand_bits(rng, (3, Hkv, D))
+    pool = dev(pool_np, torch.bfloat16)
+    st = B.Stage(pools=[pool], layer_window=[0], num_q_heads=32, num_kv_heads=Hkv, head_dim=D, max_batch=3,
+                 max_pages_per_seq=tab.shape[1])
+    st.kv_append(0, dev(k_new, torch.bfloat16), dev(v_new, torch.bfloat16), dev(np.array([19, 19, 19], np.int32)), dev(bad))
+    assert st.poll_error() == B.OPW_ERR_BAD_PAGE
+    assert st.poll_error() == B.OPW_OK                                   # cleared by the poll
+    ref = pool_np.copy()
+    oracle.kv_append(ref, Hkv, D, P, k_new, v_new, np.array([-1, -1, 19], np.int32), tab)
+    assert (pool.cpu().view(torch.int16).numpy().view(np.uint16) == ref).all()
+    st.close()
+
+
+# --------------------------------------------------------------- attention ---
+
+@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 64), (32, 8, 128), (8, 8, 64), (64, 8, 128), (16, 1, 128), (24, 2, 64), (5, 1, 64)])
+@pytest.mark.parametrize("window", [0, 40])
+def test_attention_small_shapes_match_the_oracle(Hq, Hkv, D, window):
+    rng = np.random.default_rng(40 + Hq + D)
+    lens = [1, 2, 15, 16, 17, 33, 100, 256, 777]
+    pool, tab, q, _, _ = make_case(rng, lens, Hq, Hkv, D)
+    ref, ref_lse, rc = oracle.decode_attention(pool, Hq, Hkv, D, P, q, lens, tab, window=window)
+    assert rc == 0
+    out, lse, rc, launches = gpu_attention(pool, tab, q, lens, Hq, Hkv, D, window=window)
+    assert rc == B.OPW_OK and launches == 2
+    check_close(out_to_f64(out), ref, lse, ref_lse)
+
+
+def test_config1_tiny_step_append_then_attention():
+    wl = synth.WORKLOADS["c1_tiny"]
+    inp = synth.make_inputs(wl, device="cpu", growth=3, steps=3)
+    pool_ref = oracle.as_u16(inp.pools[0]).copy()
+    pool = inp.pools[0].cuda()
+    st = B.Stage(pools=[pool], layer_window=[0], num_q_heads=wl.num_q_heads, num_kv_heads=wl.num_kv_heads,
+                 head_dim=wl.head_dim, max_batch=wl.batch, max_pages_per_seq=inp.max_pages_per_seq)
+    tab = inp.page_tables[0]
+    for step in range(3):
+        pos, n = inp.positions(step), inp.kv_lens(step)
+        q, k, v = inp.q[step, 0], inp.k_new[step, 0], inp.v_new[step, 0]
+        out = torch.empty(wl.batch, wl.num_q_heads, wl.head_dim, dtype=torch.bfloat16, device="cuda")
+        lse = torch.empty(wl.batch, wl.num_q_heads, dtype=torch.float32, device="cuda")
+        st.kv_append(0, k.cuda(), v.cuda(), dev(pos), tab.cuda())
+        st.decode_attention(0, q.cuda(), dev(n), tab.cuda(), out, lse)
+        assert st.poll_error() == B.OPW_OK
+        assert oracle.kv_append(pool_ref, wl.num_kv_heads, wl.head_dim, P, k, v, pos, tab) == 0
+        assert (pool.cpu().view(torch.int16).numpy().view(np.uint16) == pool_ref).all()     # bit-exact cache
+        ref, ref_lse, _ = oracle.decode_attention(pool_ref, wl.num_q_heads, wl.num_kv_heads, wl.head_dim, P, q, n, tab)
+        check_close(out_to_f64(out), ref, lse.cpu().numpy().astype(np.float64), ref_lse)
+    st.close()
+
+
+def test_single_key_returns_v_bit_exactly():
+    rng = np.random.default_rng(51)
+    Hq, Hkv, D = 8, 2, 64
+    pool, tab, q, ks, vs = make_case(rng, [1, 1, 1], Hq, Hkv, D)
+    out, lse, rc, _ = gpu_attention(pool, tab, q, [1, 1, 1], Hq, Hkv, D)
+    got = out.cpu().view(torch.int16).numpy().view(np.uint16)
+    for b in range(3):
+        for h in range(Hq):
+            assert (got[b, h] == vs[b][0, h // 4]).all()
+
+
+def test_q_zero_probes_every_key_counted_once_long_and_windowed():
+    rng = np.random.default_rng(52)
+    Hq, Hkv, D = 8, 2, 64
+    lens = [1, 16, 17, 4000, 9000, 33000]
+    one = bits(np.float32(1.0))
+    for window in (0, 1, 17, 4096):
+        pool, tab, q, ks, vs = make_case(rng, lens, Hq, Hkv, D)
+        q[:] = 0
+        marks = [0, 15, 16, 3999, 8999, 20000]
+        for b, n in enumerate(lens):
+            lo = max(0, n - window) if window else 0
+            v = np.zeros((n, Hkv, D), np.uint16)
+            v[:, :, 0] = one
+            for c, j0 in enumerate(marks):
+                if j0 < n:
+                    v[j0, :, 1 + c] = one
+            v[:lo, :, 10] = one
+            oracle.scatter_logical(pool, Hkv, P, D, tab[b], ks[b], v)
+        out, lse, rc, _ = gpu_attention(pool, tab, q, lens, Hq, Hkv, D, window=window)
+        got = out_to_f64(out)
+        for b, n in enumerate(lens):
+            lo = max(0, n - window) if window else 0
+            n_eff = n - lo
+            np.testing.assert_allclose(got[b, :, 0], 1.0, rtol=2 ** -7)
+            for c, j0 in enumerate(marks):
+                want = 1.0 / n_eff if lo <= j0 < n else 0.0
+                np.testing.assert_allclose(got[b, :, 1 + c], want, rtol=2 ** -7, atol=0)
+            assert (got[b, :, 10] == 0).all()
+            np.testing.assert_allclose(lse[b], np.log(n_eff), atol=1e-4)
+
+
+def test_page_permutation_is_bitwise_invisible():
+    rng = np.random.default_rng(53)
+    Hq, Hkv, D = 32, 8, 128
+    lens = [100, 2000, 5000, 257]
+    pool, tab, q, _, _ = make_case(rng, lens, Hq, Hkv, D)
+    out1, lse1, _, _ = gpu_attention(pool, tab, q, lens, Hq, Hkv, D)
+    total = pool.size // (Hkv * 2 * P * D)
+    perm = rng.permutation(total)
+    pe = Hkv * 2 * P * D
+    pool2 = np.empty_like(pool)
+    pool2.reshape(total, pe)[perm] = pool.reshape(total, pe)
+    tab2 = np.where(tab >= 0, perm[np.maximum(tab, 0)], -1).astype(np.int32)
+    out2, lse2, _, _ = gpu_attention(pool2, tab2, q, lens, Hq, Hkv, D)
+    assert torch.equal(out1.view(torch.int16), out2.view(torch.int16))
+    assert (lse1 == lse2).all()
+
+
+def test_window_poisoned_entries_and_inactive_rows():
+    rng = np.random.default_rng(54)
+    Hq, Hkv, D = 32, 8, 128
+    lens = [18, 650, 1010, 2560]
+    W = 400
+    pool, tab, q, _, _ = make_case(rng, lens, Hq, Hkv, D)
+    ref, ref_lse, _ = oracle.decode_attention(pool, Hq, Hkv, D, P, q, lens, tab, window=W)
+    poisoned = tab.copy()
+    for b, n in enumerate(lens):
+        poisoned[b, :max(0, n - W) // P] = -1
+        poisoned[b, (n + P - 1) // P:] = -1
+    out, lse, rc, _ = gpu_attention(pool, poisoned, q, lens, Hq, Hkv, D, window=W)
+    assert rc == B.OPW_OK
+    check_close(out_to_f64(out), ref, lse, ref_lse)
+    # inactive rows: zeros and -inf
+    lens2 = [18, 0, 1010, -5]
+    ref2, ref_lse2, _ = oracle.decode_attention(pool, Hq, Hkv, D, P, q, lens2, tab)
+    out2, lse2, rc2, _ = gpu_attention(pool, tab, q, lens2, Hq, Hkv, D)
+    assert rc2 == B.OPW_OK
+    check_close(out_to_f64(out2), ref2, lse2, ref_lse2)
+    assert (out_to_f64(out2)[1] == 0).all() and np.isneginf(lse2[3]).all()
+
+
+def test_bad_page_ids_are_masked_and_reported_not_dereferenced():
+    rng = np.random.default_rng(55)
+    Hq, Hkv, D = 8, 2, 64
+    lens = [100, 200]
+    pool, tab, q, ks, vs = make_case(rng, lens, Hq, Hkv, D)
+    bad = tab.copy()
+    bad[1, 3] = -1
+    bad[1, 7] = 1 << 24
+    out, lse, rc, _ = gpu_attention(pool, bad, q, lens, Hq, Hkv, D)
+    assert rc == B.OPW_ERR_BAD_PAGE
+    # row 0 is unaffected; row 1 equals attention with the two bad pages' keys removed
+    ref, _, _ = oracle.decode_attention(pool, Hq, Hkv, D, P, q, lens, tab)
+    got = out_to_f64(out)
+    assert np.abs(got[0] - ref[0]).max() <= MAX_ABS
+    keep = [j for j in range(200) if j // P not in (3, 7)]
+    pool2, tab2, _, _, _ = make_case(rng, [len(keep)], Hq, Hkv, D)
+    oracle.scatter_logical(pool2, Hkv, P, D, tab2[0], ks[1][keep], vs[1][keep])
+    ref1, _, _ = oracle.decode_attention(pool2, Hq, Hkv, D, P, q[1:2], [len(keep)], tab2)
+    assert np.abs(got[1] - ref1[0]).max() <= MAX_ABS
+
+
+@pytest.mark.parametrize("tune", [dict(tune_warps=1, tune_stages=2), dict(tune_warps=4, tune_stages=6),
+                                  dict(tune_warps=4, tune_stages=3, tune_ctas_per_sm=2), dict(tune_warps=8, tune_stages=3),
+                                  dict(tune_warps=3, tune_stages=8)])
+def test_result_does_not_depend_on_the_split(tune):
+    """The log-sum-exp merge is exact in real arithmetic: any split agrees within rounding."""
+    rng = np.random.default_rng(56)
+    Hq, Hkv, D = 32, 8, 128
+    lens = [5000, 33, 12000, 1]
+    pool, tab, q, _, _ = make_case(rng, lens, Hq, Hkv, D)
+    ref, ref_lse, _ = oracle.decode_attention(pool, Hq, Hkv, D, P, q, lens, tab)
+    out, lse, rc, _ = gpu_attention(pool, tab, q, lens, Hq, Hkv, D, **tune)
+    assert rc == B.OPW_OK
+    check_close(out_to_f64(out), ref, lse, ref_lse)
+
+
+def test_custom_scale_and_no_lse_buffer():
+    rng = np.random.default_rng(57)
+    Hq, Hkv, D = 16, 2, 128
+    lens = [300, 45]
+    pool, tab, q, _, _ = make_case(rng, lens, Hq, Hkv, D)
+    ref, _, _ = oracle.decode_attention(pool, Hq, Hkv, D, P, q, lens, tab, scale=0.25)
+    out, _, rc, _ = gpu_attention(pool, tab, q, lens, Hq, Hkv, D, scale=0.25, want_lse=False)
+    assert rc == B.OPW_OK
+    check_close(out_to_f64(out), ref)
+
+
+def test_host_buffer_step_matches_the_device_step():
+    wl = synth.Workload("h", 6, 32, 8, 128, [0, 64], "uniform_1024_4096", 77)
+    inp = synth.make_inputs(wl, device="cpu", growth=2, steps=2, lengths=np.array([5, 200, 1023, 64, 15, 4097], np.int32))
+    pools = [p.cuda() for p in inp.pools]
+    refs = [oracle.as_u16(p).copy() for p in inp.pools]
+    st = B.Stage(pools=pools, layer_window=wl.layer_window, num_q_heads=32, num_kv_heads=8, head_dim=128,
+                 max_batch=6, max_pages_per_seq=inp.max_pages_per_seq)
+    for step in range(2):
+        for layer in range(2):
+            q = inp.q[step, layer].pin_memory()
+            k = inp.k_new[step, layer].pin_memory()
+            v = inp.v_new[step, layer].pin_memory()
+            pos = torch.from_numpy(inp.positions(step)).pin_memory()
+            tab = inp.page_tables[layer].pin_memory()
+            out = torch.empty(6, 32, 128, dtype=torch.bfloat16).pin_memory()
+            lse = torch.empty(6, 32, dtype=torch.float32).pin_memory()
+            st.decode_step_host(layer, q, k, v, pos, tab if step == 0 else None, out, lse)
+            assert st.poll_error() == B.OPW_OK
+            assert oracle.kv_append(refs[layer], 8, 128, P, k, v, pos, tab) == 0
+            assert (pools[layer].cpu().view(torch.int16).numpy().view(np.uint16) == refs[layer]).all()
+            ref, ref_lse, _ = oracle.decode_attention(refs[layer], 32, 8, 128, P, q, inp.kv_lens(step), tab,
+                                                      window=wl.layer_window[layer])
+            check_close(out_to_f64(out), ref, lse.numpy().astype(np.float64), ref_lse)
+    assert st.launch_count() == 2 * 2 * 4
+    st.close()
+
+
+def test_step_calls_validate_arguments_on_the_host():
+    pool = torch.zeros(4 * 2 * 2 * 16 * 64, dtype=torch.bfloat16, device="cuda")
+    st = B.Stage(pools=[pool], layer_window=[0], num_q_heads=8, num_kv_heads=2, head_dim=64, max_batch=2, max_pages_per_seq=2)
+    L, h = B.lib(), st.handle
+    x = pool.data_ptr()
+    assert L.opw_kv_append(h, 1, 1, x, x, x, x, None) == B.OPW_ERR_INVALID_ARG          # layer out of range
+    assert L.opw_kv_append(h, 0, 3, x, x, x, x, None) == B.OPW_ERR_CAPACITY             # batch > max_batch
+    assert L.opw_kv_append(h, 0, 1, None, x, x, x, None) == B.OPW_ERR_INVALID_ARG
+    assert L.opw_kv_append(h, 0, 1, x + 2, x, x, x, None) == B.OPW_ERR_INVALID_ARG       # misaligned
+    assert L.opw_decode_attention(h, 0, 1, x, x, x, None, None, None) == B.OPW_ERR_INVALID_ARG
+    assert L.opw_decode_attention(h, 0, 0, x, x, x, x, None, None) == B.OPW_OK           # empty batch: nothing to do
+    assert st.launch_count() == 0
+    st.close()
+
+
+# ------------------------------------------------- full-size configurations ---
+
+def compact_rows(pool, table, rows, Hkv, D):
+    """Copy only the pages the sampled rows reference into a small pool (pure data movement)."""
+    pe = Hkv * 2 * P * D
+    pv = pool.view(-1, pe)
+    sub = table[rows].clone()
+    used = torch.unique(sub[sub >= 0])
+    remap = torch.full((pv.shape[0],), -1, dtype=torch.int32, device=pool.device)
+    remap[used.long()] = torch.arange(used.numel(), dtype=torch.int32, device=pool.device)
+    small = pv[used.long()].contiguous().view(-1)
+    new_tab = torch.where(sub >= 0, remap[sub.clamp(min=0).long()], torch.full_like(sub, -1))
+    return oracle.as_u16(small.cpu()), new_tab.cpu().numpy()
+
+
+def run_full_config(name, sample, layers=None, tune=None):
+    wl = synth.WORKLOADS[name]
+    inp = synth.make_inputs(wl, device="cuda", growth=1, steps=1)
+    st = B.Stage(pools=inp.pools, layer_window=wl.layer_window, num_q_heads=wl.num_q_heads, num_kv_heads=wl.num_kv_heads,
+                 head_dim=wl.head_dim, max_batch=wl.batch, max_pages_per_seq=inp.max_pages_per_seq, **(tune or {}))
+    pos, n = inp.positions(0), inp.kv_lens(0)
+    order = np.argsort(n)
+    rows = sorted(set([int(order[0]), int(order[-1])] + [int(r) for r in np.random.default_rng(wl.seed).choice(wl.batch, size=min(sample, wl.batch), replace=False)]))
+    stats = []
+    for layer in (layers if layers is not None else range(wl.num_layers)):
+        tab = inp.page_tables[layer]
+        q, k, v = inp.q[0, layer], inp.k_new[0, layer], inp.v_new[0, layer]
+        small_before, small_tab = compact_rows(inp.pools[layer], tab, rows, wl.num_kv_heads, wl.head_dim)
+        out = torch.empty(wl.batch, wl.num_q_heads, wl.head_dim, dtype=torch.bfloat16, device="cuda")
+        lse = torch.empty(wl.batch, wl.num_q_heads, dtype=torch.float32, device="cuda")
+        st.kv_append(layer, k, v, dev(pos), tab)
+        st.decode_attention(layer, q, dev(n), tab, out, lse)
+        assert st.poll_error() == B.OPW_OK
+        # append parity on the sampled rows' pages (bit-exact), then attention on the oracle's own pool
+        ref_pool = small_before.copy()
+        assert oracle.kv_append(ref_pool, wl.num_kv_heads, wl.head_dim, P, k[rows].cpu(), v[rows].cpu(), pos[rows], small_tab) == 0
+        small_after, _ = compact_rows(inp.pools[layer], tab, rows, wl.num_kv_heads, wl.head_dim)
+        assert (small_after == ref_pool).all()
+        ref, ref_lse, rc = oracle.decode_attention(ref_pool, wl.num_q_heads, wl.num_kv_heads, wl.head_dim, P, q[rows].cpu(),
+                                                   n[rows], small_tab, window=wl.layer_window[layer])
+        assert rc == 0
+        stats.append(check_close(out_to_f64(out[rows]), ref, lse[rows].cpu().numpy().astype(np.float64), ref_lse))
+    st.close()
+    return stats
+
+
+def test_config2_llama8b_shape_all_rows():
+    run_full_config("c2_llama8b", sample=64)
+
+
+def test_config3_long_context_sampled_rows():
+    run_full_config("c3_long_context", sample=3)
+
+
+def test_config4_large_batch_sampled_rows():
+    run_full_config("c4_large_batch", sample=12)
+
+
+def test_config5_hybrid_stack_sampled_rows_one_window_and_one_full_layer():
+    free, _ = torch.cuda.mem_get_info()
+    if free < 70 * (1 << 30):
+        pytest.skip("needs ~55 GB of device memory")
+    run_full_config("c5_hybrid_stack", sample=1, layers=[2, 3])
