@@ -1,0 +1,432 @@
+#!/usr/bin/env python
+"""Benchmark of the decode attention stage: KV GB/s and sequence-steps/s per layer.
+
+A "step" is one pass of the whole hot path over one batch: for every layer the stage
+owns, the paged KV append of this step's token followed by split-KV attention and the
+log-sum-exp combine.  The headline ``value`` is algorithmic KV bytes (the K and V rows the
+step must read: sum over sequences of visible tokens x 2*Hkv*D*2 bytes) divided by the
+step time, with all inputs resident in HBM.  ``e2e`` is the same metric through
+``opw_decode_step_host`` with pinned HOST buffers: the per-step copies of q, k_new,
+v_new, positions and the page table to the device and of the output back are inside the
+timed region and every step ends with a stream synchronisation.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+For N > 1 launch with torchrun (one rank per GPU); every rank runs an independent replica
+of the workload (the stage shards by sequence with no exchange), the time is the max over
+ranks and the value the sum of all ranks' bytes over that time.
+"""
+from __future__ import annotations
+
+import argparse
+import dataclasses
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode attn-stage KV GB/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+DEFAULT_WORKLOAD = "c3_long_context"
+# DRAM traffic of the split-KV kernel relative to its algorithmic KV bytes, from the ncu
+# captures summarised under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum per
+# launch / algorithmic bytes).  None = not captured yet.
+TRAFFIC_RATIO = {}
+
+
+def measured_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, torch_index: int, period: float = 0.02):
+        super().__init__(daemon=True)
+        self.period, self.samples, self.reasons, self.stop_flag = period, [], set(), False
+        self.max_mhz, self.ok = None, False
+        try:
+            import pynvml
+            import torch
+
+            pynvml.nvmlInit()
+            uuid = str(torch.cuda.get_device_properties(torch_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode() if hasattr(uuid, "encode") else uuid)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception as e:                                   # noqa: BLE001
+            self.err = repr(e)
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self.stop_flag:
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                try:
+                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                except Exception:                                # noqa: BLE001
+                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:                                    # noqa: BLE001
+                pass
+            time.sleep(self.period)
+
+    def result(self):
+        self.stop_flag = True
+        if self.is_alive():
+            self.join(timeout=2)
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": int(np.median(self.samples)), "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def build_stage(wl, rotate, total_rounds, device, tune):
+    """R identical copies of a one-layer workload (or the workload's own layer stack)."""
+    import torch
+
+    from paper_2609_14237_b200 import binding, synth
+
+    if wl.num_layers == 1 and rotate > 1:
+        wl_r = dataclasses.replace(wl, layer_window=list(wl.layer_window) * rotate)
+    else:
+        wl_r = wl
+    inp = synth.make_inputs(wl_r, device=device, growth=total_rounds + 1, steps=2)
+    st = binding.Stage(pools=inp.pools, layer_window=wl_r.layer_window, num_q_heads=wl.num_q_heads,
+                       num_kv_heads=wl.num_kv_heads, head_dim=wl.head_dim, max_batch=wl.batch,
+                       max_pages_per_seq=inp.max_pages_per_seq, **tune)
+    rounds = total_rounds + 1
+    pos_all = torch.from_numpy(np.stack([inp.positions(t) for t in range(rounds)])).to(device)
+    len_all = torch.from_numpy(np.stack([inp.kv_lens(t) for t in range(rounds)])).to(device)
+    return wl_r, inp, st, pos_all, len_all
+
+
+def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, world=1, rank=0):
+    import torch
+
+    from paper_2609_14237_b200 import binding, synth
+
+    dev = torch.device("cuda", torch.cuda.current_device())
+    wl = synth.WORKLOADS[name]
+    stack = wl.num_layers > 1                       # the hybrid stack: a step runs all its layers
+    R = wl.num_layers if stack else rotate
+    e2e_steps = max(3, min(steps, 200)) if want_e2e else 0
+    n_timed = warmup + steps + (e2e_steps + 3 if want_e2e else 0)
+    rounds = n_timed if stack else (n_timed + R - 1) // R
+    wl_r, inp, st, pos_all, len_all = build_stage(wl, R, rounds, dev, tune)
+    B, Hq, Hkv, D = wl.batch, wl.num_q_heads, wl.num_kv_heads, wl.head_dim
+    out = torch.empty(B, Hq, D, dtype=torch.bfloat16, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def layer_round(s):                             # which layers step s runs, and at which length
+        return (list(range(R)), s) if stack else ([s % R], s // R)
+
+    def kv_bytes_of_step(s):
+        layers, t = layer_round(s)
+        return sum(inp.kv_bytes(l, t) for l in layers)
+
+    def device_step(s, events=None):
+        layers, t = layer_round(s)
+        for l in layers:
+            st.kv_append(l, inp.k_new[s & 1, l], inp.v_new[s & 1, l], pos_all[t], inp.page_tables[l])
+            if events is not None:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+            st.decode_attention(l, inp.q[s & 1, l], len_all[t], inp.page_tables[l], out)
+            if events is not None:
+                e1.record(stream)
+                events.append((e0, e1))
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+
+            dist.barrier()
+
+    for s in range(warmup):
+        device_step(s)
+    torch.cuda.synchronize()
+    assert st.poll_error() == binding.OPW_OK
+    barrier()
+    sampler = ClockSampler(dev.index)
+    sampler.start()
+    launches0 = st.launch_count()
+    ev = []
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    t0.record(stream)
+    for s in range(warmup, warmup + steps):
+        device_step(s, ev)
+    t1.record(stream)
+    torch.cuda.synchronize()
+    barrier()
+    clocks = sampler.result()
+    launches = st.launch_count() - launches0
+    total_ms = t0.elapsed_time(t1)
+    attn_ms = [a.elapsed_time(b) for a, b in ev]
+    assert st.poll_error() == binding.OPW_OK
+    bytes_timed = sum(kv_bytes_of_step(s) for s in range(warmup, warmup + steps))
+    layers_per_step = len(layer_round(0)[0])
+    attn_bytes_per_launch = bytes_timed / (steps * layers_per_step)
+
+    if world > 1:
+        import torch.distributed as dist
+
+        tmax = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        total_ms = float(tmax.item())
+    value = world * bytes_timed / (total_ms * 1e-3) / 1e9
+    peak, peak_kind = measured_peak()
+    attn_avg_ms = float(np.mean(attn_ms))
+    achieved = attn_bytes_per_launch / (attn_avg_ms * 1e-3) / 1e9
+    ratio = TRAFFIC_RATIO.get(name)
+    res = {
+        "metric": METRIC, "value": round(value, 1), "unit": "GB/s", "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": round(total_ms / steps, 5), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": name, "batch": B, "num_q_heads": Hq, "num_kv_heads": Hkv, "head_dim": D, "page_size": 16,
+                   "layers_per_step": layers_per_step, "layer_window": list(wl.layer_window),
+                   "mean_context": float(np.mean(inp.lengths)),
+                   "kv_bytes_per_step": int(bytes_timed // steps),
+                   "l2": (f"inputs larger than L2: {'the stack of' if stack else 'rotating over'} {R} layer pools, "
+                          f"{sum(inp.kv_bytes(l, 0) for l in range(R)) / 1e9:.2f} GB of KV between re-reads"),
+                   "parallelism": f"replicas x{world}" if world > 1 else "1 gpu"},
+        "seq_steps_per_s_per_layer": round(world * B * layers_per_step / (total_ms / steps * 1e-3), 1),
+        "pct_of_nominal_8000": round(100 * value / world / NOMINAL_HBM_GBS, 2),
+        "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
+                     "frac": round(achieved / peak, 4), "peak_kind": peak_kind,
+                     "kernel": "attn_splitkv_kernel (+ combine_kernel, timed together per opw_decode_attention call)",
+                     "kernel_ms": round(attn_avg_ms, 5),
+                     "traffic": None if ratio is None else int(ratio * attn_bytes_per_launch)},
+        "gpu_launches": int(launches), "clocks": clocks,
+    }
+
+    if want_e2e:
+        hq = [inp.q[i].cpu().pin_memory() for i in range(2)]
+        hk = [inp.k_new[i].cpu().pin_memory() for i in range(2)]
+        hv = [inp.v_new[i].cpu().pin_memory() for i in range(2)]
+        hpos = pos_all.cpu().pin_memory()
+        htab = [t.cpu().pin_memory() for t in inp.page_tables]
+        hout = torch.empty(B, Hq, D, dtype=torch.bfloat16).pin_memory()
+        base = warmup + steps
+
+        def host_step(s):
+            layers, t = layer_round(s)
+            for l in layers:
+                st.decode_step_host(l, hq[s & 1][l], hk[s & 1][l], hv[s & 1][l], hpos[t], htab[l], hout)
+            stream.synchronize()                     # the caller reads the result every step
+
+        for s in range(base, base + 3):
+            host_step(s)
+        barrier()
+        torch.cuda.synchronize()
+        w0 = time.perf_counter()
+        t0.record(stream)
+        for s in range(base + 3, base + 3 + e2e_steps):
+            host_step(s)
+        t1.record(stream)
+        torch.cuda.synchronize()
+        wall_ms = (time.perf_counter() - w0) * 1e3
+        e_ms = max(t0.elapsed_time(t1), wall_ms)
+        if world > 1:
+            import torch.distributed as dist
+
+            tmax = torch.tensor([e_ms], dtype=torch.float64, device=dev)
+            dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+            e_ms = float(tmax.item())
+        e_bytes = sum(kv_bytes_of_step(s) for s in range(base + 3, base + 3 + e2e_steps))
+        h2d = layers_per_step * (hq[0][0].numel() * 2 + 2 * hk[0][0].numel() * 2 + B * 4 + htab[0].numel() * 4)
+        d2h = layers_per_step * hout.numel() * 2
+        assert st.poll_error() == binding.OPW_OK
+        res["e2e"] = {"value": round(world * e_bytes / (e_ms * 1e-3) / 1e9, 1), "unit": "GB/s", "steps": e2e_steps,
+                      "ms_per_step": round(e_ms / e2e_steps, 5), "h2d_bytes_per_step": int(h2d),
+                      "d2h_bytes_per_step": int(d2h)}
+    if want_cpu:
+        res["cpu_baseline"] = cpu_baseline(name, inp, budget_s=15.0)
+    st.close()
+    del inp
+    torch.cuda.empty_cache()
+    return res
+
+
+def cpu_baseline(name, inp=None, budget_s=15.0, device="cpu"):
+    """The fp64 oracle as it stands, timed on this machine's host cores over a bounded sample of
+    the workload's sequences (layer 0, step 0); value in the metric's unit."""
+    import torch
+
+    import oracle
+    from paper_2609_14237_b200 import synth
+
+    wl = synth.WORKLOADS[name]
+    if inp is None:
+        inp = synth.make_inputs(dataclasses.replace(wl, layer_window=wl.layer_window[:1]), device=device, growth=1, steps=1)
+    Hq, Hkv, D, P = wl.num_q_heads, wl.num_kv_heads, wl.head_dim, 16
+    lens = inp.kv_lens(0)
+    window = inp.wl.layer_window[0]
+    order = np.argsort(-lens.astype(np.int64), kind="stable")          # longest first
+    pe = Hkv * 2 * P * D
+
+    def sample(rows):
+        tab = inp.page_tables[0][rows].cpu()
+        used = torch.unique(tab[tab >= 0])
+        remap = torch.full((inp.num_pages[0],), -1, dtype=torch.int32)
+        remap[used.long()] = torch.arange(used.numel(), dtype=torch.int32)
+        small = inp.pools[0].view(-1, pe)[used.to(inp.pools[0].device).long()].contiguous().view(-1).cpu()
+        new_tab = torch.where(tab >= 0, remap[tab.clamp(min=0).long()], torch.full_like(tab, -1)).numpy()
+        q = inp.q[0, 0][rows].cpu()
+        k, v = inp.k_new[0, 0][rows].cpu(), inp.v_new[0, 0][rows].cpu()
+        return oracle.as_u16(small).copy(), new_tab, q, k, v
+
+    def timed(rows):
+        pool, tab, q, k, v = sample(rows)
+        n = lens[rows]
+        t0 = time.perf_counter()
+        oracle.kv_append(pool, Hkv, D, P, k, v, (n - 1).astype(np.int32), tab)
+        oracle.decode_attention(pool, Hq, Hkv, D, P, q, n, tab, window=window)
+        dt = time.perf_counter() - t0
+        vis = np.minimum(n, window) if window > 0 else n
+        return dt, int(vis.astype(np.int64).sum()) * wl.kv_bytes_per_token
+
+    probe_rows = [int(order[len(order) // 2])]
+    dt, nbytes = timed(probe_rows)
+    rate = nbytes / max(dt, 1e-6)
+    rows, acc = [], 0
+    for r in order[::max(1, len(order) // 64)].tolist() + order.tolist():
+        if r in rows:
+            continue
+        vis = min(int(lens[r]), window) if window > 0 else int(lens[r])
+        if rows and (acc + vis * wl.kv_bytes_per_token) / rate > budget_s:
+            break
+        rows.append(int(r))
+        acc += vis * wl.kv_bytes_per_token
+    dt, nbytes = timed(sorted(rows))
+    return {"value": round(nbytes / dt / 1e9, 4), "unit": "GB/s", "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{len(rows)} of {len(lens)} sequences of {name}, layer 0, one append+attention step "
+                      f"({nbytes / 1e6:.1f} MB of KV in {dt:.2f} s)",
+            "seq_steps_per_s_per_layer": round(len(rows) / dt, 3)}
+
+
+def run_reference(name, steps, warmup):
+    """The reference arm: the CPU oracle, as it stands, on the host cores."""
+    import oracle
+    from paper_2609_14237_b200 import synth
+
+    wl = synth.WORKLOADS[name]
+    inp = synth.make_inputs(dataclasses.replace(wl, layer_window=wl.layer_window[:1]), device="cpu", growth=1, steps=1)
+    total = max(1, steps + warmup)
+    budget = min(20.0, 150.0 / total)
+    vals = []
+    for i in range(total):
+        r = cpu_baseline(name, inp, budget_s=budget)
+        if i >= warmup:
+            vals.append(r)
+    v = float(np.mean([r["value"] for r in vals]))
+    ms = float(np.mean([float(r["sample"].split(" in ")[1].split(" s")[0]) for r in vals])) * 1e3
+    return {"impl": "reference", "metric": METRIC, "value": round(v, 4), "unit": "GB/s", "n_gpus": 1, "steps": steps,
+            "warmup": warmup, "ms_per_step": round(ms, 2), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": name, "batch": wl.batch, "num_q_heads": wl.num_q_heads,
+                       "num_kv_heads": wl.num_kv_heads, "head_dim": wl.head_dim, "page_size": 16,
+                       "note": "each step is a bounded sample of the workload's sequences"},
+            "cpu_baseline": {"value": round(v, 4), "unit": "GB/s", "cores": oracle.num_threads(), "kind": "oracle",
+                             "sample": vals[-1]["sample"]},
+            "e2e": {"value": round(v, 4), "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--rotate", type=int, default=4, help="layer pools cycled through by a one-layer workload")
+    ap.add_argument("--others", default="c2_llama8b,c4_large_batch,c5_hybrid_stack",
+                    help="further workloads reported under 'other_workloads' (N=1 only; '' for none)")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--warps", type=int, default=0)
+    ap.add_argument("--stages", type=int, default=0)
+    ap.add_argument("--ctas", type=int, default=0)
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank == 0:
+            steps = args.steps if args.steps is not None else 3
+            warmup = args.warmup if args.warmup is not None else 1
+            print(json.dumps(run_reference(args.workload, steps, warmup)), flush=True)
+        return
+
+    import torch
+
+    from paper_2609_14237_b200 import binding
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the attention stage has no CPU path")
+    binding.build()
+    torch.cuda.set_device(local)
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    steps = args.steps if args.steps is not None else 2000
+    warmup = args.warmup if args.warmup is not None else 20
+    tune = dict(tune_warps=args.warps, tune_stages=args.stages, tune_ctas_per_sm=args.ctas)
+    res = run_ours(args.workload, steps, max(3, warmup), args.rotate, tune, want_e2e=True,
+                   want_cpu=(world == 1 and rank == 0 and not args.no_cpu), world=world, rank=rank)
+    if world == 1 and args.others:
+        others = {}
+        for name in args.others.split(","):
+            if not name or name == args.workload:
+                continue
+            if name == "c5_hybrid_stack":
+                if torch.cuda.mem_get_info()[0] < 70 * (1 << 30):
+                    others[name] = {"skipped": "needs ~55 GB of device memory"}
+                    continue
+                k = max(10, min(steps, 100))
+            else:
+                k = max(10, min(steps, 1000))
+            r = run_ours(name, k, max(3, min(warmup, 10)), args.rotate, tune, want_e2e=False)
+            others[name] = {key: r[key] for key in ("value", "unit", "ms_per_step", "seq_steps_per_s_per_layer",
+                                                    "pct_of_nominal_8000", "roofline", "steps")}
+            others[name]["kv_bytes_per_step"] = r["config"]["kv_bytes_per_step"]
+        res["other_workloads"] = others
+    if world > 1:
+        import torch.distributed as dist
+
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(res), flush=True)
+
+
+if __name__ == "__main__":
+    main()

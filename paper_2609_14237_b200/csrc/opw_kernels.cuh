@@ -376,6 +376,17 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
     if (!mbar_wait_bounded(bar_base + 8 * slot, phase)) { failed = true; break; }
 
     const uint32_t tile = ring_base + slot * TILE;
+    const bool ragged = (t0 > 0) || (t1 < kPage);
+    if (ragged) {
+      // Slots outside [t0,t1) may hold anything (never written, or stale): their scores are
+      // masked below, and their V rows are zeroed here so that 0 * garbage cannot make a NaN.
+      for (int t = 0; t < kPage; ++t) {
+        if (t >= t0 && t < t1) continue;
+        for (int off = lane * 16; off < ROWB; off += 512)
+          asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(tile + kPage * ROWB + t * ROWB + off), "r"(0u) : "memory");
+      }
+      __syncwarp();
+    }
     // ---- S = Q K^T for the 16 tokens of the page ----
     float s[2][4];
 #pragma unroll
@@ -388,7 +399,6 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
       mma_bf16(s[1], qa[ks][0], HI ? qa[ks][1] : 0u, qa[ks][2], HI ? qa[ks][3] : 0u, r2, r3);
     }
     // ---- online softmax (base 2) ----
-    const bool ragged = (t0 > 0) || (t1 < kPage);
     float x[2][4];
 #pragma unroll
     for (int nt = 0; nt < 2; ++nt)
@@ -557,24 +567,29 @@ __global__ void combine_kernel(CombineParams p) {
   const int64_t wf = worker_of(U, ustart, p.num_workers), wl = worker_of(U, uend - 1, p.num_workers);
   if (wf == wl) return;                       // the row was finished by a single worker
   const int64_t stride = (int64_t)p.G * (D + 2);
-  // slot of worker w for this row: 0 if the row is the first one w touches, else 1
-  auto slot_of = [&](int64_t w) -> const float* {
-    const bool is_first_row = (w > wf) || (worker_begin(U, w, p.num_workers) == ustart);
+  // Walk the row's segments: the worker holding unit u owns [u, min(end of its range, uend)).
+  // (Workers with an empty range hold no unit and are never visited.)  A worker's partial is
+  // in its slot 0 if the row is the first one it touches, else in slot 1.
+  auto slot_at = [&](int64_t u, int64_t& next_u) -> const float* {
+    const int64_t w = worker_of(U, u, p.num_workers);
+    const int64_t wb = worker_begin(U, w, p.num_workers);
+    next_u = worker_begin(U, w + 1, p.num_workers);
+    const bool is_first_row = wb >= ustart;
     return p.partials + (w * 2 + (is_first_row ? 0 : 1)) * stride;
   };
   for (int h = 0; h < p.G; ++h) {
     float M = -INFINITY;
-    for (int64_t w = wf; w <= wl; ++w) M = fmaxf(M, slot_of(w)[p.G * D + h]);
+    for (int64_t u = ustart, nu; u < uend; u = nu) M = fmaxf(M, slot_at(u, nu)[p.G * D + h]);
     float L = 0.f;
-    for (int64_t w = wf; w <= wl; ++w) {
-      const float* s = slot_of(w);
+    for (int64_t u = ustart, nu; u < uend; u = nu) {
+      const float* s = slot_at(u, nu);
       L += exp2f(s[p.G * D + h] - M) * s[p.G * D + p.G + h];
     }
     const float inv = L > 0.f ? 1.f / L : 0.f;
     for (int d = threadIdx.x; d < D; d += blockDim.x) {
       float acc = 0.f;
-      for (int64_t w = wf; w <= wl; ++w) {
-        const float* s = slot_of(w);
+      for (int64_t u = ustart, nu; u < uend; u = nu) {
+        const float* s = slot_at(u, nu);
         acc += exp2f(s[p.G * D + h] - M) * s[h * D + d];
       }
       ob[h * D + d] = __float2bfloat16_rn(acc * inv);

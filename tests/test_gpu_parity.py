@@ -163,6 +163,26 @@ def test_single_key_returns_v_bit_exactly():
             assert (got[b, h] == vs[b][0, h // 4]).all()
 
 
+def test_garbage_in_unwritten_slots_cannot_leak_into_the_result():
+    """Slots after the last key (and before the window) may hold NaN/Inf bit patterns."""
+    rng = np.random.default_rng(58)
+    Hq, Hkv, D = 32, 8, 128
+    lens = [1, 17, 100, 250]
+    W = 60
+    pool, tab, q, ks, vs = make_case(rng, lens, Hq, Hkv, D)
+    ref, ref_lse, _ = oracle.decode_attention(pool, Hq, Hkv, D, P, q, lens, tab, window=W)
+    poisoned = np.full_like(pool, 0x7FC0)                            # bf16 NaN everywhere
+    for b, n in enumerate(lens):
+        lo = max(0, n - W)
+        k = np.full((n, Hkv, D), 0x7F80, np.uint16)                  # +Inf before the window
+        v = np.full((n, Hkv, D), 0x7FC0, np.uint16)
+        k[lo:], v[lo:] = ks[b][lo:], vs[b][lo:]
+        oracle.scatter_logical(poisoned, Hkv, P, D, tab[b], k, v)
+    out, lse, rc, _ = gpu_attention(poisoned, tab, q, lens, Hq, Hkv, D, window=W)
+    assert rc == B.OPW_OK
+    check_close(out_to_f64(out), ref, lse, ref_lse)
+
+
 def test_q_zero_probes_every_key_counted_once_long_and_windowed():
     rng = np.random.default_rng(52)
     Hq, Hkv, D = 8, 2, 64
