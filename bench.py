@@ -370,6 +370,7 @@ def main():
     ap.add_argument("--others", default="c2_llama8b,c4_large_batch,c5_hybrid_stack",
                     help="further workloads reported under 'other_workloads' (N=1 only; '' for none)")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--warps", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--ctas", type=int, default=0)
@@ -400,7 +401,7 @@ def main():
     steps = args.steps if args.steps is not None else 2000
     warmup = args.warmup if args.warmup is not None else 20
     tune = dict(tune_warps=args.warps, tune_stages=args.stages, tune_ctas_per_sm=args.ctas)
-    res = run_ours(args.workload, steps, max(3, warmup), args.rotate, tune, want_e2e=True,
+    res = run_ours(args.workload, steps, max(3, warmup), args.rotate, tune, want_e2e=not args.no_e2e,
                    want_cpu=(world == 1 and rank == 0 and not args.no_cpu), world=world, rank=rank)
     if world == 1 and args.others:
         others = {}

@@ -173,6 +173,18 @@ opw_status_t opw_decode_step_host(opw_attn_stage_t *stage, int32_t layer, int32_
  */
 opw_status_t opw_attn_stage_poll_error(opw_attn_stage_t *stage, void *cuda_stream);
 
+/*
+ * Tracing hook (the stage's counterpart of the offline operator profiles that feed the
+ * paper's planner, Section 4 "profiled execution latency").  With a non-NULL DEVICE buffer
+ * of at least 32 * workers bytes (8-byte aligned; *num_workers, if not NULL, receives the
+ * worker count), every later opw_decode_attention launch makes each of its workers (one
+ * warp each) record four uint64: {SM id | units << 32, begin, first tile ready, end}, the
+ * times in nanoseconds of the device's global timer.  Workers with no work leave their
+ * record untouched.  trace == NULL switches tracing off.  The buffer is caller-owned.
+ */
+opw_status_t opw_attn_stage_set_trace(opw_attn_stage_t *stage, void *trace, size_t trace_bytes,
+                                      int32_t *num_workers);
+
 /* Kernels launched through this handle since create (the library's own count). */
 int64_t opw_attn_stage_launch_count(const opw_attn_stage_t *stage);
 

@@ -23,7 +23,7 @@ OPW_OK, OPW_ERR_INVALID_ARG, OPW_ERR_UNSUPPORTED, OPW_ERR_CAPACITY, OPW_ERR_CUDA
 EXPORTS = [
     "opw_kv_pool_index", "opw_kv_pool_bytes", "opw_attn_stage_workspace_bytes", "opw_attn_stage_create",
     "opw_kv_append", "opw_decode_attention", "opw_decode_step_host", "opw_attn_stage_poll_error",
-    "opw_attn_stage_launch_count", "opw_attn_stage_destroy", "opw_status_string",
+    "opw_attn_stage_launch_count", "opw_attn_stage_destroy", "opw_status_string", "opw_attn_stage_set_trace",
 ]
 
 
@@ -104,6 +104,8 @@ def lib() -> ctypes.CDLL:
     L.opw_decode_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     L.opw_attn_stage_poll_error.restype = ctypes.c_int
     L.opw_attn_stage_poll_error.argtypes = [vp, vp]
+    L.opw_attn_stage_set_trace.restype = ctypes.c_int
+    L.opw_attn_stage_set_trace.argtypes = [vp, vp, ctypes.c_size_t, ctypes.POINTER(i32)]
     L.opw_attn_stage_launch_count.restype = i64
     L.opw_attn_stage_launch_count.argtypes = [vp]
     L.opw_attn_stage_destroy.restype = ctypes.c_int
@@ -200,6 +202,13 @@ def opw_attn_stage_poll_error(stage: int, stream: Optional[int] = None) -> int:
     return int(lib().opw_attn_stage_poll_error(stage, stream))
 
 
+def opw_attn_stage_set_trace(stage: int, trace: Optional[int], trace_bytes: int = 0) -> int:
+    """Returns the worker count; raises OpwError if the buffer is too small or misaligned."""
+    n = ctypes.c_int32(0)
+    _check(lib().opw_attn_stage_set_trace(stage, trace, trace_bytes, ctypes.byref(n)), "opw_attn_stage_set_trace")
+    return int(n.value)
+
+
 def opw_attn_stage_launch_count(stage: int) -> int:
     return int(lib().opw_attn_stage_launch_count(stage))
 
@@ -263,6 +272,15 @@ class Stage:
         opw_decode_step_host(self.handle, layer, positions.shape[0], q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(),
                              positions.data_ptr(), None if page_table is None else page_table.data_ptr(),
                              out.data_ptr(), None if lse is None else lse.data_ptr(), self._stream())
+
+    def enable_trace(self):
+        """Allocate a trace buffer (torch) and switch per-worker tracing on; returns the int64 tensor [workers, 4]."""
+        import torch
+
+        n = opw_attn_stage_set_trace(self.handle, None)
+        self.trace = torch.zeros(n, 4, dtype=torch.int64, device=self.device)
+        opw_attn_stage_set_trace(self.handle, self.trace.data_ptr(), self.trace.numel() * 8)
+        return self.trace
 
     def poll_error(self) -> int:
         return opw_attn_stage_poll_error(self.handle, self._stream())

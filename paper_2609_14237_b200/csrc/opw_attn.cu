@@ -15,7 +15,7 @@ namespace {
 
 constexpr int kDefaultSMs = 148;
 constexpr int kDefaultWarps = 8;
-constexpr int kDefaultStages = 3;
+constexpr int kDefaultStages = 2;
 constexpr int kDefaultCtasPerSm = 1;
 constexpr size_t kSmemLimit = 227 * 1024;
 
@@ -56,7 +56,7 @@ Layout carve(const opw_attn_stage_config_t* c, const Shape& s, int sms) {
   size_t off = 0;
   L.status = off;  off += 256;
   L.cum = off;     off += align_up((B + 2) * 4, 256);
-  L.partials = off; off += align_up(workers * 2 * G * (D + 2) * 4, 256);
+  L.partials = off; off += align_up(workers * 2 * opw::kSegPerShare * G * (D + 2) * 4, 256);
   L.st_q = off;    off += align_up(B * Hq * D * 2, 256);
   L.st_k = off;    off += align_up(B * Hkv * D * 2, 256);
   L.st_v = off;    off += align_up(B * Hkv * D * 2, 256);
@@ -93,6 +93,7 @@ struct opw_attn_stage {
   float scale_log2e;
   int64_t launches;
   unsigned char* ws;
+  uint64_t* trace;
 };
 
 extern "C" {
@@ -193,6 +194,7 @@ opw_status_t opw_attn_stage_create(const opw_attn_stage_config_t* cfg, opw_attn_
   const double scale = cfg->softmax_scale > 0.f ? (double)cfg->softmax_scale : 1.0 / std::sqrt((double)cfg->head_dim);
   st->scale_log2e = (float)(scale * 1.4426950408889634);
   st->launches = 0;
+  st->trace = nullptr;
   st->ws = static_cast<unsigned char*>(cfg->workspace);
   *out = st;
   return OPW_OK;
@@ -200,6 +202,17 @@ opw_status_t opw_attn_stage_create(const opw_attn_stage_config_t* cfg, opw_attn_
 
 opw_status_t opw_attn_stage_destroy(opw_attn_stage_t* st) {
   delete st;
+  return OPW_OK;
+}
+
+opw_status_t opw_attn_stage_set_trace(opw_attn_stage_t* st, void* trace, size_t trace_bytes, int32_t* num_workers) {
+  if (!st) return OPW_ERR_INVALID_ARG;
+  const size_t workers = (size_t)st->grid * st->shape.warps;
+  if (num_workers) *num_workers = (int32_t)workers;
+  if (!trace) { st->trace = nullptr; return OPW_OK; }
+  if ((uintptr_t)trace % 8) return OPW_ERR_INVALID_ARG;
+  if (trace_bytes < workers * 32) return OPW_ERR_CAPACITY;
+  st->trace = static_cast<uint64_t*>(trace);
   return OPW_OK;
 }
 
@@ -262,6 +275,8 @@ opw_status_t opw_decode_attention(opw_attn_stage_t* st, int32_t layer, int32_t b
   p.partials = reinterpret_cast<float*>(st->ws + st->lay.partials);
   p.cum = reinterpret_cast<int32_t*>(st->ws + st->lay.cum);
   p.status = reinterpret_cast<uint32_t*>(st->ws + st->lay.status);
+  p.ticket = reinterpret_cast<int32_t*>(st->ws + st->lay.status + 16);
+  p.trace = st->trace;
   p.num_pages = st->num_pages[layer];
   p.batch = batch;
   p.Hq = Hq;
@@ -285,6 +300,7 @@ opw_status_t opw_decode_attention(opw_attn_stage_t* st, int32_t layer, int32_t b
   st->launches += 1;
 
   opw::CombineParams c;
+  c.ticket = p.ticket;
   c.partials = p.partials;
   c.cum = p.cum;
   c.kv_lens = kv_lens;
@@ -298,7 +314,7 @@ opw_status_t opw_decode_attention(opw_attn_stage_t* st, int32_t layer, int32_t b
   c.max_pages = p.max_pages;
   c.window = p.window;
   c.num_workers = st->grid * st->shape.warps;
-  opw::combine_kernel<<<batch * Hkv, 128, 0, stream>>>(c);
+  opw::combine_kernel<<<dim3(batch * Hkv, (G * D + 127) / 128), 128, 0, stream>>>(c);
   if (cudaGetLastError() != cudaSuccess) return OPW_ERR_CUDA;
   st->launches += 1;
   return OPW_OK;

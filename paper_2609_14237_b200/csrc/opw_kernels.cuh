@@ -3,13 +3,18 @@
 //
 // Work decomposition of the attention kernel.  A "unit" is one (sequence b, kv head g,
 // logical page) triple inside the visible range of b; units are ordered by (b, g, page)
-// and the U units of a launch are cut into equal contiguous ranges, one per warp
-// ("worker") of a persistent grid.  A worker therefore streams one 2*P*D*2-byte tile
-// (K rows then V rows of one page and head, contiguous in the pool) per unit, and meets
-// at most two rows (b, g) it does not own completely: the first and the last of its
-// range.  Complete rows are normalised and stored directly; the (at most two) incomplete
-// ones go to fixed partial slots 2*worker and 2*worker+1 and are merged by the combine
-// kernel.  Nothing in this scheme depends on page ids, only on kv_lens and the window.
+// and the U units of a launch are cut into equal contiguous shares, one per warp
+// ("worker") of a persistent grid.  A share is cut again into kSegPerShare segments: the
+// first 7/8 is the worker's own static segment, the last 1/8 is split into six ever
+// smaller chunks that any worker may take through an atomic ticket once its static
+// segment is done (SMs do not all stream at the same rate; the chunks even out the
+// finish times).  The segment boundaries depend only on kv_lens, the window and the grid,
+// never on which warp runs a segment or on page ids, so the result is deterministic.
+// A worker streams one 2*P*D*2-byte tile (K rows then V rows of one page and head,
+// contiguous in the pool) per unit.  A segment meets at most two rows (b, g) it does not
+// cover completely, its first and its last: complete rows are normalised and stored
+// directly; the incomplete ones go to the segment's two partial slots and are merged by
+// the combine kernel.
 #pragma once
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -21,7 +26,7 @@ constexpr int kPage = 16;               // tokens per page
 constexpr uint32_t kErrBadPage = 1u;    // bits of the device status word
 constexpr uint32_t kErrTimeout = 2u;
 constexpr int kMaxWarps = 8;
-constexpr uint32_t kSpinLimit = 1u << 22;   // bounded wait on a shared-memory copy
+constexpr uint64_t kWaitLimitNs = 100ull * 1000 * 1000;   // bound of a wait on a shared-memory copy: 0.1 s
 
 struct AttnParams {
   const __nv_bfloat16* pool;
@@ -33,6 +38,8 @@ struct AttnParams {
   float* partials;       // [num_workers*2][G*(D+2)]
   int32_t* cum;          // [batch+1] pages before sequence b (written by block 0)
   uint32_t* status;
+  int32_t* ticket;       // dynamic-chunk counter, zero at launch (the combine kernel re-zeroes it)
+  uint64_t* trace;       // optional [num_workers][4]: {smid | units<<32, t_begin, t_first_tile, t_end} in ns
   int64_t num_pages;
   int32_t batch, Hq, Hkv, G;
   int32_t max_pages;     // row stride of page_table
@@ -75,11 +82,19 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
       : "memory");
   return ok;
 }
-// Bounded wait: returns false if the phase did not complete within kSpinLimit polls.
+// Bounded wait: returns false if the phase did not complete within kWaitLimitNs of the
+// device's global timer (checked every 64 polls).
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < kSpinLimit; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  return false;
+  if (mbar_try_wait(bar, parity)) return true;
+  uint64_t t0;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
+  for (;;) {
+    for (int i = 0; i < 64; ++i)
+      if (mbar_try_wait(bar, parity)) return true;
+    uint64_t t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    if (t - t0 > kWaitLimitNs) return false;
+  }
 }
 // Linear bulk copy global -> shared of this CTA, completion counted on an mbarrier.
 __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
@@ -112,6 +127,16 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
   __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<uint32_t*>(&v);
 }
+__device__ __forceinline__ uint64_t global_timer_ns() {
+  uint64_t t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ uint32_t sm_id() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %smid;" : "=r"(r));
+  return r;
+}
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -135,9 +160,38 @@ __host__ __device__ __forceinline__ void visible_pages(int32_t n, int32_t window
 __host__ __device__ __forceinline__ int64_t worker_begin(int64_t U, int64_t worker, int64_t num_workers) {
   return (U * worker) / num_workers;
 }
-// the worker whose range [begin(w), begin(w+1)) holds unit u
+// the worker whose share [begin(w), begin(w+1)) holds unit u
 __host__ __device__ __forceinline__ int64_t worker_of(int64_t U, int64_t u, int64_t num_workers) {
   return ((u + 1) * num_workers - 1) / U;
+}
+// Segments of a share: k = 0 is the static first 7/8; k = 1..kDynPerShare cut the last 1/8
+// into ever smaller chunks (cut points in sixteenths of that eighth).
+#ifndef OPW_DYN_PER_SHARE
+#define OPW_DYN_PER_SHARE 6
+#endif
+constexpr int kDynPerShare = OPW_DYN_PER_SHARE;
+constexpr int kSegPerShare = kDynPerShare + 1;
+__host__ __device__ __forceinline__ int64_t dyn_cut(int k) {   // five bits per cut point
+#if OPW_DYN_PER_SHARE == 8
+  const uint64_t cuts = 0ull | (4ull << 5) | (8ull << 10) | (10ull << 15) | (12ull << 20) | (13ull << 25) |
+                        (14ull << 30) | (15ull << 35) | (16ull << 40);       // 0,4,8,10,12,13,14,15,16
+#elif OPW_DYN_PER_SHARE == 4
+  const uint64_t cuts = 0ull | (8ull << 5) | (12ull << 10) | (14ull << 15) | (16ull << 20);   // 0,8,12,14,16
+#elif OPW_DYN_PER_SHARE == 6
+  const uint64_t cuts = 0ull | (5ull << 5) | (9ull << 10) | (12ull << 15) | (14ull << 20) | (15ull << 25) |
+                        (16ull << 30);                                        // 0,5,9,12,14,15,16
+#else
+#error "unsupported OPW_DYN_PER_SHARE"
+#endif
+  return (int64_t)((cuts >> (5 * k)) & 31);
+}
+__host__ __device__ __forceinline__ void segment_bounds(int64_t U, int64_t num_workers, int64_t w, int k,
+                                                        int64_t& a, int64_t& b) {
+  const int64_t s0 = worker_begin(U, w, num_workers), s1 = worker_begin(U, w + 1, num_workers);
+  const int64_t len = s1 - s0, dyn = len >> 3, stat = len - dyn;
+  if (k == 0) { a = s0; b = s0 + stat; return; }
+  a = s0 + stat + ((dyn * dyn_cut(k - 1)) >> 4);
+  b = s0 + stat + ((dyn * dyn_cut(k)) >> 4);
 }
 
 // ---------------------------------------------------------------------------------
@@ -252,9 +306,9 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
   const int64_t U = (int64_t)cum[p.batch] * p.Hkv;
   const int64_t num_workers = (int64_t)gridDim.x * warps;
   const int64_t worker = (int64_t)blockIdx.x * warps + warp;
-  const int64_t u0 = worker_begin(U, worker, num_workers);
-  const int64_t u1 = worker_begin(U, worker + 1, num_workers);
-  if (u0 >= u1) return;
+  if (U == 0) return;
+  uint64_t* tr = p.trace ? p.trace + worker * 4 : nullptr;
+  if (tr && lane == 0) tr[1] = global_timer_ns();
 
   // ---- this warp's ring ----
   const uint32_t ring_base = smem_u32(ring + (size_t)warp * stages * TILE);
@@ -266,11 +320,13 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
   }
   __syncwarp();
 
+  int64_t u0 = 0, u1 = 0;                     // the segment being processed: units [u0, u1)
+
   // ---- unit descriptors, 32 at a time, one per lane ----
-  auto describe = [&](int64_t u) -> UnitDesc {
+  auto describe = [&](int64_t u, int64_t u_end) -> UnitDesc {
     UnitDesc d;
     d.tile = 0; d.row = 0; d.info = 0;
-    if (u >= u1) return d;
+    if (u >= u_end) return d;
     // sequence: largest b with cum[b]*Hkv <= u
     int lo_b = 0, hi_b = p.batch;             // invariant: cum[lo_b]*Hkv <= u < cum[hi_b]*Hkv
     while (hi_b - lo_b > 1) {
@@ -297,18 +353,11 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
     return d;
   };
 
-  int64_t wbase = u0;                         // unit of lane 0 in window A
-  UnitDesc wa = describe(wbase + lane);
-  UnitDesc wb = describe(wbase + 32 + lane);
+  int64_t wbase = 0;                          // unit of lane 0 in window A
+  UnitDesc wa = {0, 0, 0}, wb = {0, 0, 0};    // descriptors of units [wbase, wbase+32) and the next 32
+  UnitDesc nx = {0, 0, 0};                    // descriptors of the first 32 units of the next segment
 
-  auto tile_of = [&](int64_t u) -> int32_t {  // warp-uniform u in [wbase, wbase+64)
-    const int rel = (int)(u - wbase);
-    const int32_t a = __shfl_sync(0xffffffffu, wa.tile, rel & 31);
-    const int32_t b = __shfl_sync(0xffffffffu, wb.tile, rel & 31);
-    return rel < 32 ? a : b;
-  };
-  auto issue = [&](int64_t u, int slot) {     // all lanes call; lane 0 issues
-    const int32_t tile = tile_of(u);
+  auto issue_tile = [&](int32_t tile, int slot) {   // lane 0 issues the copy of one K|V tile
     if (lane == 0) {
       const uint32_t bar = bar_base + 8 * slot;
       mbar_expect_tx(bar, TILE);
@@ -316,10 +365,12 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
                 TILE, bar);
     }
   };
-
-  // prologue: fill the ring
-  const int prolog = (int)((u1 - u0) < stages ? (u1 - u0) : stages);
-  for (int s = 0; s < prolog; ++s) issue(u0 + s, s);
+  auto tile_of = [&](int64_t u) -> int32_t {  // warp-uniform u in [wbase, wbase+64)
+    const int rel = (int)(u - wbase);
+    const int32_t a = __shfl_sync(0xffffffffu, wa.tile, rel & 31);
+    const int32_t b = __shfl_sync(0xffffffffu, wb.tile, rel & 31);
+    return rel < 32 ? a : b;
+  };
 
   // per-lane constant offsets of the matrix loads
   const int mi = lane >> 3, rr = lane & 7;
@@ -332,18 +383,67 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
   float o[NT][4];
   float m_lo = -1e30f, l_lo = 0.f, m_hi = -1e30f, l_hi = 0.f;
   bool seg_from_first = false;
-  bool seg_is_workers_first = true;
   bool failed = false;
 
   int slot = 0;
   uint32_t phase = 0;
-  int64_t u = u0;
-  for (; u < u1; ++u) {
+  int inflight = 0;                           // copies issued and not yet consumed
+  int64_t u = 0;
+  int64_t units_done = 0;
+  bool traced_first = false;
+  const int32_t num_tickets = (int32_t)(num_workers * kDynPerShare);
+
+  // The segment being processed is [u0,u1) with partial slots slot_base, slot_base+1; first the
+  // worker's own static segment, then whatever chunks the ticket counter hands out.  The next
+  // segment [n0,n1) is resolved a few units before the current one ends, so that its first
+  // tiles are already on their way when the current segment's last tile is consumed.
+  int64_t slot_base = 2 * (worker * kSegPerShare);
+  segment_bounds(U, num_workers, worker, 0, u0, u1);
+  int64_t n0 = 0, n1 = 0, nslot_base = 0;
+  int next_issued = 0;                        // units of the next segment already issued
+  wbase = u0;
+  wa = describe(wbase + lane, u1);
+  wb = describe(wbase + 32 + lane, u1);
+  for (;;) {
+  int32_t ticket = 0;                         // asked for now, looked at near the segment's end
+  if (lane == 0) ticket = atomicAdd(p.ticket, 1);
+  bool next_known = false;
+  bool seg_on_first_row = true;               // partial slot 0 for the segment's first row, 1 for its last
+  {
+    const int64_t len = u1 - u0;
+    const int want = (int)(len < stages ? len : stages);
+    for (int s = next_issued; s < want; ++s) {  // (re)fill the ring: what the previous segment did not prefetch
+      int sl = slot + s; if (sl >= stages) sl -= stages;
+      issue_tile(tile_of(u0 + s), sl);
+      ++inflight;
+    }
+    units_done += len;
+  }
+  // resolve the next segment: skip empty chunks, stop when the tickets run out
+  auto resolve_next = [&]() {
+    int32_t t = __shfl_sync(0xffffffffu, ticket, 0);
+    n0 = n1 = 0;
+    while (t < num_tickets) {
+      const int64_t w = t % (int32_t)num_workers;           // large chunks of every share first, small ones last
+      const int k = 1 + t / (int32_t)num_workers;
+      segment_bounds(U, num_workers, w, k, n0, n1);
+      nslot_base = 2 * (w * kSegPerShare + k);
+      if (n0 < n1) break;
+      if (lane == 0) t = atomicAdd(p.ticket, 1);
+      t = __shfl_sync(0xffffffffu, t, 0);
+    }
+    if (t >= num_tickets) n0 = n1 = 0;
+    nx = describe(n0 + lane, n1);
+    next_known = true;
+    next_issued = 0;
+  };
+  for (u = u0; u < u1; ++u) {
     if (u - wbase == 32) {                    // slide the descriptor windows
       wbase += 32;
       wa = wb;
-      wb = describe(wbase + 32 + lane);
+      wb = describe(wbase + 32 + lane, u1);
     }
+    if (!next_known && u + stages + 2 >= u1) resolve_next();
     const int rel = (int)(u - wbase);
     const int32_t row = __shfl_sync(0xffffffffu, wa.row, rel);
     const int32_t info = __shfl_sync(0xffffffffu, wa.info, rel);
@@ -374,6 +474,9 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
 
     // wait for this unit's tile
     if (!mbar_wait_bounded(bar_base + 8 * slot, phase)) { failed = true; break; }
+    --inflight;
+    if (tr && !traced_first && lane == 0) tr[2] = global_timer_ns();
+    traced_first = true;
 
     const uint32_t tile = ring_base + slot * TILE;
     const bool ragged = (t0 > 0) || (t1 < kPage);
@@ -465,9 +568,25 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
 
     // ---- refill this slot with the unit `stages` ahead ----
     __syncwarp();
-    if (u + stages < u1) {
-      if (lane == 0) fence_proxy_async();
-      issue(u + stages, slot);
+    {
+      const int64_t target = u + stages;      // this worker's stream runs on into the next segment
+      if (target < u1) {
+        const int32_t tile = tile_of(target);
+        if (lane == 0) fence_proxy_async();
+        issue_tile(tile, slot);
+        ++inflight;
+      } else {
+        // Next-segment units are prefetched strictly in order; a segment shorter than the
+        // ring starts past unit 0 here and leaves the next segment's fill to the loop top.
+        const int j = (int)(target - u1);
+        if (j == next_issued && j < 32 && j < n1 - n0) {
+          const int32_t tile = __shfl_sync(0xffffffffu, nx.tile, j);
+          if (lane == 0) fence_proxy_async();
+          issue_tile(tile, slot);
+          ++inflight;
+          next_issued = j + 1;
+        }
+      }
     }
     if (++slot == stages) { slot = 0; phase ^= 1u; }
 
@@ -501,7 +620,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
         }
       } else {
         // partial: unnormalised o, running max and sum, into this worker's slot
-        const int64_t pslot = worker * 2 + (seg_is_workers_first ? 0 : 1);
+        const int64_t pslot = slot_base + (seg_on_first_row ? 0 : 1);
         float* pb = p.partials + pslot * (int64_t)(p.G * (D + 2));
         if (qrow < p.G) {
 #pragma unroll
@@ -516,16 +635,27 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
           if ((lane & 3) == 0) { pb[p.G * D + qrow + 8] = m_hi; pb[p.G * D + p.G + qrow + 8] = l1; }
         }
       }
-      seg_is_workers_first = false;
+      seg_on_first_row = false;
     }
   }
+  if (failed) break;
+  if (!next_known) resolve_next();            // (an empty segment never enters the loop above)
+  if (n0 >= n1) break;                        // no chunk left
+  u0 = n0; u1 = n1; slot_base = nslot_base;
+  wbase = u0;
+  wa = nx;
+  wb = describe(wbase + 32 + lane, u1);
+  }
 
+  if (tr && lane == 0) {
+    tr[0] = (uint64_t)sm_id() | ((uint64_t)units_done << 32);
+    tr[3] = global_timer_ns();
+  }
   if (failed) {
     // A copy did not arrive in time: record it, then give every copy still in flight a
     // bounded chance to land before this warp's shared memory is released.
     if (lane == 0) atomicOr(p.status, kErrTimeout);
-    int64_t issued_end = u + stages < u1 ? u + stages : u1;   // units [u, issued_end) are in flight
-    for (int64_t v = u; v < issued_end; ++v) {
+    for (int i = 0; i < inflight; ++i) {
       (void)mbar_wait_bounded(bar_base + 8 * slot, phase);
       if (++slot == stages) { slot = 0; phase ^= 1u; }
     }
@@ -533,9 +663,10 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
 }
 
 // ---------------------------------------------------------------------------------
-// log-sum-exp combine: one block per (sequence, kv head) row
+// log-sum-exp combine
 // ---------------------------------------------------------------------------------
 struct CombineParams {
+  int32_t* ticket;       // the attention kernel's chunk counter: re-zeroed here for the next launch
   const float* partials;
   const int32_t* cum;
   const int32_t* kv_lens;
@@ -546,17 +677,26 @@ struct CombineParams {
   int32_t num_workers;
 };
 
+// grid = (rows, ceil(G*D/128)), 128 threads: one thread per output element of the row.
 __global__ void combine_kernel(CombineParams p) {
+  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *p.ticket = 0;
   const int row = blockIdx.x;
   const int b = row / p.Hkv, g = row - b * p.Hkv;
-  const int D = p.D;
+  const int D = p.D, G = p.G;
+  const int e = blockIdx.y * 128 + threadIdx.x;       // element of the row's [G, D] output
+  const bool valid = e < G * D;
+  const int h = valid ? e / D : G - 1;
+  const int h_first = (blockIdx.y * 128) / D;           // heads this block touches: h_first, h_first+1
+  const int nh = min(G - 1, (blockIdx.y * 128 + 127) / D) - h_first + 1;
   int32_t n = p.kv_lens[b];
   if (n > p.max_pages * kPage) n = p.max_pages * kPage;
-  __nv_bfloat16* ob = p.out + ((int64_t)b * p.Hq + (int64_t)g * p.G) * D;
+  __nv_bfloat16* ob = p.out + ((int64_t)b * p.Hq + (int64_t)g * G) * D;
+  float* lse_row = p.lse ? p.lse + (int64_t)b * p.Hq + g * G : nullptr;
   if (n <= 0) {   // inactive slot: zeros, lse = -inf
-    for (int i = threadIdx.x; i < p.G * D; i += blockDim.x) ob[i] = __float2bfloat16(0.f);
-    if (p.lse)
-      for (int i = threadIdx.x; i < p.G; i += blockDim.x) p.lse[(int64_t)b * p.Hq + g * p.G + i] = -INFINITY;
+    if (valid) {
+      ob[e] = __float2bfloat16(0.f);
+      if (lse_row && e == h * D) lse_row[h] = -INFINITY;
+    }
     return;
   }
   int32_t first, cnt, lo;
@@ -565,37 +705,102 @@ __global__ void combine_kernel(CombineParams p) {
   const int64_t ustart = (int64_t)p.cum[b] * p.Hkv + (int64_t)g * cnt;
   const int64_t uend = ustart + cnt;
   const int64_t wf = worker_of(U, ustart, p.num_workers), wl = worker_of(U, uend - 1, p.num_workers);
-  if (wf == wl) return;                       // the row was finished by a single worker
-  const int64_t stride = (int64_t)p.G * (D + 2);
-  // Walk the row's segments: the worker holding unit u owns [u, min(end of its range, uend)).
-  // (Workers with an empty range hold no unit and are never visited.)  A worker's partial is
-  // in its slot 0 if the row is the first one it touches, else in slot 1.
-  auto slot_at = [&](int64_t u, int64_t& next_u) -> const float* {
-    const int64_t w = worker_of(U, u, p.num_workers);
-    const int64_t wb = worker_begin(U, w, p.num_workers);
-    next_u = worker_begin(U, w + 1, p.num_workers);
-    const bool is_first_row = wb >= ustart;
-    return p.partials + (w * 2 + (is_first_row ? 0 : 1)) * stride;
-  };
-  for (int h = 0; h < p.G; ++h) {
-    float M = -INFINITY;
-    for (int64_t u = ustart, nu; u < uend; u = nu) M = fmaxf(M, slot_at(u, nu)[p.G * D + h]);
-    float L = 0.f;
-    for (int64_t u = ustart, nu; u < uend; u = nu) {
-      const float* s = slot_at(u, nu);
-      L += exp2f(s[p.G * D + h] - M) * s[p.G * D + p.G + h];
+  const int64_t stride = (int64_t)G * (D + 2);
+  // The row's partials come from the segments (share w in wf..wl, k in 0..kSegPerShare) that
+  // overlap it.  128 candidate segments at a time: each thread tests one, an ordered
+  // compaction lists the partial slots in shared memory, one warp per head turns the partials'
+  // running maxima into weights 2^(m - M), and every thread sums its element over the list.
+  // A segment's partial for this row is in the segment's slot 0 if the segment starts inside
+  // the row, else in slot 1.  If one segment covers the whole row, its worker has already
+  // stored the final result.
+  __shared__ int32_t seg_slot[128];
+  __shared__ int32_t warp_cnt[4];
+  __shared__ float w_s[128 * 2];                // per (segment, head of this block): m, then the weight
+  __shared__ float l_s[128 * 2];
+  __shared__ float run_M[2], run_L[2], run_scale[2];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  float acc = 0.f;
+  if (threadIdx.x < 2) { run_M[threadIdx.x] = -INFINITY; run_L[threadIdx.x] = 0.f; }
+  const int64_t ncand = (wl - wf + 1) * kSegPerShare;
+  for (int64_t base = 0; base < ncand; base += blockDim.x) {
+    const int64_t i = base + threadIdx.x;
+    bool hit = false, whole = false;
+    int32_t slot = 0;
+    if (i < ncand) {
+      const int64_t w = wf + i / kSegPerShare;
+      const int k = (int)(i % kSegPerShare);
+      int64_t a, bnd;
+      segment_bounds(U, p.num_workers, w, k, a, bnd);
+      hit = a < bnd && a < uend && bnd > ustart;
+      whole = hit && a <= ustart && bnd >= uend;
+      slot = (int32_t)(2 * (w * kSegPerShare + k) + (a >= ustart ? 0 : 1));
     }
-    const float inv = L > 0.f ? 1.f / L : 0.f;
-    for (int d = threadIdx.x; d < D; d += blockDim.x) {
-      float acc = 0.f;
-      for (int64_t u = ustart, nu; u < uend; u = nu) {
-        const float* s = slot_at(u, nu);
-        acc += exp2f(s[p.G * D + h] - M) * s[h * D + d];
+    if (__syncthreads_or(whole)) return;        // finished by a single segment: nothing to merge
+    const uint32_t bal = __ballot_sync(0xffffffffu, hit);
+    if (lane == 0) warp_cnt[warp] = __popc(bal);
+    __syncthreads();
+    int pos = __popc(bal & ((1u << lane) - 1u));
+    int nseg = 0;
+    for (int j = 0; j < 4; ++j) {
+      if (j < warp) pos += warp_cnt[j];
+      nseg += warp_cnt[j];
+    }
+    if (hit) seg_slot[pos] = slot;
+    __syncthreads();
+    for (int idx = threadIdx.x; idx < nseg * nh; idx += blockDim.x) {   // stage (m, l): independent loads
+      const int sgm = idx / nh, hh = idx - sgm * nh;
+      const float* sp = p.partials + (int64_t)seg_slot[sgm] * stride + G * D;
+      w_s[sgm * 2 + hh] = sp[h_first + hh];
+      l_s[sgm * 2 + hh] = sp[G + h_first + hh];
+    }
+    __syncthreads();
+    if (warp < nh) {                              // one warp per head: max, weights, weighted sum of l
+      const int hh = warp;
+      float Mc = run_M[hh];
+      for (int sgm = lane; sgm < nseg; sgm += 32) Mc = fmaxf(Mc, w_s[sgm * 2 + hh]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) Mc = fmaxf(Mc, __shfl_xor_sync(0xffffffffu, Mc, o));
+      float Lc = 0.f;
+      for (int sgm = lane; sgm < nseg; sgm += 32) {
+        const float wgt = exp2f(w_s[sgm * 2 + hh] - Mc);
+        w_s[sgm * 2 + hh] = wgt;
+        Lc += wgt * l_s[sgm * 2 + hh];
       }
-      ob[h * D + d] = __float2bfloat16_rn(acc * inv);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) Lc += __shfl_xor_sync(0xffffffffu, Lc, o);
+      if (lane == 0) {
+        const float sc = exp2f(run_M[hh] - Mc);   // 0 on the first batch (run_M = -inf)
+        run_L[hh] = run_L[hh] * sc + Lc;
+        run_M[hh] = Mc;
+        run_scale[hh] = sc;
+      }
     }
-    if (p.lse && threadIdx.x == 0)
-      p.lse[(int64_t)b * p.Hq + g * p.G + h] = L > 0.f ? (M + log2f(L)) * 0.6931471805599453f : -INFINITY;
+    __syncthreads();
+    if (valid) {
+      const int hh = h - h_first;
+      const float* pe = p.partials + e;
+      float a[8];
+      a[0] = acc * run_scale[hh];
+#pragma unroll
+      for (int j = 1; j < 8; ++j) a[j] = 0.f;
+      int sgm = 0;
+      for (; sgm + 8 <= nseg; sgm += 8) {         // eight independent loads in flight
+        float o[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) o[j] = pe[(int64_t)seg_slot[sgm + j] * stride];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) a[j] += w_s[(sgm + j) * 2 + hh] * o[j];
+      }
+      for (; sgm < nseg; ++sgm) a[0] += w_s[sgm * 2 + hh] * pe[(int64_t)seg_slot[sgm] * stride];
+      acc = ((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7]));
+    }
+    __syncthreads();
+  }
+  if (valid) {
+    const int hh = h - h_first;
+    const float Lh = run_L[hh];
+    ob[e] = __float2bfloat16_rn(Lh > 0.f ? acc / Lh : 0.f);
+    if (lse_row && e == h * D) lse_row[h] = Lh > 0.f ? (run_M[hh] + log2f(Lh)) * 0.6931471805599453f : -INFINITY;
   }
 }
 
