@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libopw_attn.so")
 SOURCES = [os.path.join(_HERE, "csrc", "opw_attn.cu")]
 HEADERS = [os.path.join(_HERE, "csrc", "opw_kernels.cuh"), os.path.join(_ROOT, "include", "opw_attn.h")]
 
+OPW_FLAG_PDL = 1
 OPW_OK, OPW_ERR_INVALID_ARG, OPW_ERR_UNSUPPORTED, OPW_ERR_CAPACITY, OPW_ERR_CUDA, OPW_ERR_BAD_PAGE, OPW_ERR_TIMEOUT = range(7)
 
 EXPORTS = [
@@ -226,7 +227,7 @@ class Stage:
 
     def __init__(self, *, pools, layer_window, num_q_heads, num_kv_heads, head_dim, max_batch, max_pages_per_seq,
                  layer_num_pages=None, device=None, softmax_scale=0.0, tune_warps=0, tune_stages=0,
-                 tune_ctas_per_sm=0):
+                 tune_ctas_per_sm=0, flags=0):
         import torch
 
         dev = pools[0].device if device is None else torch.device(device)
@@ -241,7 +242,7 @@ class Stage:
                   max_batch=max_batch, max_pages_per_seq=max_pages_per_seq, layer_window=layer_window,
                   layer_num_pages=layer_num_pages, layer_kv_pool=[p.data_ptr() for p in pools],
                   softmax_scale=softmax_scale, tune_warps=tune_warps, tune_stages=tune_stages,
-                  tune_ctas_per_sm=tune_ctas_per_sm)
+                  tune_ctas_per_sm=tune_ctas_per_sm, flags=flags)
         cfg, _keep = make_config(**kw)
         nbytes = opw_attn_stage_workspace_bytes(cfg)
         if nbytes == 0:

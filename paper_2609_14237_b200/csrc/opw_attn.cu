@@ -69,6 +69,25 @@ Layout carve(const opw_attn_stage_config_t* c, const Shape& s, int sms) {
   return L;
 }
 
+// Launch with (or without) the programmatic-stream-serialization attribute: the kernel may
+// start while the previous kernel in the stream is still running and synchronises with it
+// on the device (griddepcontrol.wait).
+template <typename... KArgs, typename... Args>
+cudaError_t launch(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, bool pdl,
+                   Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 int query_sms(int device) {
   int sms = 0;
   if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || sms <= 0) {
@@ -247,8 +266,12 @@ opw_status_t opw_kv_append(opw_attn_stage_t* st, int32_t layer, int32_t batch, c
   p.max_pages = st->cfg.max_pages_per_seq;
   const int groups = p.Hkv * 2 * (p.D / 8);
   const int threads = groups < 256 ? ((groups + 31) / 32 * 32) : 256;
-  opw::kv_append_kernel<<<batch, threads, 0, static_cast<cudaStream_t>(cuda_stream)>>>(p);
-  if (cudaGetLastError() != cudaSuccess) return OPW_ERR_CUDA;
+  const bool pdl = (st->cfg.flags & OPW_FLAG_PDL) != 0;
+  if (launch(opw::kv_append_kernel, dim3(batch), dim3(threads), 0, static_cast<cudaStream_t>(cuda_stream), pdl, p) !=
+      cudaSuccess) {
+    (void)cudaGetLastError();
+    return OPW_ERR_CUDA;
+  }
   st->launches += 1;
   return OPW_OK;
 }
@@ -289,14 +312,16 @@ opw_status_t opw_decode_attention(opw_attn_stage_t* st, int32_t layer, int32_t b
 
   const dim3 grid(st->grid), block(st->shape.warps * 32);
   const size_t smem = attn_smem_bytes(D, st->shape, batch);
+  const bool pdl = (st->cfg.flags & OPW_FLAG_PDL) != 0;
+  cudaError_t e;
   if (D == 64) {
-    if (G > 8) opw::attn_splitkv_kernel<64, true><<<grid, block, smem, stream>>>(p);
-    else opw::attn_splitkv_kernel<64, false><<<grid, block, smem, stream>>>(p);
+    if (G > 8) e = launch(opw::attn_splitkv_kernel<64, true>, grid, block, smem, stream, pdl, p);
+    else e = launch(opw::attn_splitkv_kernel<64, false>, grid, block, smem, stream, pdl, p);
   } else {
-    if (G > 8) opw::attn_splitkv_kernel<128, true><<<grid, block, smem, stream>>>(p);
-    else opw::attn_splitkv_kernel<128, false><<<grid, block, smem, stream>>>(p);
+    if (G > 8) e = launch(opw::attn_splitkv_kernel<128, true>, grid, block, smem, stream, pdl, p);
+    else e = launch(opw::attn_splitkv_kernel<128, false>, grid, block, smem, stream, pdl, p);
   }
-  if (cudaGetLastError() != cudaSuccess) return OPW_ERR_CUDA;
+  if (e != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
   st->launches += 1;
 
   opw::CombineParams c;
@@ -314,8 +339,10 @@ opw_status_t opw_decode_attention(opw_attn_stage_t* st, int32_t layer, int32_t b
   c.max_pages = p.max_pages;
   c.window = p.window;
   c.num_workers = st->grid * st->shape.warps;
-  opw::combine_kernel<<<dim3(batch * Hkv, (G * D + 127) / 128), 128, 0, stream>>>(c);
-  if (cudaGetLastError() != cudaSuccess) return OPW_ERR_CUDA;
+  if (launch(opw::combine_kernel, dim3(batch * Hkv), dim3(opw::kCombineThreads), 0, stream, pdl, c) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return OPW_ERR_CUDA;
+  }
   st->launches += 1;
   return OPW_OK;
 }

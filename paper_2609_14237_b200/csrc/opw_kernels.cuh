@@ -96,13 +96,26 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
     if (t - t0 > kWaitLimitNs) return false;
   }
 }
-// Linear bulk copy global -> shared of this CTA, completion counted on an mbarrier.
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+// Linear bulk copy global -> shared of this CTA, completion counted on an mbarrier.  The KV
+// stream is read once per step, so it is marked evict-first in L2 and leaves the small
+// re-read data (partials, q, page tables) alone.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t pol) {
   asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-      "l"(src), "r"(bytes), "r"(bar)
+      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+          dst),
+      "l"(src), "r"(bytes), "r"(bar), "l"(pol)
       : "memory");
 }
+// Programmatic dependent launch: a kernel launched with the stream-serialization attribute may
+// start while its predecessor in the stream still runs; it must not touch anything the
+// predecessor (or, transitively, earlier kernels) produces before pdl_wait() returns.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
@@ -185,10 +198,12 @@ __host__ __device__ __forceinline__ int64_t dyn_cut(int k) {   // five bits per 
 #endif
   return (int64_t)((cuts >> (5 * k)) & 31);
 }
+// Launches with fewer than eight units per worker have no dynamic chunks at all.
+__host__ __device__ __forceinline__ bool has_dynamic(int64_t U, int64_t num_workers) { return U >= 8 * num_workers; }
 __host__ __device__ __forceinline__ void segment_bounds(int64_t U, int64_t num_workers, int64_t w, int k,
                                                         int64_t& a, int64_t& b) {
   const int64_t s0 = worker_begin(U, w, num_workers), s1 = worker_begin(U, w + 1, num_workers);
-  const int64_t len = s1 - s0, dyn = len >> 3, stat = len - dyn;
+  const int64_t len = s1 - s0, dyn = has_dynamic(U, num_workers) ? len >> 3 : 0, stat = len - dyn;
   if (k == 0) { a = s0; b = s0 + stat; return; }
   a = s0 + stat + ((dyn * dyn_cut(k - 1)) >> 4);
   b = s0 + stat + ((dyn * dyn_cut(k)) >> 4);
@@ -198,8 +213,10 @@ __host__ __device__ __forceinline__ void segment_bounds(int64_t U, int64_t num_w
 // KV append: one thread block per sequence, one thread per 16-byte group
 // ---------------------------------------------------------------------------------
 __global__ void kv_append_kernel(AppendParams p) {
+  pdl_launch_dependents();                    // the attention kernel may start its prologue now
   const int b = blockIdx.x;
-  const int32_t pos = p.positions[b];
+  const int32_t pos = p.positions[b];         // inputs only before the wait
+  pdl_wait();                                 // everything enqueued earlier has finished
   if (pos < 0) return;
   const int32_t lp = pos / kPage, t = pos % kPage;
   if (lp >= p.max_pages) {
@@ -255,6 +272,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
   constexpr int TILE = AttnSmem<D>::kTileBytes;
   extern __shared__ __align__(128) unsigned char smem[];
 
+  pdl_launch_dependents();                    // lets the combine kernel queue up behind this grid
   const int warps = blockDim.x >> 5;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int stages = p.stages;
@@ -299,8 +317,6 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
     }
     if (threadIdx.x == 0) cum[p.batch] = carry;
     __syncthreads();
-    if (blockIdx.x == 0)
-      for (int i = threadIdx.x; i <= p.batch; i += blockDim.x) p.cum[i] = cum[i];
   }
 
   const int64_t U = (int64_t)cum[p.batch] * p.Hkv;
@@ -357,12 +373,13 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
   UnitDesc wa = {0, 0, 0}, wb = {0, 0, 0};    // descriptors of units [wbase, wbase+32) and the next 32
   UnitDesc nx = {0, 0, 0};                    // descriptors of the first 32 units of the next segment
 
+  const uint64_t kv_policy = l2_evict_first_policy();
   auto issue_tile = [&](int32_t tile, int slot) {   // lane 0 issues the copy of one K|V tile
     if (lane == 0) {
       const uint32_t bar = bar_base + 8 * slot;
       mbar_expect_tx(bar, TILE);
       bulk_load(ring_base + slot * TILE, reinterpret_cast<const unsigned char*>(p.pool) + (int64_t)tile * TILE,
-                TILE, bar);
+                TILE, bar, kv_policy);
     }
   };
   auto tile_of = [&](int64_t u) -> int32_t {  // warp-uniform u in [wbase, wbase+64)
@@ -391,7 +408,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
   int64_t u = 0;
   int64_t units_done = 0;
   bool traced_first = false;
-  const int32_t num_tickets = (int32_t)(num_workers * kDynPerShare);
+  const int32_t num_tickets = has_dynamic(U, num_workers) ? (int32_t)(num_workers * kDynPerShare) : 0;
 
   // The segment being processed is [u0,u1) with partial slots slot_base, slot_base+1; first the
   // worker's own static segment, then whatever chunks the ticket counter hands out.  The next
@@ -404,9 +421,14 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
   wbase = u0;
   wa = describe(wbase + lane, u1);
   wb = describe(wbase + 32 + lane, u1);
+  // Up to here only this step's inputs (kv_lens, page table) were read.  The pool (appended to
+  // by the previous kernel), the workspace and the outputs are touched after this point.
+  pdl_wait();
+  if (blockIdx.x == 0)
+    for (int i = lane + 32 * warp; i <= p.batch; i += blockDim.x) p.cum[i] = cum[i];
   for (;;) {
   int32_t ticket = 0;                         // asked for now, looked at near the segment's end
-  if (lane == 0) ticket = atomicAdd(p.ticket, 1);
+  if (lane == 0 && num_tickets > 0) ticket = atomicAdd(p.ticket, 1);
   bool next_known = false;
   bool seg_on_first_row = true;               // partial slot 0 for the segment's first row, 1 for its last
   {
@@ -677,61 +699,77 @@ struct CombineParams {
   int32_t num_workers;
 };
 
-// grid = (rows, ceil(G*D/128)), 128 threads: one thread per output element of the row.
-__global__ void combine_kernel(CombineParams p) {
-  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *p.ticket = 0;
+// One block of kCombineThreads per (sequence, kv head) row; thread t owns the output
+// elements t, t + kCombineThreads, ... of the row's [G, D] block.
+constexpr int kCombineThreads = 256;
+constexpr int kCombineMaxG = 16;
+constexpr int kCombineBatch = 64;               // segments merged per pass
+__global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams p) {
+  pdl_launch_dependents();
   const int row = blockIdx.x;
   const int b = row / p.Hkv, g = row - b * p.Hkv;
   const int D = p.D, G = p.G;
-  const int e = blockIdx.y * 128 + threadIdx.x;       // element of the row's [G, D] output
-  const bool valid = e < G * D;
-  const int h = valid ? e / D : G - 1;
-  const int h_first = (blockIdx.y * 128) / D;           // heads this block touches: h_first, h_first+1
-  const int nh = min(G - 1, (blockIdx.y * 128 + 127) / D) - h_first + 1;
-  int32_t n = p.kv_lens[b];
+  const int GD = G * D;
+  int32_t n = p.kv_lens[b];                    // an input: may be read before the attention kernel is done
+  pdl_wait();                                  // partials, prefix sums and complete rows are final now
+  if (blockIdx.x == 0 && threadIdx.x == 0) *p.ticket = 0;
+  const int32_t cum_b = p.cum[b], cum_all = p.cum[p.batch];     // independent of the load above
   if (n > p.max_pages * kPage) n = p.max_pages * kPage;
   __nv_bfloat16* ob = p.out + ((int64_t)b * p.Hq + (int64_t)g * G) * D;
   float* lse_row = p.lse ? p.lse + (int64_t)b * p.Hq + g * G : nullptr;
   if (n <= 0) {   // inactive slot: zeros, lse = -inf
-    if (valid) {
-      ob[e] = __float2bfloat16(0.f);
-      if (lse_row && e == h * D) lse_row[h] = -INFINITY;
-    }
+    for (int e = threadIdx.x; e < GD; e += kCombineThreads) ob[e] = __float2bfloat16(0.f);
+    if (lse_row && threadIdx.x < G) lse_row[threadIdx.x] = -INFINITY;
     return;
   }
   int32_t first, cnt, lo;
   visible_pages(n, p.window, p.max_pages, first, cnt, lo);
-  const int64_t U = (int64_t)p.cum[p.batch] * p.Hkv;
-  const int64_t ustart = (int64_t)p.cum[b] * p.Hkv + (int64_t)g * cnt;
+  const int64_t U = (int64_t)cum_all * p.Hkv;
+  const int64_t ustart = (int64_t)cum_b * p.Hkv + (int64_t)g * cnt;
   const int64_t uend = ustart + cnt;
   const int64_t wf = worker_of(U, ustart, p.num_workers), wl = worker_of(U, uend - 1, p.num_workers);
   const int64_t stride = (int64_t)G * (D + 2);
   // The row's partials come from the segments (share w in wf..wl, k in 0..kSegPerShare) that
-  // overlap it.  128 candidate segments at a time: each thread tests one, an ordered
+  // overlap it.  A batch of candidate segments at a time: each thread tests one, an ordered
   // compaction lists the partial slots in shared memory, one warp per head turns the partials'
-  // running maxima into weights 2^(m - M), and every thread sums its element over the list.
+  // running maxima into weights 2^(m - M), and every thread sums its elements over the list.
   // A segment's partial for this row is in the segment's slot 0 if the segment starts inside
   // the row, else in slot 1.  If one segment covers the whole row, its worker has already
   // stored the final result.
-  __shared__ int32_t seg_slot[128];
-  __shared__ int32_t warp_cnt[4];
-  __shared__ float w_s[128 * 2];                // per (segment, head of this block): m, then the weight
-  __shared__ float l_s[128 * 2];
-  __shared__ float run_M[2], run_L[2], run_scale[2];
+  __shared__ int32_t seg_slot[kCombineBatch];
+  __shared__ int32_t warp_cnt[kCombineThreads / 32];
+  __shared__ float w_s[kCombineBatch * kCombineMaxG];   // per (segment, head): m, then the weight
+  __shared__ float l_s[kCombineBatch * kCombineMaxG];
+  __shared__ float run_M[kCombineMaxG], run_L[kCombineMaxG], run_scale[kCombineMaxG];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  float acc = 0.f;
-  if (threadIdx.x < 2) { run_M[threadIdx.x] = -INFINITY; run_L[threadIdx.x] = 0.f; }
-  const int64_t ncand = (wl - wf + 1) * kSegPerShare;
-  for (int64_t base = 0; base < ncand; base += blockDim.x) {
+  constexpr int kMaxElems = kCombineMaxG * 128 / kCombineThreads;   // 8
+  float acc[kMaxElems];
+#pragma unroll
+  for (int j = 0; j < kMaxElems; ++j) acc[j] = 0.f;
+  if (threadIdx.x < kCombineMaxG) { run_M[threadIdx.x] = -INFINITY; run_L[threadIdx.x] = 0.f; }
+  // Candidate shares are listed by share index (wf..wl), or, when the row has fewer units than
+  // that (tiny launches: most shares are empty), by unit: the share holding unit ustart + j,
+  // counted once, at its first unit inside the row.
+  const bool by_unit = (wl - wf + 1) > (int64_t)cnt;
+  const int64_t ncand = (by_unit ? (int64_t)cnt : (wl - wf + 1)) * kSegPerShare;
+  for (int64_t base = 0; base < ncand; base += kCombineBatch) {
     const int64_t i = base + threadIdx.x;
     bool hit = false, whole = false;
     int32_t slot = 0;
-    if (i < ncand) {
-      const int64_t w = wf + i / kSegPerShare;
+    if (threadIdx.x < kCombineBatch && i < ncand) {
+      const int64_t j = i / kSegPerShare;
       const int k = (int)(i % kSegPerShare);
+      int64_t w;
+      bool counted = true;
+      if (by_unit) {
+        w = worker_of(U, ustart + j, p.num_workers);
+        counted = j == 0 || worker_of(U, ustart + j - 1, p.num_workers) != w;
+      } else {
+        w = wf + j;
+      }
       int64_t a, bnd;
       segment_bounds(U, p.num_workers, w, k, a, bnd);
-      hit = a < bnd && a < uend && bnd > ustart;
+      hit = counted && a < bnd && a < uend && bnd > ustart;
       whole = hit && a <= ustart && bnd >= uend;
       slot = (int32_t)(2 * (w * kSegPerShare + k) + (a >= ustart ? 0 : 1));
     }
@@ -741,66 +779,71 @@ __global__ void combine_kernel(CombineParams p) {
     __syncthreads();
     int pos = __popc(bal & ((1u << lane) - 1u));
     int nseg = 0;
-    for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < kCombineBatch / 32; ++j) {
       if (j < warp) pos += warp_cnt[j];
       nseg += warp_cnt[j];
     }
     if (hit) seg_slot[pos] = slot;
     __syncthreads();
-    for (int idx = threadIdx.x; idx < nseg * nh; idx += blockDim.x) {   // stage (m, l): independent loads
-      const int sgm = idx / nh, hh = idx - sgm * nh;
-      const float* sp = p.partials + (int64_t)seg_slot[sgm] * stride + G * D;
-      w_s[sgm * 2 + hh] = sp[h_first + hh];
-      l_s[sgm * 2 + hh] = sp[G + h_first + hh];
+    for (int idx = threadIdx.x; idx < nseg * G; idx += kCombineThreads) {   // stage (m, l): independent loads
+      const int sgm = idx / G, h = idx - sgm * G;
+      const float* sp = p.partials + (int64_t)seg_slot[sgm] * stride + GD;
+      w_s[idx] = sp[h];
+      l_s[idx] = sp[G + h];
     }
     __syncthreads();
-    if (warp < nh) {                              // one warp per head: max, weights, weighted sum of l
-      const int hh = warp;
-      float Mc = run_M[hh];
-      for (int sgm = lane; sgm < nseg; sgm += 32) Mc = fmaxf(Mc, w_s[sgm * 2 + hh]);
+    for (int h = warp; h < G; h += kCombineThreads / 32) {   // a warp per head: max, weights, sum of l
+      float Mc = run_M[h];
+      for (int sgm = lane; sgm < nseg; sgm += 32) Mc = fmaxf(Mc, w_s[sgm * G + h]);
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) Mc = fmaxf(Mc, __shfl_xor_sync(0xffffffffu, Mc, o));
       float Lc = 0.f;
       for (int sgm = lane; sgm < nseg; sgm += 32) {
-        const float wgt = exp2f(w_s[sgm * 2 + hh] - Mc);
-        w_s[sgm * 2 + hh] = wgt;
-        Lc += wgt * l_s[sgm * 2 + hh];
+        const float wgt = exp2f(w_s[sgm * G + h] - Mc);
+        w_s[sgm * G + h] = wgt;
+        Lc += wgt * l_s[sgm * G + h];
       }
 #pragma unroll
       for (int o = 16; o > 0; o >>= 1) Lc += __shfl_xor_sync(0xffffffffu, Lc, o);
       if (lane == 0) {
-        const float sc = exp2f(run_M[hh] - Mc);   // 0 on the first batch (run_M = -inf)
-        run_L[hh] = run_L[hh] * sc + Lc;
-        run_M[hh] = Mc;
-        run_scale[hh] = sc;
+        const float sc = exp2f(run_M[h] - Mc);    // 0 on the first batch (run_M = -inf)
+        run_L[h] = run_L[h] * sc + Lc;
+        run_M[h] = Mc;
+        run_scale[h] = sc;
       }
     }
     __syncthreads();
-    if (valid) {
-      const int hh = h - h_first;
-      const float* pe = p.partials + e;
-      float a[8];
-      a[0] = acc * run_scale[hh];
 #pragma unroll
-      for (int j = 1; j < 8; ++j) a[j] = 0.f;
-      int sgm = 0;
-      for (; sgm + 8 <= nseg; sgm += 8) {         // eight independent loads in flight
-        float o[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) o[j] = pe[(int64_t)seg_slot[sgm + j] * stride];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) a[j] += w_s[(sgm + j) * 2 + hh] * o[j];
+    for (int j = 0; j < kMaxElems; ++j) {
+      const int e = threadIdx.x + j * kCombineThreads;
+      if (e < GD) {
+        const int h = e / D;
+        const float* pe = p.partials + e;
+        float a0 = acc[j] * run_scale[h], a1 = 0.f, a2 = 0.f, a3 = 0.f;
+        int sgm = 0;
+        for (; sgm + 4 <= nseg; sgm += 4) {       // four independent loads per element, kMaxElems elements
+          const float o0 = pe[(int64_t)seg_slot[sgm] * stride], o1 = pe[(int64_t)seg_slot[sgm + 1] * stride];
+          const float o2 = pe[(int64_t)seg_slot[sgm + 2] * stride], o3 = pe[(int64_t)seg_slot[sgm + 3] * stride];
+          a0 += w_s[sgm * G + h] * o0;
+          a1 += w_s[(sgm + 1) * G + h] * o1;
+          a2 += w_s[(sgm + 2) * G + h] * o2;
+          a3 += w_s[(sgm + 3) * G + h] * o3;
+        }
+        for (; sgm < nseg; ++sgm) a0 += w_s[sgm * G + h] * pe[(int64_t)seg_slot[sgm] * stride];
+        acc[j] = (a0 + a1) + (a2 + a3);
       }
-      for (; sgm < nseg; ++sgm) a[0] += w_s[sgm * 2 + hh] * pe[(int64_t)seg_slot[sgm] * stride];
-      acc = ((a[0] + a[1]) + (a[2] + a[3])) + ((a[4] + a[5]) + (a[6] + a[7]));
     }
     __syncthreads();
   }
-  if (valid) {
-    const int hh = h - h_first;
-    const float Lh = run_L[hh];
-    ob[e] = __float2bfloat16_rn(Lh > 0.f ? acc / Lh : 0.f);
-    if (lse_row && e == h * D) lse_row[h] = Lh > 0.f ? (run_M[hh] + log2f(Lh)) * 0.6931471805599453f : -INFINITY;
+#pragma unroll
+  for (int j = 0; j < kMaxElems; ++j) {
+    const int e = threadIdx.x + j * kCombineThreads;
+    if (e < GD) {
+      const int h = e / D;
+      const float Lh = run_L[h];
+      ob[e] = __float2bfloat16_rn(Lh > 0.f ? acc[j] / Lh : 0.f);
+      if (lse_row && e == h * D) lse_row[h] = Lh > 0.f ? (run_M[h] + log2f(Lh)) * 0.6931471805599453f : -INFINITY;
+    }
   }
 }
 
