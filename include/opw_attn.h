@@ -196,6 +196,43 @@ opw_status_t opw_attn_stage_set_trace(opw_attn_stage_t *stage, void *trace, size
 /* Kernels launched through this handle since create (the library's own count). */
 int64_t opw_attn_stage_launch_count(const opw_attn_stage_t *stage);
 
+/*
+ * Decode attention without any allocation, for callers that cannot obtain device memory.
+ * (The paper has no counterpart: this entry point exists for deployment reasons only.)
+ *
+ * Some callers of this library are not allowed to call cudaMalloc, and so cannot provide the
+ * workspace a stage needs: a plug-in inside a serving process whose device memory is owned
+ * and fully pre-sized by the host framework, code running after the memory budget has been
+ * spent, a latency-critical path that must never take the allocator's lock.  This variant
+ * needs no stage handle and no workspace.  It computes exactly what opw_decode_attention
+ * computes (same arguments, same conventions, same layout of kv_pool), with the split-KV
+ * scratch held in a fixed array inside the library: about 10.7 MB of device memory on every
+ * GPU that loads the library, from load until the process exits, used or not.
+ *
+ * Limits (OPW_ERR_CAPACITY beyond them, nothing is launched): batch <= 4096;
+ * (Hq/Hkv) * (head_dim + 2) <= 1040, i.e. a group of at most 8 query heads per KV head at
+ * head_dim 128; a device with at most 160 SMs.  head_dim 64 or 128 and page_size 16, else
+ * OPW_ERR_UNSUPPORTED.  It calls no cudaMalloc, cudaFree or allocating library routine.
+ *
+ * The device that holds the buffers must be the current device.  The first call on a device
+ * also resolves the scratch array's device address and sets kernel attributes; make that
+ * first call outside any stream capture.  All calls on a device share the one array, which
+ * keeps the previous call's contents (each call clears the words that must start at zero and
+ * overwrites what it later reads): two calls whose kernels may overlap on the GPU -- on
+ * different streams, or from different host threads -- race on it and must be serialised by
+ * the caller.  It runs the split-KV kernel with equal static shares only, so it is somewhat
+ * slower than a stage on long contexts.  Bad page ids are masked out as in
+ * opw_decode_attention, but there is no status word to poll.
+ *   kv_pool : DEVICE, one layer's pool (layout at the top of this file), 128-byte aligned
+ *   q, kv_lens, page_table, out, lse : as for opw_decode_attention (lse may be NULL)
+ *   window : 0 = full attention, W > 0 = the last W keys; softmax_scale 0 -> 1/sqrt(head_dim)
+ */
+opw_status_t opw_decode_attention_noalloc(int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim,
+                                          int32_t page_size, int32_t window, float softmax_scale,
+                                          const void *kv_pool, int64_t num_pages, int32_t batch,
+                                          int32_t max_pages_per_seq, const void *q, const int32_t *kv_lens,
+                                          const int32_t *page_table, void *out, float *lse, void *cuda_stream);
+
 /* Frees the host-side handle.  Does not touch device memory.  NULL is accepted. */
 opw_status_t opw_attn_stage_destroy(opw_attn_stage_t *stage);
 

@@ -15,7 +15,7 @@ from typing import Optional, Sequence
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 LIB_PATH = os.path.join(_HERE, "libopw_attn.so")
-SOURCES = [os.path.join(_HERE, "csrc", "opw_attn.cu")]
+SOURCES = [os.path.join(_HERE, "csrc", "opw_attn.cu"), os.path.join(_HERE, "csrc", "opw_noalloc.cu")]
 HEADERS = [os.path.join(_HERE, "csrc", "opw_kernels.cuh"), os.path.join(_ROOT, "include", "opw_attn.h")]
 
 OPW_FLAG_PDL = 1
@@ -25,6 +25,7 @@ EXPORTS = [
     "opw_kv_pool_index", "opw_kv_pool_bytes", "opw_attn_stage_workspace_bytes", "opw_attn_stage_create",
     "opw_kv_append", "opw_decode_attention", "opw_decode_step_host", "opw_attn_stage_poll_error",
     "opw_attn_stage_launch_count", "opw_attn_stage_destroy", "opw_status_string", "opw_attn_stage_set_trace",
+    "opw_decode_attention_noalloc",
 ]
 
 
@@ -107,6 +108,9 @@ def lib() -> ctypes.CDLL:
     L.opw_attn_stage_poll_error.argtypes = [vp, vp]
     L.opw_attn_stage_set_trace.restype = ctypes.c_int
     L.opw_attn_stage_set_trace.argtypes = [vp, vp, ctypes.c_size_t, ctypes.POINTER(i32)]
+    L.opw_decode_attention_noalloc.restype = ctypes.c_int
+    L.opw_decode_attention_noalloc.argtypes = [i32, i32, i32, i32, i32, ctypes.c_float, vp, i64, i32, i32, vp, vp, vp, vp,
+                                               vp, vp]
     L.opw_attn_stage_launch_count.restype = i64
     L.opw_attn_stage_launch_count.argtypes = [vp]
     L.opw_attn_stage_destroy.restype = ctypes.c_int
@@ -197,6 +201,18 @@ def opw_decode_step_host(stage: int, layer: int, batch: int, q_host: int, k_new_
                          lse_host: Optional[int] = None, stream: Optional[int] = None) -> None:
     _check(lib().opw_decode_step_host(stage, layer, batch, q_host, k_new_host, v_new_host, positions_host,
                                       page_table_host, out_host, lse_host, stream), "opw_decode_step_host")
+
+
+def opw_decode_attention_noalloc(*, num_q_heads: int, num_kv_heads: int, head_dim: int, kv_pool: int, num_pages: int,
+                                 batch: int, max_pages_per_seq: int, q: int, kv_lens: int, page_table: int, out: int,
+                                 lse: Optional[int] = None, window: int = 0, softmax_scale: float = 0.0,
+                                 page_size: int = 16, stream: Optional[int] = None) -> None:
+    """Decode attention for callers that cannot allocate: no stage, no workspace (the scratch is a
+    fixed array inside the library).  The buffers' device must be current; calls sharing a device
+    must not overlap."""
+    _check(lib().opw_decode_attention_noalloc(num_q_heads, num_kv_heads, head_dim, page_size, window, softmax_scale,
+                                              kv_pool, num_pages, batch, max_pages_per_seq, q, kv_lens, page_table,
+                                              out, lse, stream), "opw_decode_attention_noalloc")
 
 
 def opw_attn_stage_poll_error(stage: int, stream: Optional[int] = None) -> int:

@@ -20,7 +20,13 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-namespace opw {
+// A second translation unit may instantiate these kernels under another namespace with
+// another OPW_DYN_PER_SHARE; the defaults below are the library's main path.
+#ifndef OPW_NAMESPACE
+#define OPW_NAMESPACE opw
+#endif
+
+namespace OPW_NAMESPACE {
 
 constexpr int kPage = 16;               // tokens per page
 constexpr uint32_t kErrBadPage = 1u;    // bits of the device status word
@@ -190,6 +196,8 @@ __host__ __device__ __forceinline__ int64_t dyn_cut(int k) {   // five bits per 
                         (14ull << 30) | (15ull << 35) | (16ull << 40);       // 0,4,8,10,12,13,14,15,16
 #elif OPW_DYN_PER_SHARE == 4
   const uint64_t cuts = 0ull | (8ull << 5) | (12ull << 10) | (14ull << 15) | (16ull << 20);   // 0,8,12,14,16
+#elif OPW_DYN_PER_SHARE == 0
+  const uint64_t cuts = 0ull;                                                 // static shares only
 #elif OPW_DYN_PER_SHARE == 6
   const uint64_t cuts = 0ull | (5ull << 5) | (9ull << 10) | (12ull << 15) | (14ull << 20) | (15ull << 25) |
                         (16ull << 30);                                        // 0,5,9,12,14,15,16
@@ -199,7 +207,9 @@ __host__ __device__ __forceinline__ int64_t dyn_cut(int k) {   // five bits per 
   return (int64_t)((cuts >> (5 * k)) & 31);
 }
 // Launches with fewer than eight units per worker have no dynamic chunks at all.
-__host__ __device__ __forceinline__ bool has_dynamic(int64_t U, int64_t num_workers) { return U >= 8 * num_workers; }
+__host__ __device__ __forceinline__ bool has_dynamic(int64_t U, int64_t num_workers) {
+  return kDynPerShare > 0 && U >= 8 * num_workers;
+}
 __host__ __device__ __forceinline__ void segment_bounds(int64_t U, int64_t num_workers, int64_t w, int k,
                                                         int64_t& a, int64_t& b) {
   const int64_t s0 = worker_begin(U, w, num_workers), s1 = worker_begin(U, w + 1, num_workers);
@@ -847,4 +857,4 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
   }
 }
 
-}  // namespace opw
+}  // namespace OPW_NAMESPACE
