@@ -175,6 +175,54 @@ opw_status_t opw_decode_step_host(opw_attn_stage_t *stage, int32_t layer, int32_
                                   void *cuda_stream);
 
 /*
+ * Plans: the per-token action sequence of a stage, enqueued by ONE native call (Section 6.2,
+ * "Single native submission": the complete per-rank sequence is compiled once and each token
+ * enqueues all graph launches with no host dispatch between stages and microbatches; Section 6,
+ * first paragraph: slots, shapes and buffers are static and bound once, only token, position
+ * and KV-cache metadata change between iterations).
+ *
+ * An item is one (layer, microbatch) visit: append k_new/v_new at `positions`, then attend
+ * with `kv_lens`, exactly as opw_kv_append followed by opw_decode_attention with the same
+ * arguments (k_new == v_new == NULL skips the append).  All pointers are DEVICE addresses of
+ * caller-owned static buffers: a plan binds them once, and each submission reads whatever
+ * they hold at that time (the caller refreshes q, k_new, v_new and, when pages are added, the
+ * page table between submissions, on the same stream or ordered by an event).
+ * Items run in the order given, one after the other (they share the stage's workspace).
+ *   OPW_PLAN_GRAPH   : capture the sequence into a CUDA graph at create; submit is one
+ *                      cudaGraphLaunch.  (Instantiating a graph lets the CUDA runtime allocate
+ *                      its own bookkeeping; the library's kernels still use caller memory only.)
+ *   OPW_PLAN_ADVANCE : after the last item, add 1 to every distinct positions array (entries
+ *                      >= 0) and kv_lens array (entries > 0), so that re-submitting the plan
+ *                      is the next decode step with no host work on the metadata.
+ * create validates every item on the host (same rules and codes as the step calls) and, with
+ * OPW_PLAN_GRAPH, captures on a private stream: nothing executes until submit.  A plan must be
+ * destroyed before its stage.
+ */
+typedef struct {
+  int32_t layer;
+  int32_t batch;
+  const void *q;             /* DEVICE bf16 [batch, Hq, D] */
+  const void *k_new;         /* DEVICE bf16 [batch, Hkv, D] or NULL (no append) */
+  const void *v_new;
+  int32_t *positions;        /* DEVICE int32 [batch]; required with k_new */
+  int32_t *kv_lens;          /* DEVICE int32 [batch] */
+  const int32_t *page_table; /* DEVICE int32 [batch, max_pages_per_seq] */
+  void *out;                 /* DEVICE bf16 [batch, Hq, D] */
+  float *lse;                /* DEVICE float [batch, Hq] or NULL */
+} opw_step_item_t;
+
+typedef struct opw_attn_plan opw_attn_plan_t;
+#define OPW_PLAN_GRAPH 1u
+#define OPW_PLAN_ADVANCE 2u
+
+opw_status_t opw_attn_plan_create(opw_attn_stage_t *stage, const opw_step_item_t *items, int32_t n_items,
+                                  uint32_t flags, opw_attn_plan_t **out);
+/* Enqueue one token's whole sequence on the stream (a graph launch, or the plain launches). */
+opw_status_t opw_attn_plan_submit(opw_attn_plan_t *plan, void *cuda_stream);
+/* NULL is accepted. */
+opw_status_t opw_attn_plan_destroy(opw_attn_plan_t *plan);
+
+/*
  * Synchronises the stream, then returns and clears the device status word: OPW_OK, or
  * the first of OPW_ERR_BAD_PAGE / OPW_ERR_TIMEOUT recorded by a kernel since the last
  * poll.  The only entry point that blocks.

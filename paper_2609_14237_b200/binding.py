@@ -25,7 +25,7 @@ EXPORTS = [
     "opw_kv_pool_index", "opw_kv_pool_bytes", "opw_attn_stage_workspace_bytes", "opw_attn_stage_create",
     "opw_kv_append", "opw_decode_attention", "opw_decode_step_host", "opw_attn_stage_poll_error",
     "opw_attn_stage_launch_count", "opw_attn_stage_destroy", "opw_status_string", "opw_attn_stage_set_trace",
-    "opw_decode_attention_noalloc",
+    "opw_decode_attention_noalloc", "opw_attn_plan_create", "opw_attn_plan_submit", "opw_attn_plan_destroy",
 ]
 
 
@@ -52,6 +52,24 @@ class StageConfig(ctypes.Structure):
         ("tune_ctas_per_sm", ctypes.c_int32),
         ("reserved", ctypes.c_int32),
     ]
+
+
+class StepItem(ctypes.Structure):
+    _fields_ = [
+        ("layer", ctypes.c_int32),
+        ("batch", ctypes.c_int32),
+        ("q", ctypes.c_void_p),
+        ("k_new", ctypes.c_void_p),
+        ("v_new", ctypes.c_void_p),
+        ("positions", ctypes.c_void_p),
+        ("kv_lens", ctypes.c_void_p),
+        ("page_table", ctypes.c_void_p),
+        ("out", ctypes.c_void_p),
+        ("lse", ctypes.c_void_p),
+    ]
+
+
+OPW_PLAN_GRAPH, OPW_PLAN_ADVANCE = 1, 2
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
@@ -111,6 +129,12 @@ def lib() -> ctypes.CDLL:
     L.opw_decode_attention_noalloc.restype = ctypes.c_int
     L.opw_decode_attention_noalloc.argtypes = [i32, i32, i32, i32, i32, ctypes.c_float, vp, i64, i32, i32, vp, vp, vp, vp,
                                                vp, vp]
+    L.opw_attn_plan_create.restype = ctypes.c_int
+    L.opw_attn_plan_create.argtypes = [vp, ctypes.POINTER(StepItem), i32, ctypes.c_uint32, ctypes.POINTER(vp)]
+    L.opw_attn_plan_submit.restype = ctypes.c_int
+    L.opw_attn_plan_submit.argtypes = [vp, vp]
+    L.opw_attn_plan_destroy.restype = ctypes.c_int
+    L.opw_attn_plan_destroy.argtypes = [vp]
     L.opw_attn_stage_launch_count.restype = i64
     L.opw_attn_stage_launch_count.argtypes = [vp]
     L.opw_attn_stage_destroy.restype = ctypes.c_int
@@ -213,6 +237,27 @@ def opw_decode_attention_noalloc(*, num_q_heads: int, num_kv_heads: int, head_di
     _check(lib().opw_decode_attention_noalloc(num_q_heads, num_kv_heads, head_dim, page_size, window, softmax_scale,
                                               kv_pool, num_pages, batch, max_pages_per_seq, q, kv_lens, page_table,
                                               out, lse, stream), "opw_decode_attention_noalloc")
+
+
+def opw_attn_plan_create(stage: int, items: Sequence[dict], flags: int = 0) -> int:
+    """items: dicts with layer, batch and the device addresses q, k_new, v_new, positions, kv_lens,
+    page_table, out, lse (missing / None = NULL).  Returns the plan handle."""
+    arr = (StepItem * len(items))()
+    for a, it in zip(arr, items):
+        a.layer, a.batch = it["layer"], it["batch"]
+        for k in ("q", "k_new", "v_new", "positions", "kv_lens", "page_table", "out", "lse"):
+            setattr(a, k, it.get(k))
+    h = ctypes.c_void_p()
+    _check(lib().opw_attn_plan_create(stage, arr, len(items), flags, ctypes.byref(h)), "opw_attn_plan_create")
+    return h.value
+
+
+def opw_attn_plan_submit(plan: int, stream: Optional[int] = None) -> None:
+    _check(lib().opw_attn_plan_submit(plan, stream), "opw_attn_plan_submit")
+
+
+def opw_attn_plan_destroy(plan: Optional[int]) -> None:
+    _check(lib().opw_attn_plan_destroy(plan), "opw_attn_plan_destroy")
 
 
 def opw_attn_stage_poll_error(stage: int, stream: Optional[int] = None) -> int:

@@ -405,4 +405,123 @@ opw_status_t opw_attn_stage_poll_error(opw_attn_stage_t* st, void* cuda_stream) 
   return OPW_OK;
 }
 
+// ---------------------------------------------------------------------------------------
+// Plans: the per-token sequence of a stage, submitted with one native call
+// ---------------------------------------------------------------------------------------
+}  // extern "C"
+
+struct opw_attn_plan {
+  opw_attn_stage* stage;
+  std::vector<opw_step_item_t> items;
+  uint32_t flags;
+  cudaGraph_t graph;
+  cudaGraphExec_t exec;
+  int64_t launches_per_submit;
+};
+
+namespace {
+
+// Enqueue the whole sequence on `stream`: for every item append then attention, then (with
+// OPW_PLAN_ADVANCE) one step forward for every distinct positions / kv_lens array.
+opw_status_t enqueue_plan(opw_attn_plan* pl, cudaStream_t stream) {
+  opw_attn_stage* st = pl->stage;
+  for (const opw_step_item_t& it : pl->items) {
+    if (it.k_new) {
+      opw_status_t rc = opw_kv_append(st, it.layer, it.batch, it.k_new, it.v_new, it.positions, it.page_table, stream);
+      if (rc != OPW_OK) return rc;
+    }
+    opw_status_t rc = opw_decode_attention(st, it.layer, it.batch, it.q, it.kv_lens, it.page_table, it.out, it.lse, stream);
+    if (rc != OPW_OK) return rc;
+  }
+  if (pl->flags & OPW_PLAN_ADVANCE) {
+    std::vector<const void*> done;
+    for (const opw_step_item_t& it : pl->items) {
+      int32_t* pos = it.positions;
+      int32_t* len = it.kv_lens;
+      for (const void* d : done) {
+        if (d == pos) pos = nullptr;
+        if (d == len) len = nullptr;
+      }
+      if (!pos && !len) continue;
+      if (pos) done.push_back(pos);
+      if (len) done.push_back(len);
+      if (it.batch == 0) continue;
+      opw::advance_kernel<<<(it.batch + 255) / 256, 256, 0, stream>>>(pos, len, it.batch);
+      if (cudaGetLastError() != cudaSuccess) return OPW_ERR_CUDA;
+      st->launches += 1;
+    }
+  }
+  return OPW_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+opw_status_t opw_attn_plan_create(opw_attn_stage_t* st, const opw_step_item_t* items, int32_t n_items, uint32_t flags,
+                                  opw_attn_plan_t** out) {
+  if (!st || !items || n_items < 1 || !out) return OPW_ERR_INVALID_ARG;
+  if (flags & ~(uint32_t)(OPW_PLAN_GRAPH | OPW_PLAN_ADVANCE)) return OPW_ERR_INVALID_ARG;
+  for (int i = 0; i < n_items; ++i) {
+    const opw_step_item_t& it = items[i];
+    opw_status_t rc = check_step(st, it.layer, it.batch);
+    if (rc != OPW_OK) return rc;
+    if (!it.q || !it.kv_lens || !it.page_table || !it.out) return OPW_ERR_INVALID_ARG;
+    if ((it.k_new == nullptr) != (it.v_new == nullptr)) return OPW_ERR_INVALID_ARG;
+    if (it.k_new && !it.positions) return OPW_ERR_INVALID_ARG;
+    if (((uintptr_t)it.q | (uintptr_t)it.out | (uintptr_t)it.k_new | (uintptr_t)it.v_new) % 16) return OPW_ERR_INVALID_ARG;
+    if (((uintptr_t)it.kv_lens | (uintptr_t)it.positions | (uintptr_t)it.page_table | (uintptr_t)it.lse) % 4)
+      return OPW_ERR_INVALID_ARG;
+  }
+  opw_attn_plan* pl = new (std::nothrow) opw_attn_plan();
+  if (!pl) return OPW_ERR_INVALID_ARG;
+  pl->stage = st;
+  pl->items.assign(items, items + n_items);
+  pl->flags = flags;
+  pl->graph = nullptr;
+  pl->exec = nullptr;
+  pl->launches_per_submit = 0;
+  if (flags & OPW_PLAN_GRAPH) {
+    // Capture the sequence once on a private stream; nothing runs during the capture.
+    cudaStream_t cs = nullptr;
+    const int64_t before = st->launches;
+    bool ok = cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaStreamBeginCapture(cs, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
+    opw_status_t rc = ok ? enqueue_plan(pl, cs) : OPW_ERR_CUDA;
+    if (ok) ok = cudaStreamEndCapture(cs, &pl->graph) == cudaSuccess && pl->graph != nullptr;
+    if (ok && rc == OPW_OK) ok = cudaGraphInstantiate(&pl->exec, pl->graph, 0) == cudaSuccess;
+    if (cs) cudaStreamDestroy(cs);
+    pl->launches_per_submit = st->launches - before;
+    st->launches = before;                      // captured, not launched
+    if (!ok || rc != OPW_OK) {
+      (void)cudaGetLastError();
+      if (pl->exec) cudaGraphExecDestroy(pl->exec);
+      if (pl->graph) cudaGraphDestroy(pl->graph);
+      delete pl;
+      return rc != OPW_OK ? rc : OPW_ERR_CUDA;
+    }
+  }
+  *out = pl;
+  return OPW_OK;
+}
+
+opw_status_t opw_attn_plan_submit(opw_attn_plan_t* pl, void* cuda_stream) {
+  if (!pl) return OPW_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (pl->exec) {
+    if (cudaGraphLaunch(pl->exec, stream) != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
+    pl->stage->launches += pl->launches_per_submit;
+    return OPW_OK;
+  }
+  return enqueue_plan(pl, stream);
+}
+
+opw_status_t opw_attn_plan_destroy(opw_attn_plan_t* pl) {
+  if (!pl) return OPW_OK;
+  if (pl->exec) cudaGraphExecDestroy(pl->exec);
+  if (pl->graph) cudaGraphDestroy(pl->graph);
+  delete pl;
+  return OPW_OK;
+}
+
 }  // extern "C"

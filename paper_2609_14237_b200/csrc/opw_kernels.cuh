@@ -249,6 +249,16 @@ __global__ void kv_append_kernel(AppendParams p) {
   }
 }
 
+// One decode step further: positions and kv_lens of active rows grow by one (plans that
+// replay a captured step sequence keep their metadata on the device).
+__global__ void advance_kernel(int32_t* positions, int32_t* kv_lens, int32_t n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) {
+    if (positions && positions[i] >= 0) positions[i] += 1;
+    if (kv_lens && kv_lens[i] > 0) kv_lens[i] += 1;
+  }
+}
+
 // kv_lens = positions + 1 for the host-buffer step (inactive rows become 0)
 __global__ void lens_from_positions_kernel(const int32_t* pos, int32_t* lens, int32_t n) {
   const int i = blockIdx.x * blockDim.x + threadIdx.x;

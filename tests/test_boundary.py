@@ -124,6 +124,15 @@ def test_step_calls_reject_a_null_handle_and_destroy_accepts_it():
     assert L.opw_attn_stage_destroy(None) == B.OPW_OK
 
 
+def test_plan_calls_reject_null_arguments():
+    L = B.lib()
+    h = ctypes.c_void_p()
+    assert L.opw_attn_plan_create(None, None, 1, 0, ctypes.byref(h)) == B.OPW_ERR_INVALID_ARG and h.value is None
+    assert L.opw_attn_plan_submit(None, None) == B.OPW_ERR_INVALID_ARG
+    assert L.opw_attn_plan_destroy(None) == B.OPW_OK
+    assert ctypes.sizeof(B.StepItem) == 72
+
+
 def test_without_a_device_create_fails_loudly_instead_of_falling_back():
     import torch
 

@@ -328,6 +328,62 @@ def test_host_buffer_step_matches_the_device_step():
     st.close()
 
 
+@pytest.mark.parametrize("flags", [0, B.OPW_PLAN_GRAPH, B.OPW_PLAN_GRAPH | B.OPW_PLAN_ADVANCE, B.OPW_PLAN_ADVANCE])
+def test_plan_submits_a_multi_layer_multi_microbatch_step_in_one_call(flags):
+    """Two layers (one windowed) x two microbatches, three decode steps, one native call per step."""
+    wl = synth.Workload("p", 6, 32, 8, 128, [0, 48], "uniform_1024_4096", 78)
+    lens = np.array([5, 200, 1023, 64, 15, 3000], np.int32)
+    inp = synth.make_inputs(wl, device="cpu", growth=3, steps=3, lengths=lens)
+    pools = [p.cuda() for p in inp.pools]
+    refs = [oracle.as_u16(p).copy() for p in inp.pools]
+    st = B.Stage(pools=pools, layer_window=wl.layer_window, num_q_heads=32, num_kv_heads=8, head_dim=128,
+                 max_batch=4, max_pages_per_seq=inp.max_pages_per_seq)
+    mbs = [slice(0, 4), slice(4, 6)]                              # microbatches of 4 and 2 sequences
+    # static device buffers, bound once
+    q = [[torch.empty(mb.stop - mb.start, 32, 128, dtype=torch.bfloat16, device="cuda") for mb in mbs] for _ in range(2)]
+    k = [[torch.empty(mb.stop - mb.start, 8, 128, dtype=torch.bfloat16, device="cuda") for mb in mbs] for _ in range(2)]
+    v = [[torch.empty_like(t) for t in row] for row in k]
+    out = [[torch.empty_like(t) for t in row] for row in q]
+    lse = [[torch.empty(mb.stop - mb.start, 32, dtype=torch.float32, device="cuda") for mb in mbs] for _ in range(2)]
+    pos = [dev(lens[mb]) for mb in mbs]
+    kvl = [dev(lens[mb] + 1) for mb in mbs]
+    tabs = [[inp.page_tables[l][mb].contiguous().cuda() for mb in mbs] for l in range(2)]
+    items = []
+    for m, mb in enumerate(mbs):
+        for l in range(2):
+            items.append(dict(layer=l, batch=mb.stop - mb.start, q=q[l][m].data_ptr(), k_new=k[l][m].data_ptr(),
+                              v_new=v[l][m].data_ptr(), positions=pos[m].data_ptr(), kv_lens=kvl[m].data_ptr(),
+                              page_table=tabs[l][m].data_ptr(), out=out[l][m].data_ptr(), lse=lse[l][m].data_ptr()))
+    plan = B.opw_attn_plan_create(st.handle, items, flags)
+    stream = torch.cuda.current_stream().cuda_stream
+    for step in range(3):
+        for m, mb in enumerate(mbs):
+            for l in range(2):
+                q[l][m].copy_(inp.q[step, l][mb])
+                k[l][m].copy_(inp.k_new[step, l][mb])
+                v[l][m].copy_(inp.v_new[step, l][mb])
+            if not flags & B.OPW_PLAN_ADVANCE:                    # the caller moves the metadata itself
+                pos[m].copy_(torch.from_numpy(inp.positions(step)[mb]))
+                kvl[m].copy_(torch.from_numpy(inp.kv_lens(step)[mb]))
+        before = st.launch_count()
+        B.opw_attn_plan_submit(plan, stream)
+        assert st.poll_error() == B.OPW_OK
+        assert st.launch_count() - before == 4 * 3 + (2 if flags & B.OPW_PLAN_ADVANCE else 0)
+        for l in range(2):
+            assert oracle.kv_append(refs[l], 8, 128, P, inp.k_new[step, l], inp.v_new[step, l], inp.positions(step),
+                                    inp.page_tables[l]) == 0
+            assert (pools[l].cpu().view(torch.int16).numpy().view(np.uint16) == refs[l]).all()
+            ref, ref_lse, _ = oracle.decode_attention(refs[l], 32, 8, 128, P, inp.q[step, l], inp.kv_lens(step),
+                                                      inp.page_tables[l], window=wl.layer_window[l])
+            got = torch.cat([out[l][m] for m in range(2)])
+            got_lse = torch.cat([lse[l][m] for m in range(2)])
+            check_close(out_to_f64(got), ref, got_lse.cpu().numpy().astype(np.float64), ref_lse)
+    if flags & B.OPW_PLAN_ADVANCE:
+        assert (pos[0].cpu().numpy() == lens[mbs[0]] + 3).all() and (kvl[1].cpu().numpy() == lens[mbs[1]] + 4).all()
+    B.opw_attn_plan_destroy(plan)
+    st.close()
+
+
 def test_step_calls_validate_arguments_on_the_host():
     pool = torch.zeros(4 * 2 * 2 * 16 * 64, dtype=torch.bfloat16, device="cuda")
     st = B.Stage(pools=[pool], layer_window=[0], num_q_heads=8, num_kv_heads=2, head_dim=64, max_batch=2, max_pages_per_seq=2)
