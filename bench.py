@@ -128,7 +128,7 @@ def build_stage(wl, rotate, total_rounds, device, tune):
     return wl_r, inp, st, pos_all, len_all
 
 
-def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, world=1, rank=0):
+def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, world=1, rank=0, want_submit=False):
     import torch
 
     from paper_2609_14237_b200 import binding, synth
@@ -139,6 +139,8 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
     R = wl.num_layers if stack else rotate
     e2e_steps = max(3, min(steps, 200)) if want_e2e else 0
     n_timed = warmup + steps + (e2e_steps + 3 if want_e2e else 0)
+    n_used = n_timed                                 # steps the call-by-call and host-buffer loops take
+    n_timed += (steps + 8) if want_submit else 0     # room in the page tables for the plan's submissions
     rounds = n_timed if stack else (n_timed + R - 1) // R
     wl_r, inp, st, pos_all, len_all = build_stage(wl, R, rounds, dev, tune)
     B, Hq, Hkv, D = wl.batch, wl.num_q_heads, wl.num_kv_heads, wl.head_dim
@@ -268,6 +270,45 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
         res["e2e"] = {"value": round(world * e_bytes / (e_ms * 1e-3) / 1e9, 1), "unit": "GB/s", "steps": e2e_steps,
                       "ms_per_step": round(e_ms / e2e_steps, 5), "h2d_bytes_per_step": int(h2d),
                       "d2h_bytes_per_step": int(d2h)}
+    if want_submit:
+        # The same steps through a plan: one native call (one CUDA graph launch) per pass over
+        # the stage's layers, metadata advanced on the device.
+        t_now = n_used if stack else (n_used + R - 1) // R       # first length not yet appended in any pool
+        gpos = pos_all[t_now].clone()
+        glen = len_all[t_now].clone()
+        room = int(pos_all.shape[0] - 1 - t_now)                 # decode steps the page tables still cover
+        items = [dict(layer=l, batch=B, q=inp.q[0, l].data_ptr(), k_new=inp.k_new[0, l].data_ptr(),
+                      v_new=inp.v_new[0, l].data_ptr(), positions=gpos.data_ptr(), kv_lens=glen.data_ptr(),
+                      page_table=inp.page_tables[l].data_ptr(), out=out.data_ptr()) for l in range(R)]
+        plan = binding.opw_attn_plan_create(st.handle, items, binding.OPW_PLAN_GRAPH | binding.OPW_PLAN_ADVANCE)
+        n_sub = max(2, min(room - 3, max(steps // R, 10) if not stack else steps))
+        if n_sub >= 2:
+            for _ in range(min(3, room - n_sub)):
+                binding.opw_attn_plan_submit(plan, stream.cuda_stream)
+            torch.cuda.synchronize()
+            first_len = glen.cpu().numpy().astype(np.int64)
+            barrier()
+            host = 0.0
+            t0.record(stream)
+            for _ in range(n_sub):
+                h0 = time.perf_counter()
+                binding.opw_attn_plan_submit(plan, stream.cuda_stream)
+                host += time.perf_counter() - h0
+            t1.record(stream)
+            torch.cuda.synchronize()
+            s_ms = t0.elapsed_time(t1)
+            assert st.poll_error() == binding.OPW_OK
+            s_bytes = 0
+            for i in range(n_sub):
+                n_i = first_len + i
+                for l in range(R):
+                    w = wl_r.layer_window[l]
+                    s_bytes += int((np.minimum(n_i, w) if w > 0 else n_i).sum()) * wl.kv_bytes_per_token
+            res["submit"] = {"mode": "plan: CUDA graph + on-device advance", "value": round(s_bytes / (s_ms * 1e-3) / 1e9, 1),
+                             "unit": "GB/s", "submits": n_sub, "layer_steps_per_submit": R,
+                             "ms_per_layer_step": round(s_ms / (n_sub * R), 5),
+                             "host_us_per_submit": round(host / n_sub * 1e6, 2)}
+        binding.opw_attn_plan_destroy(plan)
     if want_cpu:
         res["cpu_baseline"] = cpu_baseline(name, inp, budget_s=15.0)
     st.close()
@@ -405,7 +446,7 @@ def main():
     warmup = args.warmup if args.warmup is not None else 20
     tune = dict(tune_warps=args.warps, tune_stages=args.stages, tune_ctas_per_sm=args.ctas,
                 flags=1 if args.pdl else 0)
-    res = run_ours(args.workload, steps, max(3, warmup), args.rotate, tune, want_e2e=not args.no_e2e,
+    res = run_ours(args.workload, steps, max(3, warmup), args.rotate, tune, want_e2e=not args.no_e2e, want_submit=(world == 1),
                    want_cpu=(world == 1 and rank == 0 and not args.no_cpu), world=world, rank=rank)
     if world == 1 and args.others:
         others = {}
@@ -419,9 +460,9 @@ def main():
                 k = max(10, min(steps, 100))
             else:
                 k = max(10, min(steps, 1000))
-            r = run_ours(name, k, max(3, min(warmup, 10)), args.rotate, tune, want_e2e=False)
+            r = run_ours(name, k, max(3, min(warmup, 10)), args.rotate, tune, want_e2e=False, want_submit=True)
             others[name] = {key: r[key] for key in ("value", "unit", "ms_per_step", "seq_steps_per_s_per_layer",
-                                                    "pct_of_nominal_8000", "roofline", "steps")}
+                                                    "pct_of_nominal_8000", "roofline", "steps", "submit") if key in r}
             others[name]["kv_bytes_per_step"] = r["config"]["kv_bytes_per_step"]
         res["other_workloads"] = others
     if world > 1:
