@@ -128,7 +128,8 @@ def build_stage(wl, rotate, total_rounds, device, tune):
     return wl_r, inp, st, pos_all, len_all
 
 
-def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, world=1, rank=0, want_submit=False):
+def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, world=1, rank=0, want_submit=False,
+             unfused=False):
     import torch
 
     from paper_2609_14237_b200 import binding, synth
@@ -157,11 +158,18 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
     def device_step(s, events=None):
         layers, t = layer_round(s)
         for l in layers:
-            st.kv_append(l, inp.k_new[s & 1, l], inp.v_new[s & 1, l], pos_all[t], inp.page_tables[l])
             if events is not None:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                e0.record(stream)
-            st.decode_attention(l, inp.q[s & 1, l], len_all[t], inp.page_tables[l], out)
+            if unfused:
+                st.kv_append(l, inp.k_new[s & 1, l], inp.v_new[s & 1, l], pos_all[t], inp.page_tables[l])
+                if events is not None:
+                    e0.record(stream)
+                st.decode_attention(l, inp.q[s & 1, l], len_all[t], inp.page_tables[l], out)
+            else:                                   # append fused into the attention kernel: two launches
+                if events is not None:
+                    e0.record(stream)
+                st.decode_step(l, inp.q[s & 1, l], inp.k_new[s & 1, l], inp.v_new[s & 1, l], pos_all[t],
+                               inp.page_tables[l], out)
             if events is not None:
                 e1.record(stream)
                 events.append((e0, e1))
@@ -224,7 +232,9 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
         "pct_of_nominal_8000": round(100 * value / world / NOMINAL_HBM_GBS, 2),
         "roofline": {"bound": "hbm", "achieved": round(achieved, 1), "peak": peak, "unit": "GB/s",
                      "frac": round(achieved / peak, 4), "peak_kind": peak_kind,
-                     "kernel": "attn_splitkv_kernel (+ combine_kernel, timed together per opw_decode_attention call)",
+                     "kernel": ("attn_splitkv_kernel (+ combine_kernel, timed together per opw_decode_attention call)"
+                                if unfused else
+                                "attn_splitkv_kernel with fused append (+ combine_kernel, timed together per opw_decode_step call)"),
                      "kernel_ms": round(attn_avg_ms, 5),
                      "traffic": None if ratio is None else int(ratio * attn_bytes_per_launch)},
         "gpu_launches": int(launches), "clocks": clocks,
@@ -278,7 +288,8 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
         glen = len_all[t_now].clone()
         room = int(pos_all.shape[0] - 1 - t_now)                 # decode steps the page tables still cover
         items = [dict(layer=l, batch=B, q=inp.q[0, l].data_ptr(), k_new=inp.k_new[0, l].data_ptr(),
-                      v_new=inp.v_new[0, l].data_ptr(), positions=gpos.data_ptr(), kv_lens=glen.data_ptr(),
+                      v_new=inp.v_new[0, l].data_ptr(), positions=gpos.data_ptr(),
+                      kv_lens=glen.data_ptr() if unfused else None,
                       page_table=inp.page_tables[l].data_ptr(), out=out.data_ptr()) for l in range(R)]
         plan = binding.opw_attn_plan_create(st.handle, items, binding.OPW_PLAN_GRAPH | binding.OPW_PLAN_ADVANCE)
         n_sub = max(2, min(room - 3, max(steps // R, 10) if not stack else steps))
@@ -286,7 +297,7 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
             for _ in range(min(3, room - n_sub)):
                 binding.opw_attn_plan_submit(plan, stream.cuda_stream)
             torch.cuda.synchronize()
-            first_len = glen.cpu().numpy().astype(np.int64)
+            first_len = gpos.cpu().numpy().astype(np.int64) + 1
             barrier()
             host = 0.0
             t0.record(stream)
@@ -417,6 +428,7 @@ def main():
     ap.add_argument("--warps", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--ctas", type=int, default=0)
+    ap.add_argument("--unfused", action="store_true", help="separate opw_kv_append + opw_decode_attention calls")
     ap.add_argument("--pdl", action="store_true", help="launch the kernels with programmatic stream serialisation")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -446,7 +458,7 @@ def main():
     warmup = args.warmup if args.warmup is not None else 20
     tune = dict(tune_warps=args.warps, tune_stages=args.stages, tune_ctas_per_sm=args.ctas,
                 flags=1 if args.pdl else 0)
-    res = run_ours(args.workload, steps, max(3, warmup), args.rotate, tune, want_e2e=not args.no_e2e, want_submit=(world == 1),
+    res = run_ours(args.workload, steps, max(3, warmup), args.rotate, tune, want_e2e=not args.no_e2e, want_submit=(world == 1), unfused=args.unfused,
                    want_cpu=(world == 1 and rank == 0 and not args.no_cpu), world=world, rank=rank)
     if world == 1 and args.others:
         others = {}
@@ -460,7 +472,8 @@ def main():
                 k = max(10, min(steps, 100))
             else:
                 k = max(10, min(steps, 1000))
-            r = run_ours(name, k, max(3, min(warmup, 10)), args.rotate, tune, want_e2e=False, want_submit=True)
+            r = run_ours(name, k, max(3, min(warmup, 10)), args.rotate, tune, want_e2e=False, want_submit=True,
+                         unfused=args.unfused)
             others[name] = {key: r[key] for key in ("value", "unit", "ms_per_step", "seq_steps_per_s_per_layer",
                                                     "pct_of_nominal_8000", "roofline", "steps", "submit") if key in r}
             others[name]["kv_bytes_per_step"] = r["config"]["kv_bytes_per_step"]

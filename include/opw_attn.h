@@ -160,10 +160,23 @@ opw_status_t opw_decode_attention(opw_attn_stage_t *stage, int32_t layer, int32_
                                   void *cuda_stream);
 
 /*
+ * Append and attention in one call, and in one kernel fewer: exactly opw_kv_append(k_new,
+ * v_new, positions) followed by opw_decode_attention with kv_lens[b] = positions[b] + 1
+ * (0 for positions[b] < 0), but the new rows are stored by the attention kernel itself --
+ * the warp that streams the last page of sequence b and kv head g writes k_new[b,g,:] and
+ * v_new[b,g,:] into the pool and into its shared-memory copy of that page -- so no separate
+ * append launch and no dependency on one.  Same argument rules, the same bit-exact pool
+ * contents afterwards and the same status-word reporting as the two calls.
+ */
+opw_status_t opw_decode_step(opw_attn_stage_t *stage, int32_t layer, int32_t batch, const void *q,
+                             const void *k_new, const void *v_new, const int32_t *positions,
+                             const int32_t *page_table, void *out, float *lse, void *cuda_stream);
+
+/*
  * One whole stage step from HOST buffers (Section 4: the stage's activation interface
  * is the per-request q/k/v in and attention output back): copies q, k_new, v_new,
- * positions and (if not NULL) page_table to staging areas in the workspace, runs the
- * append and the attention with kv_lens = positions + 1, and copies out (and lse if
+ * positions and (if not NULL) page_table to staging areas in the workspace, runs
+ * opw_decode_step on them, and copies out (and lse if
  * not NULL) back to the host, all enqueued on the stream.  Host buffers should be
  * pinned for the copies to be asynchronous; they must stay valid and unmodified until
  * the stream has passed the step.  page_table_host == NULL reuses the table staged by
@@ -183,7 +196,8 @@ opw_status_t opw_decode_step_host(opw_attn_stage_t *stage, int32_t layer, int32_
  *
  * An item is one (layer, microbatch) visit: append k_new/v_new at `positions`, then attend
  * with `kv_lens`, exactly as opw_kv_append followed by opw_decode_attention with the same
- * arguments (k_new == v_new == NULL skips the append).  All pointers are DEVICE addresses of
+ * arguments (k_new == v_new == NULL skips the append; kv_lens == NULL with k_new set means
+ * kv_lens = positions + 1 and runs the fused opw_decode_step).  All pointers are DEVICE addresses of
  * caller-owned static buffers: a plan binds them once, and each submission reads whatever
  * they hold at that time (the caller refreshes q, k_new, v_new and, when pages are added, the
  * page table between submissions, on the same stream or ordered by an event).
@@ -205,7 +219,7 @@ typedef struct {
   const void *k_new;         /* DEVICE bf16 [batch, Hkv, D] or NULL (no append) */
   const void *v_new;
   int32_t *positions;        /* DEVICE int32 [batch]; required with k_new */
-  int32_t *kv_lens;          /* DEVICE int32 [batch] */
+  int32_t *kv_lens;          /* DEVICE int32 [batch], or NULL with k_new: positions + 1 */
   const int32_t *page_table; /* DEVICE int32 [batch, max_pages_per_seq] */
   void *out;                 /* DEVICE bf16 [batch, Hq, D] */
   float *lse;                /* DEVICE float [batch, Hq] or NULL */

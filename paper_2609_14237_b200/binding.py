@@ -26,6 +26,7 @@ EXPORTS = [
     "opw_kv_append", "opw_decode_attention", "opw_decode_step_host", "opw_attn_stage_poll_error",
     "opw_attn_stage_launch_count", "opw_attn_stage_destroy", "opw_status_string", "opw_attn_stage_set_trace",
     "opw_decode_attention_noalloc", "opw_attn_plan_create", "opw_attn_plan_submit", "opw_attn_plan_destroy",
+    "opw_decode_step",
 ]
 
 
@@ -120,6 +121,8 @@ def lib() -> ctypes.CDLL:
     L.opw_kv_append.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp]
     L.opw_decode_attention.restype = ctypes.c_int
     L.opw_decode_attention.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
+    L.opw_decode_step.restype = ctypes.c_int
+    L.opw_decode_step.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     L.opw_decode_step_host.restype = ctypes.c_int
     L.opw_decode_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     L.opw_attn_stage_poll_error.restype = ctypes.c_int
@@ -218,6 +221,12 @@ def opw_decode_attention(stage: int, layer: int, batch: int, q: int, kv_lens: in
                          lse: Optional[int] = None, stream: Optional[int] = None) -> None:
     _check(lib().opw_decode_attention(stage, layer, batch, q, kv_lens, page_table, out, lse, stream),
            "opw_decode_attention")
+
+
+def opw_decode_step(stage: int, layer: int, batch: int, q: int, k_new: int, v_new: int, positions: int,
+                    page_table: int, out: int, lse: Optional[int] = None, stream: Optional[int] = None) -> None:
+    _check(lib().opw_decode_step(stage, layer, batch, q, k_new, v_new, positions, page_table, out, lse, stream),
+           "opw_decode_step")
 
 
 def opw_decode_step_host(stage: int, layer: int, batch: int, q_host: int, k_new_host: int, v_new_host: int,
@@ -329,6 +338,11 @@ class Stage:
         opw_decode_attention(self.handle, layer, kv_lens.shape[0], q.data_ptr(), kv_lens.data_ptr(),
                              page_table.data_ptr(), out.data_ptr(), None if lse is None else lse.data_ptr(),
                              self._stream())
+
+    def decode_step(self, layer, q, k_new, v_new, positions, page_table, out, lse=None):
+        opw_decode_step(self.handle, layer, positions.shape[0], q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(),
+                        positions.data_ptr(), page_table.data_ptr(), out.data_ptr(),
+                        None if lse is None else lse.data_ptr(), self._stream())
 
     def decode_step_host(self, layer, q, k_new, v_new, positions, page_table, out, lse=None):
         opw_decode_step_host(self.handle, layer, positions.shape[0], q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(),

@@ -276,13 +276,17 @@ opw_status_t opw_kv_append(opw_attn_stage_t* st, int32_t layer, int32_t batch, c
   return OPW_OK;
 }
 
-opw_status_t opw_decode_attention(opw_attn_stage_t* st, int32_t layer, int32_t batch, const void* q,
-                                  const int32_t* kv_lens, const int32_t* page_table, void* out, float* lse,
-                                  void* cuda_stream) {
+static opw_status_t enqueue_attention(opw_attn_stage_t* st, int32_t layer, int32_t batch, const void* q,
+                                      const int32_t* kv_lens, const void* k_new, const void* v_new,
+                                      const int32_t* positions, const int32_t* page_table, void* out, float* lse,
+                                      void* cuda_stream) {
   opw_status_t rc = check_step(st, layer, batch);
   if (rc != OPW_OK) return rc;
-  if (!q || !kv_lens || !page_table || !out) return OPW_ERR_INVALID_ARG;
-  if (((uintptr_t)q | (uintptr_t)out) % 16 || (uintptr_t)kv_lens % 4 || (uintptr_t)page_table % 4 || (uintptr_t)lse % 4)
+  const bool fused = k_new != nullptr;
+  if (!q || !page_table || !out) return OPW_ERR_INVALID_ARG;
+  if (fused ? (!v_new || !positions || kv_lens) : (!kv_lens || v_new || positions)) return OPW_ERR_INVALID_ARG;
+  if (((uintptr_t)q | (uintptr_t)out | (uintptr_t)k_new | (uintptr_t)v_new) % 16 || (uintptr_t)kv_lens % 4 ||
+      (uintptr_t)positions % 4 || (uintptr_t)page_table % 4 || (uintptr_t)lse % 4)
     return OPW_ERR_INVALID_ARG;
   if (batch == 0) return OPW_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -293,6 +297,10 @@ opw_status_t opw_decode_attention(opw_attn_stage_t* st, int32_t layer, int32_t b
   p.q = static_cast<const __nv_bfloat16*>(q);
   p.kv_lens = kv_lens;
   p.page_table = page_table;
+  p.k_new = static_cast<const __nv_bfloat16*>(k_new);
+  p.v_new = static_cast<const __nv_bfloat16*>(v_new);
+  p.positions = positions;
+  p.pool_w = static_cast<__nv_bfloat16*>(st->pool[layer]);
   p.out = static_cast<__nv_bfloat16*>(out);
   p.lse = lse;
   p.partials = reinterpret_cast<float*>(st->ws + st->lay.partials);
@@ -329,6 +337,7 @@ opw_status_t opw_decode_attention(opw_attn_stage_t* st, int32_t layer, int32_t b
   c.partials = p.partials;
   c.cum = p.cum;
   c.kv_lens = kv_lens;
+  c.positions = positions;
   c.out = p.out;
   c.lse = lse;
   c.batch = batch;
@@ -347,6 +356,21 @@ opw_status_t opw_decode_attention(opw_attn_stage_t* st, int32_t layer, int32_t b
   return OPW_OK;
 }
 
+
+opw_status_t opw_decode_attention(opw_attn_stage_t* st, int32_t layer, int32_t batch, const void* q,
+                                  const int32_t* kv_lens, const int32_t* page_table, void* out, float* lse,
+                                  void* cuda_stream) {
+  if (!kv_lens) return OPW_ERR_INVALID_ARG;
+  return enqueue_attention(st, layer, batch, q, kv_lens, nullptr, nullptr, nullptr, page_table, out, lse, cuda_stream);
+}
+
+opw_status_t opw_decode_step(opw_attn_stage_t* st, int32_t layer, int32_t batch, const void* q, const void* k_new,
+                             const void* v_new, const int32_t* positions, const int32_t* page_table, void* out,
+                             float* lse, void* cuda_stream) {
+  if (!k_new || !v_new || !positions) return OPW_ERR_INVALID_ARG;
+  return enqueue_attention(st, layer, batch, q, nullptr, k_new, v_new, positions, page_table, out, lse, cuda_stream);
+}
+
 opw_status_t opw_decode_step_host(opw_attn_stage_t* st, int32_t layer, int32_t batch, const void* q_host,
                                   const void* k_new_host, const void* v_new_host, const int32_t* positions_host,
                                   const int32_t* page_table_host, void* out_host, float* lse_host, void* cuda_stream) {
@@ -361,7 +385,6 @@ opw_status_t opw_decode_step_host(opw_attn_stage_t* st, int32_t layer, int32_t b
   void* d_k = ws + st->lay.st_k;
   void* d_v = ws + st->lay.st_v;
   int32_t* d_pos = reinterpret_cast<int32_t*>(ws + st->lay.st_pos);
-  int32_t* d_lens = reinterpret_cast<int32_t*>(ws + st->lay.st_lens);
   void* d_out = ws + st->lay.st_out;
   float* d_lse = reinterpret_cast<float*>(ws + st->lay.st_lse);
   const size_t table_elems = (size_t)st->cfg.max_batch * st->cfg.max_pages_per_seq;
@@ -376,13 +399,7 @@ opw_status_t opw_decode_step_host(opw_attn_stage_t* st, int32_t layer, int32_t b
     ok &= cudaMemcpyAsync(d_table, page_table_host, B * st->cfg.max_pages_per_seq * 4, cudaMemcpyHostToDevice,
                           stream) == cudaSuccess;
   if (!ok) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
-  // kv_lens = positions + 1 on the device (inactive rows become 0)
-  opw::lens_from_positions_kernel<<<(batch + 255) / 256, 256, 0, stream>>>(d_pos, d_lens, batch);
-  if (cudaGetLastError() != cudaSuccess) return OPW_ERR_CUDA;
-  st->launches += 1;
-  rc = opw_kv_append(st, layer, batch, d_k, d_v, d_pos, d_table, cuda_stream);
-  if (rc != OPW_OK) return rc;
-  rc = opw_decode_attention(st, layer, batch, d_q, d_lens, d_table, d_out, lse_host ? d_lse : nullptr, cuda_stream);
+  rc = opw_decode_step(st, layer, batch, d_q, d_k, d_v, d_pos, d_table, d_out, lse_host ? d_lse : nullptr, cuda_stream);
   if (rc != OPW_OK) return rc;
   ok &= cudaMemcpyAsync(out_host, d_out, B * Hq * D * 2, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
   if (lse_host) ok &= cudaMemcpyAsync(lse_host, d_lse, B * Hq * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
@@ -426,11 +443,17 @@ namespace {
 opw_status_t enqueue_plan(opw_attn_plan* pl, cudaStream_t stream) {
   opw_attn_stage* st = pl->stage;
   for (const opw_step_item_t& it : pl->items) {
-    if (it.k_new) {
-      opw_status_t rc = opw_kv_append(st, it.layer, it.batch, it.k_new, it.v_new, it.positions, it.page_table, stream);
-      if (rc != OPW_OK) return rc;
+    opw_status_t rc;
+    if (it.k_new && !it.kv_lens) {              // one fused launch: append inside the attention kernel
+      rc = opw_decode_step(st, it.layer, it.batch, it.q, it.k_new, it.v_new, it.positions, it.page_table, it.out,
+                           it.lse, stream);
+    } else {
+      if (it.k_new) {
+        rc = opw_kv_append(st, it.layer, it.batch, it.k_new, it.v_new, it.positions, it.page_table, stream);
+        if (rc != OPW_OK) return rc;
+      }
+      rc = opw_decode_attention(st, it.layer, it.batch, it.q, it.kv_lens, it.page_table, it.out, it.lse, stream);
     }
-    opw_status_t rc = opw_decode_attention(st, it.layer, it.batch, it.q, it.kv_lens, it.page_table, it.out, it.lse, stream);
     if (rc != OPW_OK) return rc;
   }
   if (pl->flags & OPW_PLAN_ADVANCE) {
@@ -466,7 +489,8 @@ opw_status_t opw_attn_plan_create(opw_attn_stage_t* st, const opw_step_item_t* i
     const opw_step_item_t& it = items[i];
     opw_status_t rc = check_step(st, it.layer, it.batch);
     if (rc != OPW_OK) return rc;
-    if (!it.q || !it.kv_lens || !it.page_table || !it.out) return OPW_ERR_INVALID_ARG;
+    if (!it.q || !it.page_table || !it.out) return OPW_ERR_INVALID_ARG;
+    if (!it.kv_lens && !it.k_new) return OPW_ERR_INVALID_ARG;
     if ((it.k_new == nullptr) != (it.v_new == nullptr)) return OPW_ERR_INVALID_ARG;
     if (it.k_new && !it.positions) return OPW_ERR_INVALID_ARG;
     if (((uintptr_t)it.q | (uintptr_t)it.out | (uintptr_t)it.k_new | (uintptr_t)it.v_new) % 16) return OPW_ERR_INVALID_ARG;

@@ -5,10 +5,10 @@
 // logical page) triple inside the visible range of b; units are ordered by (b, g, page)
 // and the U units of a launch are cut into equal contiguous shares, one per warp
 // ("worker") of a persistent grid.  A share is cut again into kSegPerShare segments: the
-// first 7/8 is the worker's own static segment, the last 1/8 is split into six ever
+// first 13/16 is the worker's own static segment, the last 3/16 is split into six ever
 // smaller chunks that any worker may take through an atomic ticket once its static
-// segment is done (SMs do not all stream at the same rate; the chunks even out the
-// finish times).  The segment boundaries depend only on kv_lens, the window and the grid,
+// segment is done (SMs do not all stream at the same rate -- finish times of equal static
+// shares spread by about 15 % -- and the chunks even them out).  The segment boundaries depend only on kv_lens, the window and the grid,
 // never on which warp runs a segment or on page ids, so the result is deterministic.
 // A worker streams one 2*P*D*2-byte tile (K rows then V rows of one page and head,
 // contiguous in the pool) per unit.  A segment meets at most two rows (b, g) it does not
@@ -37,8 +37,15 @@ constexpr uint64_t kWaitLimitNs = 100ull * 1000 * 1000;   // bound of a wait on 
 struct AttnParams {
   const __nv_bfloat16* pool;
   const __nv_bfloat16* q;
-  const int32_t* kv_lens;
+  const int32_t* kv_lens;      // keys visible per sequence, or null: then positions[b] + 1
   const int32_t* page_table;
+  // Fused append (all three null or all three set): the worker that streams the last page of
+  // row (b, g) also stores k_new[b,g,:] / v_new[b,g,:] into slot positions[b] of that page,
+  // in the pool and in its shared-memory copy of the tile.
+  const __nv_bfloat16* k_new;
+  const __nv_bfloat16* v_new;
+  const int32_t* positions;
+  __nv_bfloat16* pool_w;
   __nv_bfloat16* out;
   float* lse;            // may be null
   float* partials;       // [num_workers*2][G*(D+2)]
@@ -165,6 +172,12 @@ __device__ __forceinline__ float fast_exp2(float x) {
 // ---------------------------------------------------------------------------------
 // shared host/device arithmetic of the unit decomposition
 // ---------------------------------------------------------------------------------
+// keys visible to sequence b: given directly, or one more than its pre-append length
+__device__ __forceinline__ int32_t visible_keys(const int32_t* kv_lens, const int32_t* positions, int b) {
+  if (kv_lens) return kv_lens[b];
+  const int32_t pos = positions[b];
+  return pos >= 0 ? pos + 1 : 0;
+}
 // pages of sequence with n visible keys under `window` : first logical page and count
 __host__ __device__ __forceinline__ void visible_pages(int32_t n, int32_t window, int32_t max_pages,
                                                        int32_t& first, int32_t& count, int32_t& lo) {
@@ -183,10 +196,13 @@ __host__ __device__ __forceinline__ int64_t worker_begin(int64_t U, int64_t work
 __host__ __device__ __forceinline__ int64_t worker_of(int64_t U, int64_t u, int64_t num_workers) {
   return ((u + 1) * num_workers - 1) / U;
 }
-// Segments of a share: k = 0 is the static first 7/8; k = 1..kDynPerShare cut the last 1/8
-// into ever smaller chunks (cut points in sixteenths of that eighth).
+// Segments of a share: k = 0 is the static first 13/16; k = 1..kDynPerShare cut the last 3/16
+// into ever smaller chunks (cut points in sixteenths of that part).
 #ifndef OPW_DYN_PER_SHARE
 #define OPW_DYN_PER_SHARE 6
+#endif
+#ifndef OPW_DYN_32NDS
+#define OPW_DYN_32NDS 6          /* the dynamic part of a share, in 32nds: 6/32 = 3/16 */
 #endif
 constexpr int kDynPerShare = OPW_DYN_PER_SHARE;
 constexpr int kSegPerShare = kDynPerShare + 1;
@@ -213,7 +229,7 @@ __host__ __device__ __forceinline__ bool has_dynamic(int64_t U, int64_t num_work
 __host__ __device__ __forceinline__ void segment_bounds(int64_t U, int64_t num_workers, int64_t w, int k,
                                                         int64_t& a, int64_t& b) {
   const int64_t s0 = worker_begin(U, w, num_workers), s1 = worker_begin(U, w + 1, num_workers);
-  const int64_t len = s1 - s0, dyn = has_dynamic(U, num_workers) ? len >> 3 : 0, stat = len - dyn;
+  const int64_t len = s1 - s0, dyn = has_dynamic(U, num_workers) ? (len * OPW_DYN_32NDS) >> 5 : 0, stat = len - dyn;
   if (k == 0) { a = s0; b = s0 + stat; return; }
   a = s0 + stat + ((dyn * dyn_cut(k - 1)) >> 4);
   b = s0 + stat + ((dyn * dyn_cut(k)) >> 4);
@@ -311,7 +327,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
       const int b = base + threadIdx.x;
       int32_t cnt = 0, n = 0;
       if (b < p.batch) {
-        n = p.kv_lens[b];
+        n = visible_keys(p.kv_lens, p.positions, b);
         int32_t first, lo;
         if (n > p.max_pages * kPage) {            // beyond the table: clamp and record
           n = p.max_pages * kPage;
@@ -489,6 +505,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
     const int rel = (int)(u - wbase);
     const int32_t row = __shfl_sync(0xffffffffu, wa.row, rel);
     const int32_t info = __shfl_sync(0xffffffffu, wa.info, rel);
+    const int32_t this_tile = __shfl_sync(0xffffffffu, wa.tile, rel);
     const int t0 = info & 0xff, t1 = (info >> 8) & 0xff;
     const bool first = (info >> 16) & 1, last = (info >> 17) & 1;
     const int b = row / p.Hkv, g = row - b * p.Hkv;
@@ -514,6 +531,15 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
       l_lo = l_hi = 0.f;
     }
 
+    // fused append: this unit is the page that receives the step's new key/value row
+    const bool patch = p.k_new != nullptr && last && t1 > 0;
+    uint4 new_row = make_uint4(0u, 0u, 0u, 0u);
+    const int pc = lane & 15;                  // 16-byte group of the row; lanes 0..15 K, 16..31 V
+    if (patch && pc < D / 8) {
+      const __nv_bfloat16* src = (lane < 16 ? p.k_new : p.v_new) + ((int64_t)b * p.Hkv + g) * D + pc * 8;
+      new_row = *reinterpret_cast<const uint4*>(src);
+    }
+
     // wait for this unit's tile
     if (!mbar_wait_bounded(bar_base + 8 * slot, phase)) { failed = true; break; }
     --inflight;
@@ -521,6 +547,17 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
     traced_first = true;
 
     const uint32_t tile = ring_base + slot * TILE;
+    if (patch) {
+      if (pc < D / 8) {
+        const int tn = t1 - 1;                 // slot of the newest key inside this page
+        const uint32_t off = (uint32_t)((lane < 16 ? 0 : kPage * ROWB) + tn * ROWB + ((pc ^ (tn & 7)) << 4));
+        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(tile + off), "r"(new_row.x), "r"(new_row.y),
+                     "r"(new_row.z), "r"(new_row.w)
+                     : "memory");
+        *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(p.pool_w) + (int64_t)this_tile * TILE + off) = new_row;
+      }
+      __syncwarp();
+    }
     const bool ragged = (t0 > 0) || (t1 < kPage);
     if (ragged) {
       // Slots outside [t0,t1) may hold anything (never written, or stale): their scores are
@@ -711,7 +748,8 @@ struct CombineParams {
   int32_t* ticket;       // the attention kernel's chunk counter: re-zeroed here for the next launch
   const float* partials;
   const int32_t* cum;
-  const int32_t* kv_lens;
+  const int32_t* kv_lens;     // or null: then positions[b] + 1
+  const int32_t* positions;
   __nv_bfloat16* out;
   float* lse;
   int32_t batch, Hq, Hkv, G, D;
@@ -724,13 +762,51 @@ struct CombineParams {
 constexpr int kCombineThreads = 256;
 constexpr int kCombineMaxG = 16;
 constexpr int kCombineBatch = 64;               // segments merged per pass
+// acc[j] = acc[j] * scale[h] + sum over the listed partials of weight * o, for the thread's
+// elements e = tid + j * kCombineThreads.  The loads of one pass are all independent.
+template <int NEL>
+__device__ __forceinline__ void combine_accumulate(float* acc, const float* partials, const int32_t* seg_slot,
+                                                   const float* w_s, const float* run_scale, int nseg, int64_t stride,
+                                                   int G, int D, int GD) {
+  constexpr int US = 32 / NEL;
+  int hh[NEL];
+  bool ok[NEL];
+#pragma unroll
+  for (int j = 0; j < NEL; ++j) {
+    const int e = threadIdx.x + j * kCombineThreads;
+    ok[j] = e < GD;
+    hh[j] = ok[j] ? e / D : 0;
+    acc[j] *= run_scale[hh[j]];
+  }
+  int sgm = 0;
+  for (; sgm + US <= nseg; sgm += US) {
+    float o[NEL][US];
+#pragma unroll
+    for (int u = 0; u < US; ++u) {
+      const float* sp = partials + (int64_t)seg_slot[sgm + u] * stride + threadIdx.x;
+#pragma unroll
+      for (int j = 0; j < NEL; ++j) o[j][u] = ok[j] ? sp[j * kCombineThreads] : 0.f;
+    }
+#pragma unroll
+    for (int u = 0; u < US; ++u)
+#pragma unroll
+      for (int j = 0; j < NEL; ++j) acc[j] += w_s[(sgm + u) * G + hh[j]] * o[j][u];
+  }
+  for (; sgm < nseg; ++sgm) {
+    const float* sp = partials + (int64_t)seg_slot[sgm] * stride + threadIdx.x;
+#pragma unroll
+    for (int j = 0; j < NEL; ++j)
+      if (ok[j]) acc[j] += w_s[sgm * G + hh[j]] * sp[j * kCombineThreads];
+  }
+}
+
 __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams p) {
   pdl_launch_dependents();
   const int row = blockIdx.x;
   const int b = row / p.Hkv, g = row - b * p.Hkv;
   const int D = p.D, G = p.G;
   const int GD = G * D;
-  int32_t n = p.kv_lens[b];                    // an input: may be read before the attention kernel is done
+  int32_t n = visible_keys(p.kv_lens, p.positions, b);   // an input: may be read before the attention kernel is done
   pdl_wait();                                  // partials, prefix sums and complete rows are final now
   if (blockIdx.x == 0 && threadIdx.x == 0) *p.ticket = 0;
   const int32_t cum_b = p.cum[b], cum_all = p.cum[p.batch];     // independent of the load above
@@ -763,6 +839,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
   __shared__ float run_M[kCombineMaxG], run_L[kCombineMaxG], run_scale[kCombineMaxG];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   constexpr int kMaxElems = kCombineMaxG * 128 / kCombineThreads;   // 8
+  const int nel = (GD + kCombineThreads - 1) / kCombineThreads;
   float acc[kMaxElems];
 #pragma unroll
   for (int j = 0; j < kMaxElems; ++j) acc[j] = 0.f;
@@ -833,26 +910,11 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
       }
     }
     __syncthreads();
-#pragma unroll
-    for (int j = 0; j < kMaxElems; ++j) {
-      const int e = threadIdx.x + j * kCombineThreads;
-      if (e < GD) {
-        const int h = e / D;
-        const float* pe = p.partials + e;
-        float a0 = acc[j] * run_scale[h], a1 = 0.f, a2 = 0.f, a3 = 0.f;
-        int sgm = 0;
-        for (; sgm + 4 <= nseg; sgm += 4) {       // four independent loads per element, kMaxElems elements
-          const float o0 = pe[(int64_t)seg_slot[sgm] * stride], o1 = pe[(int64_t)seg_slot[sgm + 1] * stride];
-          const float o2 = pe[(int64_t)seg_slot[sgm + 2] * stride], o3 = pe[(int64_t)seg_slot[sgm + 3] * stride];
-          a0 += w_s[sgm * G + h] * o0;
-          a1 += w_s[(sgm + 1) * G + h] * o1;
-          a2 += w_s[(sgm + 2) * G + h] * o2;
-          a3 += w_s[(sgm + 3) * G + h] * o3;
-        }
-        for (; sgm < nseg; ++sgm) a0 += w_s[sgm * G + h] * pe[(int64_t)seg_slot[sgm] * stride];
-        acc[j] = (a0 + a1) + (a2 + a3);
-      }
-    }
+    // about 32 independent loads in flight per thread: NEL elements x (32 / NEL) segments
+    if (nel <= 1) combine_accumulate<1>(acc, p.partials, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
+    else if (nel <= 2) combine_accumulate<2>(acc, p.partials, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
+    else if (nel <= 4) combine_accumulate<4>(acc, p.partials, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
+    else combine_accumulate<8>(acc, p.partials, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
     __syncthreads();
   }
 #pragma unroll

@@ -25,6 +25,7 @@
 #include "opw_attn.h"
 
 #define OPW_NAMESPACE opw_na
+#undef OPW_DYN_PER_SHARE
 #define OPW_DYN_PER_SHARE 0
 #include "opw_kernels.cuh"
 
@@ -124,6 +125,10 @@ extern "C" opw_status_t opw_decode_attention_noalloc(int32_t num_q_heads, int32_
   p.q = static_cast<const __nv_bfloat16*>(q);
   p.kv_lens = kv_lens;
   p.page_table = page_table;
+  p.k_new = nullptr;                  // no fused append here
+  p.v_new = nullptr;
+  p.positions = nullptr;
+  p.pool_w = nullptr;
   p.out = static_cast<__nv_bfloat16*>(out);
   p.lse = lse;
   p.partials = reinterpret_cast<float*>(ws + kStatusBytes + kCumBytes);
@@ -159,6 +164,7 @@ extern "C" opw_status_t opw_decode_attention_noalloc(int32_t num_q_heads, int32_
   c.partials = p.partials;
   c.cum = p.cum;
   c.kv_lens = kv_lens;
+  c.positions = nullptr;
   c.out = p.out;
   c.lse = lse;
   c.batch = batch;

@@ -152,6 +152,35 @@ def test_config1_tiny_step_append_then_attention():
     st.close()
 
 
+@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 64), (32, 8, 128), (24, 2, 64)])
+def test_fused_step_appends_bit_exactly_and_attends_over_the_new_key(Hq, Hkv, D):
+    """opw_decode_step == opw_kv_append + opw_decode_attention: same pool bytes, same output."""
+    wl = synth.Workload("f", 9, Hq, Hkv, D, [0, 40], "tiny", 79)
+    lens = np.array([0, 15, 16, 255, 100, 17, 64, 2000, 31], np.int32)
+    inp = synth.make_inputs(wl, device="cpu", growth=3, steps=3, lengths=lens)
+    pools = [p.cuda() for p in inp.pools]
+    refs = [oracle.as_u16(p).copy() for p in inp.pools]
+    st = B.Stage(pools=pools, layer_window=wl.layer_window, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D,
+                 max_batch=9, max_pages_per_seq=inp.max_pages_per_seq)
+    for step in range(3):
+        pos = inp.positions(step).copy()
+        pos[5] = -1                                                   # an inactive slot every step
+        n = np.where(pos >= 0, pos + 1, 0).astype(np.int32)
+        for layer in range(2):
+            q, k, v = inp.q[step, layer], inp.k_new[step, layer], inp.v_new[step, layer]
+            out = torch.full((9, Hq, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+            lse = torch.full((9, Hq), float("nan"), dtype=torch.float32, device="cuda")
+            before = st.launch_count()
+            st.decode_step(layer, q.cuda(), k.cuda(), v.cuda(), dev(pos), inp.page_tables[layer].cuda(), out, lse)
+            assert st.poll_error() == B.OPW_OK and st.launch_count() - before == 2
+            assert oracle.kv_append(refs[layer], Hkv, D, P, k, v, pos, inp.page_tables[layer]) == 0
+            assert (pools[layer].cpu().view(torch.int16).numpy().view(np.uint16) == refs[layer]).all()
+            ref, ref_lse, _ = oracle.decode_attention(refs[layer], Hq, Hkv, D, P, q, n, inp.page_tables[layer],
+                                                      window=wl.layer_window[layer])
+            check_close(out_to_f64(out), ref, lse.cpu().numpy().astype(np.float64), ref_lse)
+    st.close()
+
+
 def test_single_key_returns_v_bit_exactly():
     rng = np.random.default_rng(51)
     Hq, Hkv, D = 8, 2, 64
@@ -324,12 +353,13 @@ def test_host_buffer_step_matches_the_device_step():
             ref, ref_lse, _ = oracle.decode_attention(refs[layer], 32, 8, 128, P, q, inp.kv_lens(step), tab,
                                                       window=wl.layer_window[layer])
             check_close(out_to_f64(out), ref, lse.numpy().astype(np.float64), ref_lse)
-    assert st.launch_count() == 2 * 2 * 4
+    assert st.launch_count() == 2 * 2 * 2
     st.close()
 
 
+@pytest.mark.parametrize("fused", [False, True])
 @pytest.mark.parametrize("flags", [0, B.OPW_PLAN_GRAPH, B.OPW_PLAN_GRAPH | B.OPW_PLAN_ADVANCE, B.OPW_PLAN_ADVANCE])
-def test_plan_submits_a_multi_layer_multi_microbatch_step_in_one_call(flags):
+def test_plan_submits_a_multi_layer_multi_microbatch_step_in_one_call(flags, fused):
     """Two layers (one windowed) x two microbatches, three decode steps, one native call per step."""
     wl = synth.Workload("p", 6, 32, 8, 128, [0, 48], "uniform_1024_4096", 78)
     lens = np.array([5, 200, 1023, 64, 15, 3000], np.int32)
@@ -352,7 +382,8 @@ def test_plan_submits_a_multi_layer_multi_microbatch_step_in_one_call(flags):
     for m, mb in enumerate(mbs):
         for l in range(2):
             items.append(dict(layer=l, batch=mb.stop - mb.start, q=q[l][m].data_ptr(), k_new=k[l][m].data_ptr(),
-                              v_new=v[l][m].data_ptr(), positions=pos[m].data_ptr(), kv_lens=kvl[m].data_ptr(),
+                              v_new=v[l][m].data_ptr(), positions=pos[m].data_ptr(),
+                              kv_lens=None if fused else kvl[m].data_ptr(),
                               page_table=tabs[l][m].data_ptr(), out=out[l][m].data_ptr(), lse=lse[l][m].data_ptr()))
     plan = B.opw_attn_plan_create(st.handle, items, flags)
     stream = torch.cuda.current_stream().cuda_stream
@@ -368,7 +399,7 @@ def test_plan_submits_a_multi_layer_multi_microbatch_step_in_one_call(flags):
         before = st.launch_count()
         B.opw_attn_plan_submit(plan, stream)
         assert st.poll_error() == B.OPW_OK
-        assert st.launch_count() - before == 4 * 3 + (2 if flags & B.OPW_PLAN_ADVANCE else 0)
+        assert st.launch_count() - before == 4 * (2 if fused else 3) + (2 if flags & B.OPW_PLAN_ADVANCE else 0)
         for l in range(2):
             assert oracle.kv_append(refs[l], 8, 128, P, inp.k_new[step, l], inp.v_new[step, l], inp.positions(step),
                                     inp.page_tables[l]) == 0
@@ -379,7 +410,8 @@ def test_plan_submits_a_multi_layer_multi_microbatch_step_in_one_call(flags):
             got_lse = torch.cat([lse[l][m] for m in range(2)])
             check_close(out_to_f64(got), ref, got_lse.cpu().numpy().astype(np.float64), ref_lse)
     if flags & B.OPW_PLAN_ADVANCE:
-        assert (pos[0].cpu().numpy() == lens[mbs[0]] + 3).all() and (kvl[1].cpu().numpy() == lens[mbs[1]] + 4).all()
+        assert (pos[0].cpu().numpy() == lens[mbs[0]] + 3).all()
+        assert fused or (kvl[1].cpu().numpy() == lens[mbs[1]] + 4).all()
     B.opw_attn_plan_destroy(plan)
     st.close()
 
