@@ -18,6 +18,7 @@ constexpr int kDefaultWarps = 8;
 constexpr int kDefaultStages = 2;
 constexpr int kDefaultCtasPerSm = 1;
 constexpr size_t kSmemLimit = 227 * 1024;
+constexpr int kCombineScratchSlots = 1024;       // rows * splits of the split combine never exceed this
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
@@ -26,7 +27,7 @@ struct Shape {
 };
 
 struct Layout {          // byte offsets into the caller's workspace
-  size_t status, cum, partials, st_q, st_k, st_v, st_pos, st_lens, st_out, st_lse, st_table, total;
+  size_t status, cum, partials, comb_scratch, row_count, st_q, st_k, st_v, st_pos, st_lens, st_out, st_lse, st_table, total;
 };
 
 bool shape_ok(const opw_attn_stage_config_t* c) {
@@ -57,6 +58,8 @@ Layout carve(const opw_attn_stage_config_t* c, const Shape& s, int sms) {
   L.status = off;  off += 256;
   L.cum = off;     off += align_up((B + 2) * 4, 256);
   L.partials = off; off += align_up(workers * 2 * opw::kSegPerShare * G * (D + 2) * 4, 256);
+  L.comb_scratch = off; off += align_up((size_t)kCombineScratchSlots * G * (D + 2) * 4, 256);
+  L.row_count = off; off += align_up(B * Hkv * 4, 256);
   L.st_q = off;    off += align_up(B * Hq * D * 2, 256);
   L.st_k = off;    off += align_up(B * Hkv * D * 2, 256);
   L.st_v = off;    off += align_up(B * Hkv * D * 2, 256);
@@ -193,7 +196,12 @@ opw_status_t opw_attn_stage_create(const opw_attn_stage_config_t* cfg, opw_attn_
       e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_i);
   }
   if (e != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
-  if (cudaMemset(cfg->workspace, 0, 256) != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
+  if (cudaMemset(cfg->workspace, 0, 256) != cudaSuccess ||
+      cudaMemset(static_cast<unsigned char*>(cfg->workspace) + lay.row_count, 0,
+                 (size_t)cfg->max_batch * cfg->num_kv_heads * 4) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return OPW_ERR_CUDA;
+  }
   if (cudaDeviceSynchronize() != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
 
   opw_attn_stage* st = new (std::nothrow) opw_attn_stage();
@@ -348,7 +356,16 @@ static opw_status_t enqueue_attention(opw_attn_stage_t* st, int32_t layer, int32
   c.max_pages = p.max_pages;
   c.window = p.window;
   c.num_workers = st->grid * st->shape.warps;
-  if (launch(opw::combine_kernel, dim3(batch * Hkv), dim3(opw::kCombineThreads), 0, stream, pdl, c) != cudaSuccess) {
+  c.scratch = reinterpret_cast<float*>(st->ws + st->lay.comb_scratch);
+  c.row_count = reinterpret_cast<int32_t*>(st->ws + st->lay.row_count);
+  // Few rows can have very many partials each (long contexts at small batch): split each row's
+  // merge over several blocks so that about two blocks per SM are busy.
+  const int rows = batch * Hkv;
+  int splits = (2 * st->sms) / rows;
+  if (splits > opw::kCombineBatch) splits = opw::kCombineBatch;
+  if (splits > kCombineScratchSlots / rows) splits = kCombineScratchSlots / rows;
+  if (splits < 1) splits = 1;
+  if (launch(opw::combine_kernel, dim3(rows, splits), dim3(opw::kCombineThreads), 0, stream, pdl, c) != cudaSuccess) {
     (void)cudaGetLastError();
     return OPW_ERR_CUDA;
   }

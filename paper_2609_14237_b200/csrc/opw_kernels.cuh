@@ -196,43 +196,44 @@ __host__ __device__ __forceinline__ int64_t worker_begin(int64_t U, int64_t work
 __host__ __device__ __forceinline__ int64_t worker_of(int64_t U, int64_t u, int64_t num_workers) {
   return ((u + 1) * num_workers - 1) / U;
 }
-// Segments of a share: k = 0 is the static first 13/16; k = 1..kDynPerShare cut the last 3/16
-// into ever smaller chunks (cut points in sixteenths of that part).
+// Segments of a share: k = 0 is the static first 13/16; k = 1..J cut the last 3/16 into ever
+// smaller chunks (cut points in sixteenths of that part).  J depends on the share length
+// only (the same for every share of a launch): a segment costs a couple of microseconds of
+// fixed work (ticket, descriptors, Q reload, partial flush), so short shares get fewer chunks.
 #ifndef OPW_DYN_PER_SHARE
-#define OPW_DYN_PER_SHARE 6
+#define OPW_DYN_PER_SHARE 6      /* upper bound of J; 0 builds static shares only */
 #endif
 #ifndef OPW_DYN_32NDS
 #define OPW_DYN_32NDS 6          /* the dynamic part of a share, in 32nds: 6/32 = 3/16 */
 #endif
 constexpr int kDynPerShare = OPW_DYN_PER_SHARE;
-constexpr int kSegPerShare = kDynPerShare + 1;
-__host__ __device__ __forceinline__ int64_t dyn_cut(int k) {   // five bits per cut point
-#if OPW_DYN_PER_SHARE == 8
-  const uint64_t cuts = 0ull | (4ull << 5) | (8ull << 10) | (10ull << 15) | (12ull << 20) | (13ull << 25) |
-                        (14ull << 30) | (15ull << 35) | (16ull << 40);       // 0,4,8,10,12,13,14,15,16
-#elif OPW_DYN_PER_SHARE == 4
-  const uint64_t cuts = 0ull | (8ull << 5) | (12ull << 10) | (14ull << 15) | (16ull << 20);   // 0,8,12,14,16
-#elif OPW_DYN_PER_SHARE == 0
-  const uint64_t cuts = 0ull;                                                 // static shares only
-#elif OPW_DYN_PER_SHARE == 6
-  const uint64_t cuts = 0ull | (5ull << 5) | (9ull << 10) | (12ull << 15) | (14ull << 20) | (15ull << 25) |
-                        (16ull << 30);                                        // 0,5,9,12,14,15,16
-#else
+constexpr int kSegPerShare = kDynPerShare + 1;   // partial slots are indexed with this stride
+#if OPW_DYN_PER_SHARE != 0 && OPW_DYN_PER_SHARE != 6
 #error "unsupported OPW_DYN_PER_SHARE"
 #endif
-  return (int64_t)((cuts >> (5 * k)) & 31);
+// number of dynamic chunks per share for a launch of U units on num_workers workers
+__host__ __device__ __forceinline__ int dyn_chunks(int64_t U, int64_t num_workers) {
+  if (kDynPerShare == 0) return 0;
+  const int64_t per = U / num_workers;
+  return per < 8 ? 0 : per < 48 ? 2 : per < 128 ? 4 : 6;
 }
-// Launches with fewer than eight units per worker have no dynamic chunks at all.
-__host__ __device__ __forceinline__ bool has_dynamic(int64_t U, int64_t num_workers) {
-  return kDynPerShare > 0 && U >= 8 * num_workers;
+__host__ __device__ __forceinline__ int64_t dyn_cut(int J, int k) {   // five bits per cut point
+  const uint64_t cuts6 = 0ull | (5ull << 5) | (9ull << 10) | (12ull << 15) | (14ull << 20) | (15ull << 25) |
+                         (16ull << 30);                                  // 0,5,9,12,14,15,16
+  const uint64_t cuts4 = 0ull | (6ull << 5) | (11ull << 10) | (14ull << 15) | (16ull << 20);   // 0,6,11,14,16
+  const uint64_t cuts2 = 0ull | (9ull << 5) | (16ull << 10);            // 0,9,16
+  const uint64_t cuts = J == 6 ? cuts6 : J == 4 ? cuts4 : cuts2;
+  return (int64_t)((cuts >> (5 * k)) & 31);
 }
 __host__ __device__ __forceinline__ void segment_bounds(int64_t U, int64_t num_workers, int64_t w, int k,
                                                         int64_t& a, int64_t& b) {
+  const int J = dyn_chunks(U, num_workers);
   const int64_t s0 = worker_begin(U, w, num_workers), s1 = worker_begin(U, w + 1, num_workers);
-  const int64_t len = s1 - s0, dyn = has_dynamic(U, num_workers) ? (len * OPW_DYN_32NDS) >> 5 : 0, stat = len - dyn;
+  const int64_t len = s1 - s0, dyn = J > 0 ? (len * OPW_DYN_32NDS) >> 5 : 0, stat = len - dyn;
   if (k == 0) { a = s0; b = s0 + stat; return; }
-  a = s0 + stat + ((dyn * dyn_cut(k - 1)) >> 4);
-  b = s0 + stat + ((dyn * dyn_cut(k)) >> 4);
+  if (k > J) { a = b = s1; return; }            // this launch has fewer chunks per share
+  a = s0 + stat + ((dyn * dyn_cut(J, k - 1)) >> 4);
+  b = s0 + stat + ((dyn * dyn_cut(J, k)) >> 4);
 }
 
 // ---------------------------------------------------------------------------------
@@ -444,7 +445,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnPar
   int64_t u = 0;
   int64_t units_done = 0;
   bool traced_first = false;
-  const int32_t num_tickets = has_dynamic(U, num_workers) ? (int32_t)(num_workers * kDynPerShare) : 0;
+  const int32_t num_tickets = (int32_t)(num_workers * dyn_chunks(U, num_workers));
 
   // The segment being processed is [u0,u1) with partial slots slot_base, slot_base+1; first the
   // worker's own static segment, then whatever chunks the ticket counter hands out.  The next
@@ -750,6 +751,8 @@ struct CombineParams {
   const int32_t* cum;
   const int32_t* kv_lens;     // or null: then positions[b] + 1
   const int32_t* positions;
+  float* scratch;             // [rows * splits][G*(D+2)] intermediates (used when gridDim.y > 1)
+  int32_t* row_count;         // [rows] arrival counters, zero between launches
   __nv_bfloat16* out;
   float* lse;
   int32_t batch, Hq, Hkv, G, D;
@@ -785,7 +788,7 @@ __device__ __forceinline__ void combine_accumulate(float* acc, const float* part
     for (int u = 0; u < US; ++u) {
       const float* sp = partials + (int64_t)seg_slot[sgm + u] * stride + threadIdx.x;
 #pragma unroll
-      for (int j = 0; j < NEL; ++j) o[j][u] = ok[j] ? sp[j * kCombineThreads] : 0.f;
+      for (int j = 0; j < NEL; ++j) o[j][u] = ok[j] ? __ldcg(sp + j * kCombineThreads) : 0.f;
     }
 #pragma unroll
     for (int u = 0; u < US; ++u)
@@ -796,26 +799,34 @@ __device__ __forceinline__ void combine_accumulate(float* acc, const float* part
     const float* sp = partials + (int64_t)seg_slot[sgm] * stride + threadIdx.x;
 #pragma unroll
     for (int j = 0; j < NEL; ++j)
-      if (ok[j]) acc[j] += w_s[sgm * G + hh[j]] * sp[j * kCombineThreads];
+      if (ok[j]) acc[j] += w_s[sgm * G + hh[j]] * __ldcg(sp + j * kCombineThreads);
   }
 }
 
+// grid = (rows, splits).  With splits == 1 a block merges all of its row's partials and writes
+// the output.  With splits > 1 (few rows, many partials each: long contexts at small batch)
+// block (row, y) merges every splits-th batch of the row's partials into one intermediate
+// partial in `scratch`, and the block that finishes last for the row (an atomic counter,
+// nothing waits) merges those `splits` intermediates and writes the output.
 __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams p) {
   pdl_launch_dependents();
   const int row = blockIdx.x;
+  const int splits = gridDim.y, split = blockIdx.y;
   const int b = row / p.Hkv, g = row - b * p.Hkv;
   const int D = p.D, G = p.G;
   const int GD = G * D;
   int32_t n = visible_keys(p.kv_lens, p.positions, b);   // an input: may be read before the attention kernel is done
   pdl_wait();                                  // partials, prefix sums and complete rows are final now
-  if (blockIdx.x == 0 && threadIdx.x == 0) *p.ticket = 0;
+  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *p.ticket = 0;
   const int32_t cum_b = p.cum[b], cum_all = p.cum[p.batch];     // independent of the load above
   if (n > p.max_pages * kPage) n = p.max_pages * kPage;
   __nv_bfloat16* ob = p.out + ((int64_t)b * p.Hq + (int64_t)g * G) * D;
   float* lse_row = p.lse ? p.lse + (int64_t)b * p.Hq + g * G : nullptr;
   if (n <= 0) {   // inactive slot: zeros, lse = -inf
-    for (int e = threadIdx.x; e < GD; e += kCombineThreads) ob[e] = __float2bfloat16(0.f);
-    if (lse_row && threadIdx.x < G) lse_row[threadIdx.x] = -INFINITY;
+    if (split == 0) {
+      for (int e = threadIdx.x; e < GD; e += kCombineThreads) ob[e] = __float2bfloat16(0.f);
+      if (lse_row && threadIdx.x < G) lse_row[threadIdx.x] = -INFINITY;
+    }
     return;
   }
   int32_t first, cnt, lo;
@@ -825,18 +836,29 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
   const int64_t uend = ustart + cnt;
   const int64_t wf = worker_of(U, ustart, p.num_workers), wl = worker_of(U, uend - 1, p.num_workers);
   const int64_t stride = (int64_t)G * (D + 2);
+  // If the segment that holds the row's first unit also holds its last, that segment's worker
+  // has already stored the final result: nothing to merge (every block of the row sees this).
+  {
+    bool whole = false;
+    if (threadIdx.x < kSegPerShare) {
+      int64_t a, bnd;
+      segment_bounds(U, p.num_workers, wf, (int)threadIdx.x, a, bnd);
+      whole = a <= ustart && ustart < bnd && bnd >= uend;
+    }
+    if (__syncthreads_or(whole)) return;
+  }
   // The row's partials come from the segments (share w in wf..wl, k in 0..kSegPerShare) that
   // overlap it.  A batch of candidate segments at a time: each thread tests one, an ordered
   // compaction lists the partial slots in shared memory, one warp per head turns the partials'
   // running maxima into weights 2^(m - M), and every thread sums its elements over the list.
   // A segment's partial for this row is in the segment's slot 0 if the segment starts inside
-  // the row, else in slot 1.  If one segment covers the whole row, its worker has already
-  // stored the final result.
+  // the row, else in slot 1.
   __shared__ int32_t seg_slot[kCombineBatch];
   __shared__ int32_t warp_cnt[kCombineThreads / 32];
   __shared__ float w_s[kCombineBatch * kCombineMaxG];   // per (segment, head): m, then the weight
   __shared__ float l_s[kCombineBatch * kCombineMaxG];
   __shared__ float run_M[kCombineMaxG], run_L[kCombineMaxG], run_scale[kCombineMaxG];
+  __shared__ int32_t is_last;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   constexpr int kMaxElems = kCombineMaxG * 128 / kCombineThreads;   // 8
   const int nel = (GD + kCombineThreads - 1) / kCombineThreads;
@@ -849,9 +871,49 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
   // counted once, at its first unit inside the row.
   const bool by_unit = (wl - wf + 1) > (int64_t)cnt;
   const int64_t ncand = (by_unit ? (int64_t)cnt : (wl - wf + 1)) * kSegPerShare;
-  for (int64_t base = 0; base < ncand; base += kCombineBatch) {
+
+  // One merge pass over `nseg` listed partials at `base_ptr` (slot stride `stride`): stage
+  // (m, l), weights per head, then the weighted sums.
+  auto merge_listed = [&](const float* base_ptr, int nseg) {
+    for (int idx = threadIdx.x; idx < nseg * G; idx += kCombineThreads) {   // stage (m, l): independent loads
+      const int sgm = idx / G, h = idx - sgm * G;
+      const float* sp = base_ptr + (int64_t)seg_slot[sgm] * stride + GD;
+      w_s[idx] = __ldcg(sp + h);
+      l_s[idx] = __ldcg(sp + G + h);
+    }
+    __syncthreads();
+    for (int h = warp; h < G; h += kCombineThreads / 32) {   // a warp per head: max, weights, sum of l
+      float Mc = run_M[h];
+      for (int sgm = lane; sgm < nseg; sgm += 32) Mc = fmaxf(Mc, w_s[sgm * G + h]);
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) Mc = fmaxf(Mc, __shfl_xor_sync(0xffffffffu, Mc, o));
+      float Lc = 0.f;
+      for (int sgm = lane; sgm < nseg; sgm += 32) {
+        const float wgt = Mc == -INFINITY ? 0.f : exp2f(w_s[sgm * G + h] - Mc);
+        w_s[sgm * G + h] = wgt;
+        Lc += wgt * l_s[sgm * G + h];
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) Lc += __shfl_xor_sync(0xffffffffu, Lc, o);
+      if (lane == 0) {
+        const float sc = Mc == -INFINITY ? 0.f : exp2f(run_M[h] - Mc);   // 0 on the first batch (run_M = -inf)
+        run_L[h] = run_L[h] * sc + Lc;
+        run_M[h] = Mc;
+        run_scale[h] = sc;
+      }
+    }
+    __syncthreads();
+    // about 32 independent loads in flight per thread: NEL elements x (32 / NEL) segments
+    if (nel <= 1) combine_accumulate<1>(acc, base_ptr, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
+    else if (nel <= 2) combine_accumulate<2>(acc, base_ptr, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
+    else if (nel <= 4) combine_accumulate<4>(acc, base_ptr, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
+    else combine_accumulate<8>(acc, base_ptr, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
+    __syncthreads();
+  };
+
+  for (int64_t base = (int64_t)split * kCombineBatch; base < ncand; base += (int64_t)splits * kCombineBatch) {
     const int64_t i = base + threadIdx.x;
-    bool hit = false, whole = false;
+    bool hit = false;
     int32_t slot = 0;
     if (threadIdx.x < kCombineBatch && i < ncand) {
       const int64_t j = i / kSegPerShare;
@@ -867,10 +929,8 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
       int64_t a, bnd;
       segment_bounds(U, p.num_workers, w, k, a, bnd);
       hit = counted && a < bnd && a < uend && bnd > ustart;
-      whole = hit && a <= ustart && bnd >= uend;
       slot = (int32_t)(2 * (w * kSegPerShare + k) + (a >= ustart ? 0 : 1));
     }
-    if (__syncthreads_or(whole)) return;        // finished by a single segment: nothing to merge
     const uint32_t bal = __ballot_sync(0xffffffffu, hit);
     if (lane == 0) warp_cnt[warp] = __popc(bal);
     __syncthreads();
@@ -882,40 +942,38 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
     }
     if (hit) seg_slot[pos] = slot;
     __syncthreads();
-    for (int idx = threadIdx.x; idx < nseg * G; idx += kCombineThreads) {   // stage (m, l): independent loads
-      const int sgm = idx / G, h = idx - sgm * G;
-      const float* sp = p.partials + (int64_t)seg_slot[sgm] * stride + GD;
-      w_s[idx] = sp[h];
-      l_s[idx] = sp[G + h];
+    merge_listed(p.partials, nseg);
+  }
+
+  if (splits > 1) {
+    // hand this block's intermediate (un-normalised sums relative to run_M) to the row's last block
+    float* mine = p.scratch + ((int64_t)row * splits + split) * stride;
+#pragma unroll
+    for (int j = 0; j < kMaxElems; ++j) {
+      const int e = threadIdx.x + j * kCombineThreads;
+      if (e < GD) __stcg(mine + e, acc[j]);
+    }
+    if (threadIdx.x < G) {
+      __stcg(mine + GD + threadIdx.x, run_M[threadIdx.x]);
+      __stcg(mine + GD + G + threadIdx.x, run_L[threadIdx.x]);
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      const int32_t arrived = atomicAdd(p.row_count + row, 1);
+      is_last = arrived == splits - 1;
+      if (is_last) p.row_count[row] = 0;        // ready for the next launch
     }
     __syncthreads();
-    for (int h = warp; h < G; h += kCombineThreads / 32) {   // a warp per head: max, weights, sum of l
-      float Mc = run_M[h];
-      for (int sgm = lane; sgm < nseg; sgm += 32) Mc = fmaxf(Mc, w_s[sgm * G + h]);
+    if (!is_last) return;
+    __threadfence();
+    // merge the row's `splits` intermediates (splits <= kCombineBatch), in split order
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) Mc = fmaxf(Mc, __shfl_xor_sync(0xffffffffu, Mc, o));
-      float Lc = 0.f;
-      for (int sgm = lane; sgm < nseg; sgm += 32) {
-        const float wgt = exp2f(w_s[sgm * G + h] - Mc);
-        w_s[sgm * G + h] = wgt;
-        Lc += wgt * l_s[sgm * G + h];
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) Lc += __shfl_xor_sync(0xffffffffu, Lc, o);
-      if (lane == 0) {
-        const float sc = exp2f(run_M[h] - Mc);    // 0 on the first batch (run_M = -inf)
-        run_L[h] = run_L[h] * sc + Lc;
-        run_M[h] = Mc;
-        run_scale[h] = sc;
-      }
-    }
+    for (int j = 0; j < kMaxElems; ++j) acc[j] = 0.f;
+    if (threadIdx.x < kCombineMaxG) { run_M[threadIdx.x] = -INFINITY; run_L[threadIdx.x] = 0.f; }
+    if (threadIdx.x < splits) seg_slot[threadIdx.x] = row * splits + threadIdx.x;
     __syncthreads();
-    // about 32 independent loads in flight per thread: NEL elements x (32 / NEL) segments
-    if (nel <= 1) combine_accumulate<1>(acc, p.partials, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
-    else if (nel <= 2) combine_accumulate<2>(acc, p.partials, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
-    else if (nel <= 4) combine_accumulate<4>(acc, p.partials, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
-    else combine_accumulate<8>(acc, p.partials, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
-    __syncthreads();
+    merge_listed(p.scratch, splits);
   }
 #pragma unroll
   for (int j = 0; j < kMaxElems; ++j) {

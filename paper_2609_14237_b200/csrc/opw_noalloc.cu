@@ -165,6 +165,8 @@ extern "C" opw_status_t opw_decode_attention_noalloc(int32_t num_q_heads, int32_
   c.cum = p.cum;
   c.kv_lens = kv_lens;
   c.positions = nullptr;
+  c.scratch = nullptr;                // one block per row: no intermediates
+  c.row_count = nullptr;
   c.out = p.out;
   c.lse = lse;
   c.batch = batch;
