@@ -208,6 +208,12 @@ opw_status_t opw_decode_step_host(opw_attn_stage_t *stage, int32_t layer, int32_
  *   OPW_PLAN_ADVANCE : after the last item, add 1 to every distinct positions array (entries
  *                      >= 0) and kv_lens array (entries > 0), so that re-submitting the plan
  *                      is the next decode step with no host work on the metadata.
+ *   OPW_PLAN_OVERLAP : run item i's combine kernel on a private side stream (a parallel branch
+ *                      of the graph) beside item i+1's split-KV kernel, alternating between the
+ *                      stage's two workspace sets; the submission still completes only when
+ *                      every output is final.  Consecutive items must then have different out
+ *                      (and lse) buffers (OPW_ERR_INVALID_ARG otherwise).  Takes the combine and
+ *                      one launch gap off the critical path of all items but the last.
  * create validates every item on the host (same rules and codes as the step calls) and, with
  * OPW_PLAN_GRAPH, captures on a private stream: nothing executes until submit.  A plan must be
  * destroyed before its stage.
@@ -228,6 +234,7 @@ typedef struct {
 typedef struct opw_attn_plan opw_attn_plan_t;
 #define OPW_PLAN_GRAPH 1u
 #define OPW_PLAN_ADVANCE 2u
+#define OPW_PLAN_OVERLAP 4u
 
 opw_status_t opw_attn_plan_create(opw_attn_stage_t *stage, const opw_step_item_t *items, int32_t n_items,
                                   uint32_t flags, opw_attn_plan_t **out);

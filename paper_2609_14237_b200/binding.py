@@ -70,7 +70,7 @@ class StepItem(ctypes.Structure):
     ]
 
 
-OPW_PLAN_GRAPH, OPW_PLAN_ADVANCE = 1, 2
+OPW_PLAN_GRAPH, OPW_PLAN_ADVANCE, OPW_PLAN_OVERLAP = 1, 2, 4
 
 
 def build(force: bool = False, verbose: bool = False) -> str:

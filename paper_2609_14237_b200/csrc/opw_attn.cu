@@ -27,7 +27,7 @@ struct Shape {
 };
 
 struct Layout {          // byte offsets into the caller's workspace
-  size_t status, cum, partials, comb_scratch, row_count, st_q, st_k, st_v, st_pos, st_lens, st_out, st_lse, st_table, total;
+  size_t status, cum[2], partials[2], comb_scratch, row_count, st_q, st_k, st_v, st_pos, st_lens, st_out, st_lse, st_table, total;
 };
 
 bool shape_ok(const opw_attn_stage_config_t* c) {
@@ -56,8 +56,10 @@ Layout carve(const opw_attn_stage_config_t* c, const Shape& s, int sms) {
   const size_t workers = (size_t)sms * s.ctas_per_sm * s.warps;
   size_t off = 0;
   L.status = off;  off += 256;
-  L.cum = off;     off += align_up((B + 2) * 4, 256);
-  L.partials = off; off += align_up(workers * 2 * opw::kSegPerShare * G * (D + 2) * 4, 256);
+  for (int i = 0; i < 2; ++i) {        // two sets: a plan may run a step's combine beside the next attention
+    L.cum[i] = off;      off += align_up((B + 2) * 4, 256);
+    L.partials[i] = off; off += align_up(workers * 2 * opw::kSegPerShare * G * (D + 2) * 4, 256);
+  }
   L.comb_scratch = off; off += align_up((size_t)kCombineScratchSlots * G * (D + 2) * 4, 256);
   L.row_count = off; off += align_up(B * Hkv * 4, 256);
   L.st_q = off;    off += align_up(B * Hq * D * 2, 256);
@@ -284,50 +286,61 @@ opw_status_t opw_kv_append(opw_attn_stage_t* st, int32_t layer, int32_t batch, c
   return OPW_OK;
 }
 
-static opw_status_t enqueue_attention(opw_attn_stage_t* st, int32_t layer, int32_t batch, const void* q,
-                                      const int32_t* kv_lens, const void* k_new, const void* v_new,
-                                      const int32_t* positions, const int32_t* page_table, void* out, float* lse,
-                                      void* cuda_stream) {
-  opw_status_t rc = check_step(st, layer, batch);
-  if (rc != OPW_OK) return rc;
-  const bool fused = k_new != nullptr;
-  if (!q || !page_table || !out) return OPW_ERR_INVALID_ARG;
-  if (fused ? (!v_new || !positions || kv_lens) : (!kv_lens || v_new || positions)) return OPW_ERR_INVALID_ARG;
-  if (((uintptr_t)q | (uintptr_t)out | (uintptr_t)k_new | (uintptr_t)v_new) % 16 || (uintptr_t)kv_lens % 4 ||
-      (uintptr_t)positions % 4 || (uintptr_t)page_table % 4 || (uintptr_t)lse % 4)
-    return OPW_ERR_INVALID_ARG;
-  if (batch == 0) return OPW_OK;
-  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  const int D = st->cfg.head_dim, Hq = st->cfg.num_q_heads, Hkv = st->cfg.num_kv_heads, G = Hq / Hkv;
+struct StepArgs {
+  int32_t layer, batch;
+  const void* q;
+  const int32_t* kv_lens;      // or null with the fused append
+  const void* k_new;           // fused append: all three set, else all null
+  const void* v_new;
+  const int32_t* positions;
+  const int32_t* page_table;
+  void* out;
+  float* lse;
+};
 
+static opw_status_t validate_step(opw_attn_stage_t* st, const StepArgs& a) {
+  opw_status_t rc = check_step(st, a.layer, a.batch);
+  if (rc != OPW_OK) return rc;
+  const bool fused = a.k_new != nullptr;
+  if (!a.q || !a.page_table || !a.out) return OPW_ERR_INVALID_ARG;
+  if (fused ? (!a.v_new || !a.positions || a.kv_lens) : (!a.kv_lens || a.v_new || a.positions)) return OPW_ERR_INVALID_ARG;
+  if (((uintptr_t)a.q | (uintptr_t)a.out | (uintptr_t)a.k_new | (uintptr_t)a.v_new) % 16 || (uintptr_t)a.kv_lens % 4 ||
+      (uintptr_t)a.positions % 4 || (uintptr_t)a.page_table % 4 || (uintptr_t)a.lse % 4)
+    return OPW_ERR_INVALID_ARG;
+  return OPW_OK;
+}
+
+// The split-KV kernel of one step, using workspace set `ws_set` (0 or 1).
+static opw_status_t launch_attention(opw_attn_stage_t* st, const StepArgs& a, int ws_set, cudaStream_t stream) {
+  const int D = st->cfg.head_dim, Hq = st->cfg.num_q_heads, Hkv = st->cfg.num_kv_heads, G = Hq / Hkv;
   opw::AttnParams p;
-  p.pool = static_cast<const __nv_bfloat16*>(st->pool[layer]);
-  p.q = static_cast<const __nv_bfloat16*>(q);
-  p.kv_lens = kv_lens;
-  p.page_table = page_table;
-  p.k_new = static_cast<const __nv_bfloat16*>(k_new);
-  p.v_new = static_cast<const __nv_bfloat16*>(v_new);
-  p.positions = positions;
-  p.pool_w = static_cast<__nv_bfloat16*>(st->pool[layer]);
-  p.out = static_cast<__nv_bfloat16*>(out);
-  p.lse = lse;
-  p.partials = reinterpret_cast<float*>(st->ws + st->lay.partials);
-  p.cum = reinterpret_cast<int32_t*>(st->ws + st->lay.cum);
+  p.pool = static_cast<const __nv_bfloat16*>(st->pool[a.layer]);
+  p.q = static_cast<const __nv_bfloat16*>(a.q);
+  p.kv_lens = a.kv_lens;
+  p.page_table = a.page_table;
+  p.k_new = static_cast<const __nv_bfloat16*>(a.k_new);
+  p.v_new = static_cast<const __nv_bfloat16*>(a.v_new);
+  p.positions = a.positions;
+  p.pool_w = static_cast<__nv_bfloat16*>(st->pool[a.layer]);
+  p.out = static_cast<__nv_bfloat16*>(a.out);
+  p.lse = a.lse;
+  p.partials = reinterpret_cast<float*>(st->ws + st->lay.partials[ws_set]);
+  p.cum = reinterpret_cast<int32_t*>(st->ws + st->lay.cum[ws_set]);
   p.status = reinterpret_cast<uint32_t*>(st->ws + st->lay.status);
-  p.ticket = reinterpret_cast<int32_t*>(st->ws + st->lay.status + 16);
+  p.ticket = reinterpret_cast<int32_t*>(st->ws + st->lay.status + 16 + 16 * ws_set);
   p.trace = st->trace;
-  p.num_pages = st->num_pages[layer];
-  p.batch = batch;
+  p.num_pages = st->num_pages[a.layer];
+  p.batch = a.batch;
   p.Hq = Hq;
   p.Hkv = Hkv;
   p.G = G;
   p.max_pages = st->cfg.max_pages_per_seq;
-  p.window = st->window[layer];
+  p.window = st->window[a.layer];
   p.stages = st->shape.stages;
   p.scale_log2e = st->scale_log2e;
 
   const dim3 grid(st->grid), block(st->shape.warps * 32);
-  const size_t smem = attn_smem_bytes(D, st->shape, batch);
+  const size_t smem = attn_smem_bytes(D, st->shape, a.batch);
   const bool pdl = (st->cfg.flags & OPW_FLAG_PDL) != 0;
   cudaError_t e;
   if (D == 64) {
@@ -339,40 +352,61 @@ static opw_status_t enqueue_attention(opw_attn_stage_t* st, int32_t layer, int32
   }
   if (e != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
   st->launches += 1;
+  return OPW_OK;
+}
 
+// The log-sum-exp combine of the same step.  `small` picks the 128-thread instance, which
+// fits on an SM beside a split-KV block.
+static opw_status_t launch_combine(opw_attn_stage_t* st, const StepArgs& a, int ws_set, cudaStream_t stream, bool small) {
+  const int D = st->cfg.head_dim, Hq = st->cfg.num_q_heads, Hkv = st->cfg.num_kv_heads, G = Hq / Hkv;
   opw::CombineParams c;
-  c.ticket = p.ticket;
-  c.partials = p.partials;
-  c.cum = p.cum;
-  c.kv_lens = kv_lens;
-  c.positions = positions;
-  c.out = p.out;
-  c.lse = lse;
-  c.batch = batch;
+  c.ticket = reinterpret_cast<int32_t*>(st->ws + st->lay.status + 16 + 16 * ws_set);
+  c.partials = reinterpret_cast<const float*>(st->ws + st->lay.partials[ws_set]);
+  c.cum = reinterpret_cast<const int32_t*>(st->ws + st->lay.cum[ws_set]);
+  c.kv_lens = a.kv_lens;
+  c.positions = a.positions;
+  c.out = static_cast<__nv_bfloat16*>(a.out);
+  c.lse = a.lse;
+  c.batch = a.batch;
   c.Hq = Hq;
   c.Hkv = Hkv;
   c.G = G;
   c.D = D;
-  c.max_pages = p.max_pages;
-  c.window = p.window;
+  c.max_pages = st->cfg.max_pages_per_seq;
+  c.window = st->window[a.layer];
   c.num_workers = st->grid * st->shape.warps;
   c.scratch = reinterpret_cast<float*>(st->ws + st->lay.comb_scratch);
   c.row_count = reinterpret_cast<int32_t*>(st->ws + st->lay.row_count);
   // Few rows can have very many partials each (long contexts at small batch): split each row's
   // merge over several blocks so that about two blocks per SM are busy.
-  const int rows = batch * Hkv;
+  const int rows = a.batch * Hkv;
   int splits = (2 * st->sms) / rows;
   if (splits > opw::kCombineBatch) splits = opw::kCombineBatch;
   if (splits > kCombineScratchSlots / rows) splits = kCombineScratchSlots / rows;
   if (splits < 1) splits = 1;
-  if (launch(opw::combine_kernel, dim3(rows, splits), dim3(opw::kCombineThreads), 0, stream, pdl, c) != cudaSuccess) {
-    (void)cudaGetLastError();
-    return OPW_ERR_CUDA;
-  }
+  const bool pdl = (st->cfg.flags & OPW_FLAG_PDL) != 0 && !small;
+  cudaError_t e = small ? launch(opw::combine_kernel<opw::kCombineThreadsSmall>, dim3(rows, splits),
+                                 dim3(opw::kCombineThreadsSmall), 0, stream, false, c)
+                        : launch(opw::combine_kernel<opw::kCombineThreads>, dim3(rows, splits),
+                                 dim3(opw::kCombineThreads), 0, stream, pdl, c);
+  if (e != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
   st->launches += 1;
   return OPW_OK;
 }
 
+static opw_status_t enqueue_attention(opw_attn_stage_t* st, int32_t layer, int32_t batch, const void* q,
+                                      const int32_t* kv_lens, const void* k_new, const void* v_new,
+                                      const int32_t* positions, const int32_t* page_table, void* out, float* lse,
+                                      void* cuda_stream) {
+  const StepArgs a = {layer, batch, q, kv_lens, k_new, v_new, positions, page_table, out, lse};
+  opw_status_t rc = validate_step(st, a);
+  if (rc != OPW_OK) return rc;
+  if (batch == 0) return OPW_OK;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  rc = launch_attention(st, a, 0, stream);
+  if (rc != OPW_OK) return rc;
+  return launch_combine(st, a, 0, stream, false);
+}
 
 opw_status_t opw_decode_attention(opw_attn_stage_t* st, int32_t layer, int32_t batch, const void* q,
                                   const int32_t* kv_lens, const int32_t* page_table, void* out, float* lse,
@@ -448,6 +482,8 @@ struct opw_attn_plan {
   opw_attn_stage* stage;
   std::vector<opw_step_item_t> items;
   uint32_t flags;
+  cudaStream_t side;                     // OPW_PLAN_OVERLAP: the combines run here
+  std::vector<cudaEvent_t> ev_attn, ev_comb;
   cudaGraph_t graph;
   cudaGraphExec_t exec;
   int64_t launches_per_submit;
@@ -457,8 +493,44 @@ namespace {
 
 // Enqueue the whole sequence on `stream`: for every item append then attention, then (with
 // OPW_PLAN_ADVANCE) one step forward for every distinct positions / kv_lens array.
-opw_status_t enqueue_plan(opw_attn_plan* pl, cudaStream_t stream) {
+// OPW_PLAN_OVERLAP: item i's combine runs on a side stream beside item i+1's split-KV kernel.
+// The two alternate between the stage's two workspace sets; item i+2's split-KV kernel waits
+// for item i's combine (same set); the main stream rejoins the side stream at the end.
+opw_status_t enqueue_plan_overlapped(opw_attn_plan* pl, cudaStream_t stream, cudaStream_t side) {
   opw_attn_stage* st = pl->stage;
+  const int n = (int)pl->items.size();
+  int last = -1;
+  for (int i = 0; i < n; ++i) {
+    const opw_step_item_t& it = pl->items[i];
+    if (it.batch == 0) continue;
+    const bool fused = it.k_new && !it.kv_lens;
+    if (it.k_new && !fused) {
+      opw_status_t rc = opw_kv_append(st, it.layer, it.batch, it.k_new, it.v_new, it.positions, it.page_table, stream);
+      if (rc != OPW_OK) return rc;
+    }
+    const StepArgs a = {it.layer, it.batch, it.q, fused ? nullptr : it.kv_lens, fused ? it.k_new : nullptr,
+                        fused ? it.v_new : nullptr, fused ? it.positions : nullptr, it.page_table, it.out, it.lse};
+    const int set = i & 1;
+    if (i >= 2 && cudaStreamWaitEvent(stream, pl->ev_comb[i - 2], 0) != cudaSuccess) return OPW_ERR_CUDA;
+    opw_status_t rc = launch_attention(st, a, set, stream);
+    if (rc != OPW_OK) return rc;
+    if (cudaEventRecord(pl->ev_attn[i], stream) != cudaSuccess || cudaStreamWaitEvent(side, pl->ev_attn[i], 0) != cudaSuccess)
+      return OPW_ERR_CUDA;
+    rc = launch_combine(st, a, set, side, true);
+    if (rc != OPW_OK) return rc;
+    if (cudaEventRecord(pl->ev_comb[i], side) != cudaSuccess) return OPW_ERR_CUDA;
+    last = i;
+  }
+  if (last >= 0 && cudaStreamWaitEvent(stream, pl->ev_comb[last], 0) != cudaSuccess) return OPW_ERR_CUDA;
+  return OPW_OK;
+}
+
+opw_status_t enqueue_plan(opw_attn_plan* pl, cudaStream_t stream, cudaStream_t side) {
+  opw_attn_stage* st = pl->stage;
+  if (pl->flags & OPW_PLAN_OVERLAP) {
+    opw_status_t rc = enqueue_plan_overlapped(pl, stream, side);
+    if (rc != OPW_OK) { (void)cudaGetLastError(); return rc; }
+  } else
   for (const opw_step_item_t& it : pl->items) {
     opw_status_t rc;
     if (it.k_new && !it.kv_lens) {              // one fused launch: append inside the attention kernel
@@ -501,7 +573,7 @@ extern "C" {
 opw_status_t opw_attn_plan_create(opw_attn_stage_t* st, const opw_step_item_t* items, int32_t n_items, uint32_t flags,
                                   opw_attn_plan_t** out) {
   if (!st || !items || n_items < 1 || !out) return OPW_ERR_INVALID_ARG;
-  if (flags & ~(uint32_t)(OPW_PLAN_GRAPH | OPW_PLAN_ADVANCE)) return OPW_ERR_INVALID_ARG;
+  if (flags & ~(uint32_t)(OPW_PLAN_GRAPH | OPW_PLAN_ADVANCE | OPW_PLAN_OVERLAP)) return OPW_ERR_INVALID_ARG;
   for (int i = 0; i < n_items; ++i) {
     const opw_step_item_t& it = items[i];
     opw_status_t rc = check_step(st, it.layer, it.batch);
@@ -514,11 +586,31 @@ opw_status_t opw_attn_plan_create(opw_attn_stage_t* st, const opw_step_item_t* i
     if (((uintptr_t)it.kv_lens | (uintptr_t)it.positions | (uintptr_t)it.page_table | (uintptr_t)it.lse) % 4)
       return OPW_ERR_INVALID_ARG;
   }
+  if (flags & OPW_PLAN_OVERLAP) {
+    // a step's combine runs beside the next step's attention: they must not share outputs
+    for (int i = 0; i + 1 < n_items; ++i)
+      if (items[i].out == items[i + 1].out || (items[i].lse && items[i].lse == items[i + 1].lse))
+        return OPW_ERR_INVALID_ARG;
+  }
   opw_attn_plan* pl = new (std::nothrow) opw_attn_plan();
   if (!pl) return OPW_ERR_INVALID_ARG;
   pl->stage = st;
   pl->items.assign(items, items + n_items);
   pl->flags = flags;
+  pl->side = nullptr;
+  if (flags & OPW_PLAN_OVERLAP) {
+    bool ok = cudaStreamCreateWithFlags(&pl->side, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; ok && i < 2 * n_items; ++i) {
+      cudaEvent_t ev = nullptr;
+      ok = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) == cudaSuccess;
+      if (ok) (i < n_items ? pl->ev_attn : pl->ev_comb).push_back(ev);
+    }
+    if (!ok) {
+      (void)cudaGetLastError();
+      opw_attn_plan_destroy(pl);
+      return OPW_ERR_CUDA;
+    }
+  }
   pl->graph = nullptr;
   pl->exec = nullptr;
   pl->launches_per_submit = 0;
@@ -528,7 +620,7 @@ opw_status_t opw_attn_plan_create(opw_attn_stage_t* st, const opw_step_item_t* i
     const int64_t before = st->launches;
     bool ok = cudaStreamCreateWithFlags(&cs, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaStreamBeginCapture(cs, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
-    opw_status_t rc = ok ? enqueue_plan(pl, cs) : OPW_ERR_CUDA;
+    opw_status_t rc = ok ? enqueue_plan(pl, cs, pl->side) : OPW_ERR_CUDA;
     if (ok) ok = cudaStreamEndCapture(cs, &pl->graph) == cudaSuccess && pl->graph != nullptr;
     if (ok && rc == OPW_OK) ok = cudaGraphInstantiate(&pl->exec, pl->graph, 0) == cudaSuccess;
     if (cs) cudaStreamDestroy(cs);
@@ -536,9 +628,7 @@ opw_status_t opw_attn_plan_create(opw_attn_stage_t* st, const opw_step_item_t* i
     st->launches = before;                      // captured, not launched
     if (!ok || rc != OPW_OK) {
       (void)cudaGetLastError();
-      if (pl->exec) cudaGraphExecDestroy(pl->exec);
-      if (pl->graph) cudaGraphDestroy(pl->graph);
-      delete pl;
+      opw_attn_plan_destroy(pl);
       return rc != OPW_OK ? rc : OPW_ERR_CUDA;
     }
   }
@@ -554,13 +644,16 @@ opw_status_t opw_attn_plan_submit(opw_attn_plan_t* pl, void* cuda_stream) {
     pl->stage->launches += pl->launches_per_submit;
     return OPW_OK;
   }
-  return enqueue_plan(pl, stream);
+  return enqueue_plan(pl, stream, pl->side);
 }
 
 opw_status_t opw_attn_plan_destroy(opw_attn_plan_t* pl) {
   if (!pl) return OPW_OK;
   if (pl->exec) cudaGraphExecDestroy(pl->exec);
   if (pl->graph) cudaGraphDestroy(pl->graph);
+  for (cudaEvent_t ev : pl->ev_attn) cudaEventDestroy(ev);
+  for (cudaEvent_t ev : pl->ev_comb) cudaEventDestroy(ev);
+  if (pl->side) cudaStreamDestroy(pl->side);
   delete pl;
   return OPW_OK;
 }

@@ -760,14 +760,17 @@ struct CombineParams {
   int32_t num_workers;
 };
 
-// One block of kCombineThreads per (sequence, kv head) row; thread t owns the output
-// elements t, t + kCombineThreads, ... of the row's [G, D] block.
+// One block of kCT threads per (sequence, kv head) row (and split); thread t owns the output
+// elements t, t + kCT, ... of the row's [G, D] block.  256 threads by default; the 128-thread
+// instance is small enough (registers) to share an SM with a split-KV block, which lets a plan
+// run a step's combine beside the next step's attention.
 constexpr int kCombineThreads = 256;
+constexpr int kCombineThreadsSmall = 128;
 constexpr int kCombineMaxG = 16;
 constexpr int kCombineBatch = 64;               // segments merged per pass
 // acc[j] = acc[j] * scale[h] + sum over the listed partials of weight * o, for the thread's
-// elements e = tid + j * kCombineThreads.  The loads of one pass are all independent.
-template <int NEL>
+// elements e = tid + j * kCT.  The loads of one pass are all independent.
+template <int NEL, int kCT>
 __device__ __forceinline__ void combine_accumulate(float* acc, const float* partials, const int32_t* seg_slot,
                                                    const float* w_s, const float* run_scale, int nseg, int64_t stride,
                                                    int G, int D, int GD) {
@@ -776,7 +779,7 @@ __device__ __forceinline__ void combine_accumulate(float* acc, const float* part
   bool ok[NEL];
 #pragma unroll
   for (int j = 0; j < NEL; ++j) {
-    const int e = threadIdx.x + j * kCombineThreads;
+    const int e = threadIdx.x + j * kCT;
     ok[j] = e < GD;
     hh[j] = ok[j] ? e / D : 0;
     acc[j] *= run_scale[hh[j]];
@@ -788,7 +791,7 @@ __device__ __forceinline__ void combine_accumulate(float* acc, const float* part
     for (int u = 0; u < US; ++u) {
       const float* sp = partials + (int64_t)seg_slot[sgm + u] * stride + threadIdx.x;
 #pragma unroll
-      for (int j = 0; j < NEL; ++j) o[j][u] = ok[j] ? __ldcg(sp + j * kCombineThreads) : 0.f;
+      for (int j = 0; j < NEL; ++j) o[j][u] = ok[j] ? __ldcg(sp + j * kCT) : 0.f;
     }
 #pragma unroll
     for (int u = 0; u < US; ++u)
@@ -799,7 +802,7 @@ __device__ __forceinline__ void combine_accumulate(float* acc, const float* part
     const float* sp = partials + (int64_t)seg_slot[sgm] * stride + threadIdx.x;
 #pragma unroll
     for (int j = 0; j < NEL; ++j)
-      if (ok[j]) acc[j] += w_s[sgm * G + hh[j]] * __ldcg(sp + j * kCombineThreads);
+      if (ok[j]) acc[j] += w_s[sgm * G + hh[j]] * __ldcg(sp + j * kCT);
   }
 }
 
@@ -808,7 +811,8 @@ __device__ __forceinline__ void combine_accumulate(float* acc, const float* part
 // block (row, y) merges every splits-th batch of the row's partials into one intermediate
 // partial in `scratch`, and the block that finishes last for the row (an atomic counter,
 // nothing waits) merges those `splits` intermediates and writes the output.
-__global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams p) {
+template <int kCT>
+__global__ void __launch_bounds__(kCT) combine_kernel(CombineParams p) {
   pdl_launch_dependents();
   const int row = blockIdx.x;
   const int splits = gridDim.y, split = blockIdx.y;
@@ -824,7 +828,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
   float* lse_row = p.lse ? p.lse + (int64_t)b * p.Hq + g * G : nullptr;
   if (n <= 0) {   // inactive slot: zeros, lse = -inf
     if (split == 0) {
-      for (int e = threadIdx.x; e < GD; e += kCombineThreads) ob[e] = __float2bfloat16(0.f);
+      for (int e = threadIdx.x; e < GD; e += kCT) ob[e] = __float2bfloat16(0.f);
       if (lse_row && threadIdx.x < G) lse_row[threadIdx.x] = -INFINITY;
     }
     return;
@@ -854,14 +858,14 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
   // A segment's partial for this row is in the segment's slot 0 if the segment starts inside
   // the row, else in slot 1.
   __shared__ int32_t seg_slot[kCombineBatch];
-  __shared__ int32_t warp_cnt[kCombineThreads / 32];
+  __shared__ int32_t warp_cnt[kCT / 32];
   __shared__ float w_s[kCombineBatch * kCombineMaxG];   // per (segment, head): m, then the weight
   __shared__ float l_s[kCombineBatch * kCombineMaxG];
   __shared__ float run_M[kCombineMaxG], run_L[kCombineMaxG], run_scale[kCombineMaxG];
   __shared__ int32_t is_last;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  constexpr int kMaxElems = kCombineMaxG * 128 / kCombineThreads;   // 8
-  const int nel = (GD + kCombineThreads - 1) / kCombineThreads;
+  constexpr int kMaxElems = kCombineMaxG * 128 / kCT;   // 8 (256 threads) or 16 (128 threads)
+  const int nel = (GD + kCT - 1) / kCT;
   float acc[kMaxElems];
 #pragma unroll
   for (int j = 0; j < kMaxElems; ++j) acc[j] = 0.f;
@@ -875,14 +879,14 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
   // One merge pass over `nseg` listed partials at `base_ptr` (slot stride `stride`): stage
   // (m, l), weights per head, then the weighted sums.
   auto merge_listed = [&](const float* base_ptr, int nseg) {
-    for (int idx = threadIdx.x; idx < nseg * G; idx += kCombineThreads) {   // stage (m, l): independent loads
+    for (int idx = threadIdx.x; idx < nseg * G; idx += kCT) {   // stage (m, l): independent loads
       const int sgm = idx / G, h = idx - sgm * G;
       const float* sp = base_ptr + (int64_t)seg_slot[sgm] * stride + GD;
       w_s[idx] = __ldcg(sp + h);
       l_s[idx] = __ldcg(sp + G + h);
     }
     __syncthreads();
-    for (int h = warp; h < G; h += kCombineThreads / 32) {   // a warp per head: max, weights, sum of l
+    for (int h = warp; h < G; h += kCT / 32) {   // a warp per head: max, weights, sum of l
       float Mc = run_M[h];
       for (int sgm = lane; sgm < nseg; sgm += 32) Mc = fmaxf(Mc, w_s[sgm * G + h]);
 #pragma unroll
@@ -904,10 +908,11 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
     }
     __syncthreads();
     // about 32 independent loads in flight per thread: NEL elements x (32 / NEL) segments
-    if (nel <= 1) combine_accumulate<1>(acc, base_ptr, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
-    else if (nel <= 2) combine_accumulate<2>(acc, base_ptr, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
-    else if (nel <= 4) combine_accumulate<4>(acc, base_ptr, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
-    else combine_accumulate<8>(acc, base_ptr, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
+    if (nel <= 1) combine_accumulate<1, kCT>(acc, base_ptr, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
+    else if (nel <= 2) combine_accumulate<2, kCT>(acc, base_ptr, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
+    else if (nel <= 4) combine_accumulate<4, kCT>(acc, base_ptr, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
+    else if (nel <= 8 || kMaxElems <= 8) combine_accumulate<(kMaxElems < 8 ? kMaxElems : 8), kCT>(acc, base_ptr, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
+    else combine_accumulate<kMaxElems, kCT>(acc, base_ptr, seg_slot, w_s, run_scale, nseg, stride, G, D, GD);
     __syncthreads();
   };
 
@@ -950,7 +955,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
     float* mine = p.scratch + ((int64_t)row * splits + split) * stride;
 #pragma unroll
     for (int j = 0; j < kMaxElems; ++j) {
-      const int e = threadIdx.x + j * kCombineThreads;
+      const int e = threadIdx.x + j * kCT;
       if (e < GD) __stcg(mine + e, acc[j]);
     }
     if (threadIdx.x < G) {
@@ -977,7 +982,7 @@ __global__ void __launch_bounds__(kCombineThreads) combine_kernel(CombineParams 
   }
 #pragma unroll
   for (int j = 0; j < kMaxElems; ++j) {
-    const int e = threadIdx.x + j * kCombineThreads;
+    const int e = threadIdx.x + j * kCT;
     if (e < GD) {
       const int h = e / D;
       const float Lh = run_L[h];

@@ -177,7 +177,7 @@ extern "C" opw_status_t opw_decode_attention_noalloc(int32_t num_q_heads, int32_
   c.max_pages = max_pages_per_seq;
   c.window = window;
   c.num_workers = d->sms * kWarps;
-  opw_na::combine_kernel<<<batch * num_kv_heads, opw_na::kCombineThreads, 0, stream>>>(c);
+  opw_na::combine_kernel<opw_na::kCombineThreads><<<batch * num_kv_heads, opw_na::kCombineThreads, 0, stream>>>(c);
   if (cudaGetLastError() != cudaSuccess) return OPW_ERR_CUDA;
   return OPW_OK;
 }

@@ -358,7 +358,8 @@ def test_host_buffer_step_matches_the_device_step():
 
 
 @pytest.mark.parametrize("fused", [False, True])
-@pytest.mark.parametrize("flags", [0, B.OPW_PLAN_GRAPH, B.OPW_PLAN_GRAPH | B.OPW_PLAN_ADVANCE, B.OPW_PLAN_ADVANCE])
+@pytest.mark.parametrize("flags", [0, B.OPW_PLAN_GRAPH, B.OPW_PLAN_GRAPH | B.OPW_PLAN_ADVANCE, B.OPW_PLAN_ADVANCE,
+                                   B.OPW_PLAN_OVERLAP, B.OPW_PLAN_GRAPH | B.OPW_PLAN_ADVANCE | B.OPW_PLAN_OVERLAP])
 def test_plan_submits_a_multi_layer_multi_microbatch_step_in_one_call(flags, fused):
     """Two layers (one windowed) x two microbatches, three decode steps, one native call per step."""
     wl = synth.Workload("p", 6, 32, 8, 128, [0, 48], "uniform_1024_4096", 78)
@@ -412,6 +413,19 @@ def test_plan_submits_a_multi_layer_multi_microbatch_step_in_one_call(flags, fus
     if flags & B.OPW_PLAN_ADVANCE:
         assert (pos[0].cpu().numpy() == lens[mbs[0]] + 3).all()
         assert fused or (kvl[1].cpu().numpy() == lens[mbs[1]] + 4).all()
+    B.opw_attn_plan_destroy(plan)
+    st.close()
+
+
+def test_overlapped_plan_needs_distinct_outputs_for_consecutive_items():
+    pool = torch.zeros(4 * 2 * 2 * 16 * 64, dtype=torch.bfloat16, device="cuda")
+    st = B.Stage(pools=[pool], layer_window=[0], num_q_heads=8, num_kv_heads=2, head_dim=64, max_batch=2, max_pages_per_seq=2)
+    x = pool.data_ptr()
+    item = dict(layer=0, batch=1, q=x, k_new=x, v_new=x, positions=x, page_table=x, out=x)
+    with pytest.raises(B.OpwError) as ei:
+        B.opw_attn_plan_create(st.handle, [item, dict(item)], B.OPW_PLAN_OVERLAP)
+    assert ei.value.status == B.OPW_ERR_INVALID_ARG
+    plan = B.opw_attn_plan_create(st.handle, [item, dict(item, out=x + 4096)], B.OPW_PLAN_OVERLAP)
     B.opw_attn_plan_destroy(plan)
     st.close()
 
