@@ -27,7 +27,7 @@ struct Shape {
 };
 
 struct Layout {          // byte offsets into the caller's workspace
-  size_t status, cum[2], partials[2], comb_scratch, row_count, st_q, st_k, st_v, st_pos, st_lens, st_out, st_lse, st_table, total;
+  size_t status, cum[2], partials[2], comb_scratch, row_count, st_q, st_k, st_v, st_pos, st_out, st_lse, st_table, total;
 };
 
 bool shape_ok(const opw_attn_stage_config_t* c) {
@@ -66,7 +66,6 @@ Layout carve(const opw_attn_stage_config_t* c, const Shape& s, int sms) {
   L.st_k = off;    off += align_up(B * Hkv * D * 2, 256);
   L.st_v = off;    off += align_up(B * Hkv * D * 2, 256);
   L.st_pos = off;  off += align_up(B * 4, 256);
-  L.st_lens = off; off += align_up(B * 4, 256);
   L.st_out = off;  off += align_up(B * Hq * D * 2, 256);
   L.st_lse = off;  off += align_up(B * Hq * 4, 256);
   L.st_table = off; off += align_up((size_t)c->num_layers * B * c->max_pages_per_seq * 4, 256);

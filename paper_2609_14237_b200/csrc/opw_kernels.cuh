@@ -276,12 +276,6 @@ __global__ void advance_kernel(int32_t* positions, int32_t* kv_lens, int32_t n) 
   }
 }
 
-// kv_lens = positions + 1 for the host-buffer step (inactive rows become 0)
-__global__ void lens_from_positions_kernel(const int32_t* pos, int32_t* lens, int32_t n) {
-  const int i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) lens[i] = pos[i] >= 0 ? pos[i] + 1 : 0;
-}
-
 // ---------------------------------------------------------------------------------
 // split-KV partial attention
 // ---------------------------------------------------------------------------------

@@ -3,7 +3,7 @@
 length, window), the operator profile a serving planner consumes for attention stages
 (paper, Section 4: stage latencies come from "profiled execution latency").
 
-    python -m paper_2609_14237_b200.profile_table [--out gpurun_out/attn_profile.json]
+    python -m paper_2609_14237_b200.profile_table [--out attn_profile.json]
 
 Every point runs the fused decode step (append + attention + combine) through a plan (CUDA
 graph, metadata advanced on the device) over enough identical layers that consecutive reads
@@ -70,7 +70,7 @@ def measure_point(batch, seq_len, window, Hq=32, Hkv=8, D=128, submits=30):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--out", default=os.path.join(ROOT, "gpurun_out", "attn_profile.json"))
+    ap.add_argument("--out", default="attn_profile.json")
     ap.add_argument("--batches", default="1,4,16,64,256")
     ap.add_argument("--seq-lens", default="1024,4096,16384,65536")
     ap.add_argument("--windows", default="0,4096")
@@ -97,7 +97,8 @@ def main():
                 r = measure_point(b, s, w)
                 rows.append(r)
                 print(json.dumps(r), flush=True)
-    os.makedirs(os.path.dirname(args.out), exist_ok=True)
+    if os.path.dirname(args.out):
+        os.makedirs(os.path.dirname(args.out), exist_ok=True)
     with open(args.out, "w") as fh:
         json.dump({"shape": {"num_q_heads": 32, "num_kv_heads": 8, "head_dim": 128, "page_size": 16}, "points": rows}, fh,
                   indent=1)
