@@ -41,7 +41,7 @@ DEFAULT_WORKLOAD = "c3_long_context"
 # launch / algorithmic bytes).  Workloads without a capture report null; the hybrid stack's
 # kernels are the same code on the same tile stream, but its 52 GB of pools are above the
 # size a capture may hold, so it has none.
-TRAFFIC_RATIO = {"c3_long_context": 1.0063, "c4_large_batch": 1.0137}
+TRAFFIC_RATIO = {"c2_llama8b": 1.011, "c3_long_context": 1.0038, "c4_large_batch": 1.0063}
 
 
 def measured_peak():

@@ -296,7 +296,7 @@ struct UnitDesc {   // one per lane, describing unit (window base + lane)
 };
 
 template <int D, bool HI>   // HI: query rows 8..15 of the MMA tile are in use (8 < G <= 16)
-__global__ void __launch_bounds__(kMaxWarps * 32, 1) attn_splitkv_kernel(AttnParams p) {
+__global__ void __maxnreg__(200) attn_splitkv_kernel(AttnParams p) {
   constexpr int KS = D / 16;                 // k-steps of Q*K^T
   constexpr int NT = D / 8;                  // n-tiles of P*V
   constexpr int ROWB = D * 2;                // bytes per token row
