@@ -63,8 +63,8 @@ typedef struct {
   int32_t device;                 /* CUDA ordinal the stage lives on */
   int32_t num_layers;             /* layers this stage owns (>= 1) */
   int32_t num_q_heads;            /* Hq */
-  int32_t num_kv_heads;           /* Hkv; Hq % Hkv == 0 and Hq / Hkv <= 16 */
-  int32_t head_dim;               /* D: 64 or 128 */
+  int32_t num_kv_heads;           /* Hkv; Hq % Hkv == 0 and Hq / Hkv <= 16 (<= 8 at head_dim 256) */
+  int32_t head_dim;               /* D: 64, 128 or 256 */
   int32_t page_size;              /* 16 */
   int32_t max_batch;              /* static slot count; every call has batch <= max_batch */
   int32_t max_pages_per_seq;      /* row stride (entries) of every page table */
@@ -78,7 +78,7 @@ typedef struct {
   size_t workspace_bytes;         /* >= opw_attn_stage_workspace_bytes(cfg) */
   float softmax_scale;            /* 0 -> 1/sqrt(head_dim) */
   uint32_t flags;                 /* OPW_FLAG_* */
-  int32_t tune_warps;             /* 0 = default; warps per thread block (1..8) */
+  int32_t tune_warps;             /* 0 = default (8; 6 at head_dim 256); warps per thread block (1..8) */
   int32_t tune_stages;            /* 0 = default; shared-memory ring depth per warp (2..16) */
   int32_t tune_ctas_per_sm;       /* 0 = default; resident thread blocks per SM (1..4) */
   int32_t reserved;               /* must be 0 */

@@ -36,7 +36,8 @@ bool shape_ok(const opw_attn_stage_config_t* c) {
 }
 
 opw_status_t resolve_shape(const opw_attn_stage_config_t* c, Shape* s) {
-  s->warps = c->tune_warps ? c->tune_warps : kDefaultWarps;
+  // head_dim 256 doubles the tile: six warps x two stages x 16 KB fill an SM's shared memory
+  s->warps = c->tune_warps ? c->tune_warps : (c->head_dim > 128 ? 6 : kDefaultWarps);
   s->stages = c->tune_stages ? c->tune_stages : kDefaultStages;
   s->ctas_per_sm = c->tune_ctas_per_sm ? c->tune_ctas_per_sm : kDefaultCtasPerSm;
   if (s->warps < 1 || s->warps > opw::kMaxWarps || s->stages < 2 || s->stages > 16 || s->ctas_per_sm < 1 ||
@@ -46,7 +47,9 @@ opw_status_t resolve_shape(const opw_attn_stage_config_t* c, Shape* s) {
 }
 
 size_t attn_smem_bytes(int D, const Shape& s, int batch) {
-  return D == 64 ? opw::AttnSmem<64>::bytes(s.warps, s.stages, batch) : opw::AttnSmem<128>::bytes(s.warps, s.stages, batch);
+  return D == 64    ? opw::AttnSmem<64>::bytes(s.warps, s.stages, batch)
+         : D == 128 ? opw::AttnSmem<128>::bytes(s.warps, s.stages, batch)
+                    : opw::AttnSmem<256>::bytes(s.warps, s.stages, batch);
 }
 
 Layout carve(const opw_attn_stage_config_t* c, const Shape& s, int sms) {
@@ -157,10 +160,10 @@ opw_status_t opw_attn_stage_create(const opw_attn_stage_config_t* cfg, opw_attn_
   if (cfg->struct_size != sizeof(opw_attn_stage_config_t) || cfg->reserved != 0) return OPW_ERR_INVALID_ARG;
   if (!shape_ok(cfg) || cfg->device < 0) return OPW_ERR_INVALID_ARG;
   if (!cfg->layer_window || !cfg->layer_num_pages || !cfg->layer_kv_pool || !cfg->workspace) return OPW_ERR_INVALID_ARG;
-  if (cfg->head_dim != 64 && cfg->head_dim != 128) return OPW_ERR_UNSUPPORTED;
+  if (cfg->head_dim != 64 && cfg->head_dim != 128 && cfg->head_dim != 256) return OPW_ERR_UNSUPPORTED;
   if (cfg->page_size != opw::kPage) return OPW_ERR_UNSUPPORTED;
   const int G = cfg->num_q_heads / cfg->num_kv_heads;
-  if (G > 16) return OPW_ERR_UNSUPPORTED;
+  if (G > 16 || (cfg->head_dim == 256 && G > 8)) return OPW_ERR_UNSUPPORTED;
   if (cfg->max_batch > 32768) return OPW_ERR_UNSUPPORTED;
   if ((int64_t)cfg->max_pages_per_seq * opw::kPage > INT32_MAX) return OPW_ERR_UNSUPPORTED;
   if (!(cfg->softmax_scale >= 0.f) || !std::isfinite(cfg->softmax_scale)) return OPW_ERR_INVALID_ARG;
@@ -191,10 +194,12 @@ opw_status_t opw_attn_stage_create(const opw_attn_stage_config_t* cfg, opw_attn_
     e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_i);
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_i);
-  } else {
+  } else if (cfg->head_dim == 128) {
     e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_i);
     if (e == cudaSuccess)
       e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_i);
+  } else {
+    e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_i);
   }
   if (e != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
   if (cudaMemset(cfg->workspace, 0, 256) != cudaSuccess ||
@@ -345,9 +350,11 @@ static opw_status_t launch_attention(opw_attn_stage_t* st, const StepArgs& a, in
   if (D == 64) {
     if (G > 8) e = launch(opw::attn_splitkv_kernel<64, true>, grid, block, smem, stream, pdl, p);
     else e = launch(opw::attn_splitkv_kernel<64, false>, grid, block, smem, stream, pdl, p);
-  } else {
+  } else if (D == 128) {
     if (G > 8) e = launch(opw::attn_splitkv_kernel<128, true>, grid, block, smem, stream, pdl, p);
     else e = launch(opw::attn_splitkv_kernel<128, false>, grid, block, smem, stream, pdl, p);
+  } else {
+    e = launch(opw::attn_splitkv_kernel<256, false>, grid, block, smem, stream, pdl, p);   // G <= 8 (checked at create)
   }
   if (e != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
   st->launches += 1;

@@ -296,7 +296,7 @@ struct UnitDesc {   // one per lane, describing unit (window base + lane)
 };
 
 template <int D, bool HI>   // HI: query rows 8..15 of the MMA tile are in use (8 < G <= 16)
-__global__ void __maxnreg__(200) attn_splitkv_kernel(AttnParams p) {
+__global__ void __maxnreg__(D > 128 ? 255 : 200) attn_splitkv_kernel(AttnParams p) {
   constexpr int KS = D / 16;                 // k-steps of Q*K^T
   constexpr int NT = D / 8;                  // n-tiles of P*V
   constexpr int ROWB = D * 2;                // bytes per token row
@@ -528,11 +528,20 @@ __global__ void __maxnreg__(200) attn_splitkv_kernel(AttnParams p) {
 
     // fused append: this unit is the page that receives the step's new key/value row
     const bool patch = p.k_new != nullptr && last && t1 > 0;
-    uint4 new_row = make_uint4(0u, 0u, 0u, 0u);
-    const int pc = lane & 15;                  // 16-byte group of the row; lanes 0..15 K, 16..31 V
-    if (patch && pc < D / 8) {
-      const __nv_bfloat16* src = (lane < 16 ? p.k_new : p.v_new) + ((int64_t)b * p.Hkv + g) * D + pc * 8;
-      new_row = *reinterpret_cast<const uint4*>(src);
+    // lanes 0..15 carry the K row, 16..31 the V row; a lane holds the row's 16-byte groups
+    // pc, pc + 16 (the second only for head_dim 256)
+    constexpr int NG = D / 8;                  // 16-byte groups per row
+    constexpr int GPL = (NG + 15) / 16;        // groups per lane
+    uint4 new_row[GPL];
+    const int pc = lane & 15;
+#pragma unroll
+    for (int i = 0; i < GPL; ++i) {
+      new_row[i] = make_uint4(0u, 0u, 0u, 0u);
+      if (patch && pc + 16 * i < NG) {
+        const __nv_bfloat16* src =
+            (lane < 16 ? p.k_new : p.v_new) + ((int64_t)b * p.Hkv + g) * D + (pc + 16 * i) * 8;
+        new_row[i] = *reinterpret_cast<const uint4*>(src);
+      }
     }
 
     // wait for this unit's tile
@@ -543,13 +552,18 @@ __global__ void __maxnreg__(200) attn_splitkv_kernel(AttnParams p) {
 
     const uint32_t tile = ring_base + slot * TILE;
     if (patch) {
-      if (pc < D / 8) {
-        const int tn = t1 - 1;                 // slot of the newest key inside this page
-        const uint32_t off = (uint32_t)((lane < 16 ? 0 : kPage * ROWB) + tn * ROWB + ((pc ^ (tn & 7)) << 4));
-        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(tile + off), "r"(new_row.x), "r"(new_row.y),
-                     "r"(new_row.z), "r"(new_row.w)
-                     : "memory");
-        *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(p.pool_w) + (int64_t)this_tile * TILE + off) = new_row;
+      const int tn = t1 - 1;                   // slot of the newest key inside this page
+#pragma unroll
+      for (int i = 0; i < GPL; ++i) {
+        const int c = pc + 16 * i;
+        if (c < NG) {
+          const uint32_t off = (uint32_t)((lane < 16 ? 0 : kPage * ROWB) + tn * ROWB + ((c ^ (tn & 7)) << 4));
+          asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(tile + off), "r"(new_row[i].x),
+                       "r"(new_row[i].y), "r"(new_row[i].z), "r"(new_row[i].w)
+                       : "memory");
+          *reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(p.pool_w) + (int64_t)this_tile * TILE + off) =
+              new_row[i];
+        }
       }
       __syncwarp();
     }

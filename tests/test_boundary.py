@@ -46,7 +46,7 @@ def test_status_strings():
 
 
 def test_pool_index_agrees_with_the_oracles_own_formula():
-    for Hkv, D in [(2, 64), (8, 128)]:
+    for Hkv, D in [(2, 64), (8, 128), (2, 256)]:
         for p in (0, 3):
             for g in range(Hkv):
                 for kv in range(2):
@@ -87,6 +87,8 @@ def test_workspace_bytes_needs_a_valid_shape():
     (dict(num_q_heads=7), B.OPW_ERR_INVALID_ARG),
     (dict(head_dim=96), B.OPW_ERR_UNSUPPORTED),
     (dict(page_size=32), B.OPW_ERR_UNSUPPORTED),
+    (dict(head_dim=256, num_q_heads=32, num_kv_heads=2), B.OPW_ERR_UNSUPPORTED),
+    (dict(head_dim=256, tune_warps=8), B.OPW_ERR_CAPACITY),
     (dict(num_q_heads=34, num_kv_heads=2), B.OPW_ERR_UNSUPPORTED),
     (dict(workspace=0), B.OPW_ERR_INVALID_ARG),
     (dict(workspace=0x100010), B.OPW_ERR_INVALID_ARG),

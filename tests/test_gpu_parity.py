@@ -116,7 +116,8 @@ def test_append_reports_bad_pages_without_writing():
 
 # --------------------------------------------------------------- attention ---
 
-@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 64), (32, 8, 128), (8, 8, 64), (64, 8, 128), (16, 1, 128), (24, 2, 64), (5, 1, 64)])
+@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 64), (32, 8, 128), (8, 8, 64), (64, 8, 128), (16, 1, 128), (24, 2, 64), (5, 1, 64),
+                                      (16, 2, 256), (4, 2, 256)])
 @pytest.mark.parametrize("window", [0, 40])
 def test_attention_small_shapes_match_the_oracle(Hq, Hkv, D, window):
     rng = np.random.default_rng(40 + Hq + D)
@@ -152,7 +153,7 @@ def test_config1_tiny_step_append_then_attention():
     st.close()
 
 
-@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 64), (32, 8, 128), (24, 2, 64)])
+@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 64), (32, 8, 128), (24, 2, 64), (16, 2, 256)])
 def test_fused_step_appends_bit_exactly_and_attends_over_the_new_key(Hq, Hkv, D):
     """opw_decode_step == opw_kv_append + opw_decode_attention: same pool bytes, same output."""
     wl = synth.Workload("f", 9, Hq, Hkv, D, [0, 40], "tiny", 79)
@@ -481,6 +482,19 @@ def test_many_short_sequences_fill_the_static_batch():
     # where half a bf16 ulp is already 1.6e-2.  The absolute bound is stated for the benchmark
     # configurations; here the bound relative to the value (2^-8 |ref|, in check_close) is the binding one.
     check_close(out_to_f64(out), ref, lse, ref_lse, max_abs=2.0 ** -8 * float(np.abs(ref).max()) + 1e-3)
+
+
+def test_head_dim_256_long_rows_full_and_windowed():
+    """16 query / 2 KV heads at head_dim 256 (the shape of a Qwen3-Next full-attention layer)."""
+    rng = np.random.default_rng(63)
+    Hq, Hkv, D = 16, 2, 256
+    lens = [30000, 41, 7000, 1]
+    pool, tab, q, _, _ = make_case(rng, lens, Hq, Hkv, D)
+    for window in (0, 4096):
+        ref, ref_lse, _ = oracle.decode_attention(pool, Hq, Hkv, D, P, q, lens, tab, window=window)
+        out, lse, rc, _ = gpu_attention(pool, tab, q, lens, Hq, Hkv, D, window=window)
+        assert rc == B.OPW_OK
+        check_close(out_to_f64(out), ref, lse, ref_lse)
 
 
 def test_sixteen_query_heads_per_kv_head_on_long_rows():

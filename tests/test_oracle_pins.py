@@ -54,7 +54,7 @@ def brute_force(q_bits, k_bits, v_bits, Hq, Hkv, D, lo, scale):
 
 # ------------------------------------------------------------------ layout ---
 
-@pytest.mark.parametrize("Hkv,D", [(2, 64), (8, 128), (1, 64)])
+@pytest.mark.parametrize("Hkv,D", [(2, 64), (8, 128), (1, 64), (2, 256)])
 def test_pool_index_is_a_bijection_with_contiguous_tiles(Hkv, D):
     pages = 3
     seen = np.zeros(oracle.pool_elems(pages, Hkv, P, D), dtype=np.int32)
@@ -163,7 +163,8 @@ def test_attention_matches_brute_force_grouped_heads_and_window():
             np.testing.assert_allclose(lse[b], ref_l, rtol=0, atol=1e-12)
 
 
-@pytest.mark.parametrize("Hq,Hkv,D,scale", [(8, 2, 64, None), (32, 8, 128, None), (16, 2, 128, 0.37), (4, 4, 64, None)])
+@pytest.mark.parametrize("Hq,Hkv,D,scale", [(8, 2, 64, None), (32, 8, 128, None), (16, 2, 128, 0.37), (4, 4, 64, None),
+                                            (16, 2, 256, None)])
 def test_attention_matches_torch_sdpa_float64_on_dense_pages(Hq, Hkv, D, scale):
     rng = np.random.default_rng(21)
     lens = [96, 96, 96]
