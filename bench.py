@@ -209,7 +209,7 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
     if world > 1:
         import torch.distributed as dist
 
-        tmax = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+        tmax = torch.tensor([total_ms], dtype=torch.float64, device=dev if dist.get_backend() == "nccl" else "cpu")
         dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
         total_ms = float(tmax.item())
     value = world * bytes_timed / (total_ms * 1e-3) / 1e9
@@ -270,7 +270,7 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
         if world > 1:
             import torch.distributed as dist
 
-            tmax = torch.tensor([e_ms], dtype=torch.float64, device=dev)
+            tmax = torch.tensor([e_ms], dtype=torch.float64, device=dev if dist.get_backend() == "nccl" else "cpu")
             dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
             e_ms = float(tmax.item())
         e_bytes = sum(kv_bytes_of_step(s) for s in range(base + 3, base + 3 + e2e_steps))
@@ -456,11 +456,18 @@ def main():
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the attention stage has no CPU path")
     binding.build()
+    # One rank per GPU.  OPW_BENCH_BACKEND=gloo (with fewer GPUs than ranks: ranks share devices)
+    # exists to exercise the multi-rank bookkeeping on a single-GPU machine; its numbers mean nothing.
+    backend = os.environ.get("OPW_BENCH_BACKEND", "nccl")
+    local = local % torch.cuda.device_count() if backend != "nccl" else local
     torch.cuda.set_device(local)
     if world > 1:
         import torch.distributed as dist
 
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        if backend == "nccl":
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        else:
+            dist.init_process_group(backend)
     steps = args.steps if args.steps is not None else 2000
     warmup = args.warmup if args.warmup is not None else 20
     tune = dict(tune_warps=args.warps, tune_stages=args.stages, tune_ctas_per_sm=args.ctas,
