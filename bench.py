@@ -241,10 +241,16 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
     }
 
     if want_e2e:
-        hq = [inp.q[i].cpu().pin_memory() for i in range(2)]
-        hk = [inp.k_new[i].cpu().pin_memory() for i in range(2)]
-        hv = [inp.v_new[i].cpu().pin_memory() for i in range(2)]
-        hpos = pos_all.cpu().pin_memory()
+        # q, k_new, v_new and positions of one call sit in one pinned buffer at the stage's packed
+        # offsets (they travel as one copy); the page table and the output have buffers of their own
+        packs = [[st.packed_host_buffers(B) for _ in range(R)] for _ in range(2)]
+        for i in range(2):
+            for l in range(R):
+                _, pq, pk, pv, _ = packs[i][l]
+                pq.copy_(inp.q[i, l].cpu())
+                pk.copy_(inp.k_new[i, l].cpu())
+                pv.copy_(inp.v_new[i, l].cpu())
+        hpos = pos_all.cpu()
         htab = [t.cpu().pin_memory() for t in inp.page_tables]
         hout = torch.empty(B, Hq, D, dtype=torch.bfloat16).pin_memory()
         base = warmup + steps
@@ -252,7 +258,9 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
         def host_step(s):
             layers, t = layer_round(s)
             for l in layers:
-                st.decode_step_host(l, hq[s & 1][l], hk[s & 1][l], hv[s & 1][l], hpos[t], htab[l], hout)
+                _, pq, pk, pv, ppos = packs[s & 1][l]
+                ppos.copy_(hpos[t])                  # this step's positions, written by the host
+                st.decode_step_host(l, pq, pk, pv, ppos, htab[l], hout)
             stream.synchronize()                     # the caller reads the result every step
 
         for s in range(base, base + 3):
@@ -274,7 +282,7 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
             dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
             e_ms = float(tmax.item())
         e_bytes = sum(kv_bytes_of_step(s) for s in range(base + 3, base + 3 + e2e_steps))
-        h2d = layers_per_step * (hq[0][0].numel() * 2 + 2 * hk[0][0].numel() * 2 + B * 4 + htab[0].numel() * 4)
+        h2d = layers_per_step * (B * Hq * D * 2 + 2 * B * Hkv * D * 2 + B * 4 + htab[0].numel() * 4)
         d2h = layers_per_step * hout.numel() * 2
         assert st.poll_error() == binding.OPW_OK
         res["e2e"] = {"value": round(world * e_bytes / (e_ms * 1e-3) / 1e9, 1), "unit": "GB/s", "steps": e2e_steps,

@@ -182,6 +182,17 @@ opw_status_t opw_decode_step(opw_attn_stage_t *stage, int32_t layer, int32_t bat
  * the stream has passed the step.  page_table_host == NULL reuses the table staged by
  * the previous call for this layer's slot (tables rarely change between steps).
  */
+/*
+ * Tensor packing for opw_decode_step_host (Section 6.2, low-overhead communication: many short
+ * transfers per token cost more than the bytes they carry).  Returns byte offsets inside one
+ * host buffer of total_bytes at which q, k_new, v_new and positions may be placed; when the
+ * four host pointers given to opw_decode_step_host sit at exactly these offsets of one buffer,
+ * they are sent with a single copy instead of four.  The offsets depend on the stage's
+ * max_batch and head counts only.
+ */
+opw_status_t opw_attn_stage_host_layout(const opw_attn_stage_t *stage, size_t *q_off, size_t *k_off, size_t *v_off,
+                                        size_t *pos_off, size_t *total_bytes);
+
 opw_status_t opw_decode_step_host(opw_attn_stage_t *stage, int32_t layer, int32_t batch, const void *q_host,
                                   const void *k_new_host, const void *v_new_host, const int32_t *positions_host,
                                   const int32_t *page_table_host, void *out_host, float *lse_host,

@@ -26,7 +26,7 @@ EXPORTS = [
     "opw_kv_append", "opw_decode_attention", "opw_decode_step_host", "opw_attn_stage_poll_error",
     "opw_attn_stage_launch_count", "opw_attn_stage_destroy", "opw_status_string", "opw_attn_stage_set_trace",
     "opw_decode_attention_noalloc", "opw_attn_plan_create", "opw_attn_plan_submit", "opw_attn_plan_destroy",
-    "opw_decode_step",
+    "opw_decode_step", "opw_attn_stage_host_layout",
 ]
 
 
@@ -123,6 +123,8 @@ def lib() -> ctypes.CDLL:
     L.opw_decode_attention.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp]
     L.opw_decode_step.restype = ctypes.c_int
     L.opw_decode_step.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.opw_attn_stage_host_layout.restype = ctypes.c_int
+    L.opw_attn_stage_host_layout.argtypes = [vp] + [ctypes.POINTER(ctypes.c_size_t)] * 5
     L.opw_decode_step_host.restype = ctypes.c_int
     L.opw_decode_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
     L.opw_attn_stage_poll_error.restype = ctypes.c_int
@@ -227,6 +229,13 @@ def opw_decode_step(stage: int, layer: int, batch: int, q: int, k_new: int, v_ne
                     page_table: int, out: int, lse: Optional[int] = None, stream: Optional[int] = None) -> None:
     _check(lib().opw_decode_step(stage, layer, batch, q, k_new, v_new, positions, page_table, out, lse, stream),
            "opw_decode_step")
+
+
+def opw_attn_stage_host_layout(stage: int):
+    """Returns (q_off, k_off, v_off, pos_off, total_bytes) of the packed host buffer."""
+    v = [ctypes.c_size_t(0) for _ in range(5)]
+    _check(lib().opw_attn_stage_host_layout(stage, *[ctypes.byref(x) for x in v]), "opw_attn_stage_host_layout")
+    return tuple(int(x.value) for x in v)
 
 
 def opw_decode_step_host(stage: int, layer: int, batch: int, q_host: int, k_new_host: int, v_new_host: int,
@@ -357,6 +366,20 @@ class Stage:
         self.trace = torch.zeros(n, 4, dtype=torch.int64, device=self.device)
         opw_attn_stage_set_trace(self.handle, self.trace.data_ptr(), self.trace.numel() * 8)
         return self.trace
+
+    def packed_host_buffers(self, batch):
+        """One pinned host buffer holding q, k_new, v_new, positions at the packed offsets;
+        returns (buffer, q, k_new, v_new, positions) -- the last four are views into it."""
+        import torch
+
+        qo, ko, vo, po, total = opw_attn_stage_host_layout(self.handle)
+        buf = torch.empty(total, dtype=torch.uint8).pin_memory()
+        Hq, Hkv, D = self.num_q_heads, self.num_kv_heads, self.head_dim
+        q = buf[qo:qo + batch * Hq * D * 2].view(torch.bfloat16).view(batch, Hq, D)
+        k = buf[ko:ko + batch * Hkv * D * 2].view(torch.bfloat16).view(batch, Hkv, D)
+        v = buf[vo:vo + batch * Hkv * D * 2].view(torch.bfloat16).view(batch, Hkv, D)
+        pos = buf[po:po + batch * 4].view(torch.int32)
+        return buf, q, k, v, pos
 
     def poll_error(self) -> int:
         return opw_attn_stage_poll_error(self.handle, self._stream())

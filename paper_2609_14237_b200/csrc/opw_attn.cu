@@ -428,6 +428,17 @@ opw_status_t opw_decode_step(opw_attn_stage_t* st, int32_t layer, int32_t batch,
   return enqueue_attention(st, layer, batch, q, nullptr, k_new, v_new, positions, page_table, out, lse, cuda_stream);
 }
 
+opw_status_t opw_attn_stage_host_layout(const opw_attn_stage_t* st, size_t* q_off, size_t* k_off, size_t* v_off,
+                                        size_t* pos_off, size_t* total_bytes) {
+  if (!st || !q_off || !k_off || !v_off || !pos_off || !total_bytes) return OPW_ERR_INVALID_ARG;
+  *q_off = 0;
+  *k_off = st->lay.st_k - st->lay.st_q;
+  *v_off = st->lay.st_v - st->lay.st_q;
+  *pos_off = st->lay.st_pos - st->lay.st_q;
+  *total_bytes = (st->lay.st_pos - st->lay.st_q) + (size_t)st->cfg.max_batch * 4;
+  return OPW_OK;
+}
+
 opw_status_t opw_decode_step_host(opw_attn_stage_t* st, int32_t layer, int32_t batch, const void* q_host,
                                   const void* k_new_host, const void* v_new_host, const int32_t* positions_host,
                                   const int32_t* page_table_host, void* out_host, float* lse_host, void* cuda_stream) {
@@ -448,10 +459,20 @@ opw_status_t opw_decode_step_host(opw_attn_stage_t* st, int32_t layer, int32_t b
   int32_t* d_table = reinterpret_cast<int32_t*>(ws + st->lay.st_table) + (size_t)layer * table_elems;
 
   bool ok = true;
-  ok &= cudaMemcpyAsync(d_q, q_host, B * Hq * D * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
-  ok &= cudaMemcpyAsync(d_k, k_new_host, B * Hkv * D * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
-  ok &= cudaMemcpyAsync(d_v, v_new_host, B * Hkv * D * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
-  ok &= cudaMemcpyAsync(d_pos, positions_host, B * 4, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  // Tensor packing: if the caller laid q, k_new, v_new and positions out in one host buffer at the
+  // offsets of opw_attn_stage_host_layout, they travel as a single copy.
+  const unsigned char* hq = static_cast<const unsigned char*>(q_host);
+  const bool packed = static_cast<const unsigned char*>(k_new_host) == hq + (st->lay.st_k - st->lay.st_q) &&
+                      static_cast<const unsigned char*>(v_new_host) == hq + (st->lay.st_v - st->lay.st_q) &&
+                      reinterpret_cast<const unsigned char*>(positions_host) == hq + (st->lay.st_pos - st->lay.st_q);
+  if (packed) {
+    ok &= cudaMemcpyAsync(d_q, q_host, (st->lay.st_pos - st->lay.st_q) + B * 4, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  } else {
+    ok &= cudaMemcpyAsync(d_q, q_host, B * Hq * D * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d_k, k_new_host, B * Hkv * D * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d_v, v_new_host, B * Hkv * D * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d_pos, positions_host, B * 4, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+  }
   if (page_table_host)
     ok &= cudaMemcpyAsync(d_table, page_table_host, B * st->cfg.max_pages_per_seq * 4, cudaMemcpyHostToDevice,
                           stream) == cudaSuccess;

@@ -527,7 +527,8 @@ __global__ void __maxnreg__(D > 128 ? 255 : 200) attn_splitkv_kernel(AttnParams 
     }
 
     // fused append: this unit is the page that receives the step's new key/value row
-    const bool patch = p.k_new != nullptr && last && t1 > 0;
+    // (not when kv_lens was clamped to the table: a position beyond the table appends nowhere)
+    const bool patch = p.k_new != nullptr && last && t1 > 0 && p.positions[b] + 1 == lens[b];
     // lanes 0..15 carry the K row, 16..31 the V row; a lane holds the row's 16-byte groups
     // pc, pc + 16 (the second only for head_dim 256)
     constexpr int NG = D / 8;                  // 16-byte groups per row

@@ -182,6 +182,25 @@ def test_fused_step_appends_bit_exactly_and_attends_over_the_new_key(Hq, Hkv, D)
     st.close()
 
 
+def test_fused_step_with_a_position_beyond_the_table_appends_nothing_for_that_row():
+    rng = np.random.default_rng(64)
+    Hq, Hkv, D = 8, 2, 64
+    pool_np, tab, q, _, _ = make_case(rng, [33, 48], Hq, Hkv, D)          # tables of 3 pages: 48 positions
+    k_new, v_new = rand_bits(rng, (2, Hkv, D)), rand_bits(rng, (2, Hkv, D))
+    pool = dev(pool_np, torch.bfloat16)
+    st = B.Stage(pools=[pool], layer_window=[0], num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, max_batch=2,
+                 max_pages_per_seq=tab.shape[1])
+    out = torch.empty(2, Hq, D, dtype=torch.bfloat16, device="cuda")
+    pos = np.array([32, 48], np.int32)                                    # row 1 points past its table
+    st.decode_step(0, dev(q, torch.bfloat16), dev(k_new, torch.bfloat16), dev(v_new, torch.bfloat16), dev(pos),
+                   dev(tab), out)
+    assert st.poll_error() == B.OPW_ERR_BAD_PAGE
+    ref = pool_np.copy()
+    oracle.kv_append(ref, Hkv, D, P, k_new, v_new, np.array([32, -1], np.int32), tab)
+    assert (pool.cpu().view(torch.int16).numpy().view(np.uint16) == ref).all()
+    st.close()
+
+
 def test_single_key_returns_v_bit_exactly():
     rng = np.random.default_rng(51)
     Hq, Hkv, D = 8, 2, 64
@@ -340,10 +359,17 @@ def test_host_buffer_step_matches_the_device_step():
                  max_batch=6, max_pages_per_seq=inp.max_pages_per_seq)
     for step in range(2):
         for layer in range(2):
-            q = inp.q[step, layer].pin_memory()
-            k = inp.k_new[step, layer].pin_memory()
-            v = inp.v_new[step, layer].pin_memory()
-            pos = torch.from_numpy(inp.positions(step)).pin_memory()
+            if layer == 0:                                # separate host buffers: four copies
+                q = inp.q[step, layer].pin_memory()
+                k = inp.k_new[step, layer].pin_memory()
+                v = inp.v_new[step, layer].pin_memory()
+                pos = torch.from_numpy(inp.positions(step)).pin_memory()
+            else:                                         # one packed host buffer: a single copy
+                _, q, k, v, pos = st.packed_host_buffers(6)
+                q.copy_(inp.q[step, layer])
+                k.copy_(inp.k_new[step, layer])
+                v.copy_(inp.v_new[step, layer])
+                pos.copy_(torch.from_numpy(inp.positions(step)))
             tab = inp.page_tables[layer].pin_memory()
             out = torch.empty(6, 32, 128, dtype=torch.bfloat16).pin_memory()
             lse = torch.empty(6, 32, dtype=torch.float32).pin_memory()
