@@ -255,6 +255,15 @@ opw_status_t opw_attn_plan_submit(opw_attn_plan_t *plan, void *cuda_stream);
 opw_status_t opw_attn_plan_destroy(opw_attn_plan_t *plan);
 
 /*
+ * Failure-detection self-test.  Enqueues a one-warp kernel that waits, with the same bounded
+ * wait the attention kernel uses for its shared-memory copies, on a barrier nothing will ever
+ * complete; after the bound (0.1 s) it records OPW_ERR_TIMEOUT in the status word and exits.
+ * The next opw_attn_stage_poll_error must return OPW_ERR_TIMEOUT, and the stage must keep
+ * working afterwards.  No fault, trap or endless loop is involved.
+ */
+opw_status_t opw_attn_stage_probe_timeout(opw_attn_stage_t *stage, void *cuda_stream);
+
+/*
  * Synchronises the stream, then returns and clears the device status word: OPW_OK, or
  * the first of OPW_ERR_BAD_PAGE / OPW_ERR_TIMEOUT recorded by a kernel since the last
  * poll.  The only entry point that blocks.

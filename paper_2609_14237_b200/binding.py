@@ -26,7 +26,7 @@ EXPORTS = [
     "opw_kv_append", "opw_decode_attention", "opw_decode_step_host", "opw_attn_stage_poll_error",
     "opw_attn_stage_launch_count", "opw_attn_stage_destroy", "opw_status_string", "opw_attn_stage_set_trace",
     "opw_decode_attention_noalloc", "opw_attn_plan_create", "opw_attn_plan_submit", "opw_attn_plan_destroy",
-    "opw_decode_step", "opw_attn_stage_host_layout",
+    "opw_decode_step", "opw_attn_stage_host_layout", "opw_attn_stage_probe_timeout",
 ]
 
 
@@ -127,6 +127,8 @@ def lib() -> ctypes.CDLL:
     L.opw_attn_stage_host_layout.argtypes = [vp] + [ctypes.POINTER(ctypes.c_size_t)] * 5
     L.opw_decode_step_host.restype = ctypes.c_int
     L.opw_decode_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.opw_attn_stage_probe_timeout.restype = ctypes.c_int
+    L.opw_attn_stage_probe_timeout.argtypes = [vp, vp]
     L.opw_attn_stage_poll_error.restype = ctypes.c_int
     L.opw_attn_stage_poll_error.argtypes = [vp, vp]
     L.opw_attn_stage_set_trace.restype = ctypes.c_int
@@ -276,6 +278,10 @@ def opw_attn_plan_submit(plan: int, stream: Optional[int] = None) -> None:
 
 def opw_attn_plan_destroy(plan: Optional[int]) -> None:
     _check(lib().opw_attn_plan_destroy(plan), "opw_attn_plan_destroy")
+
+
+def opw_attn_stage_probe_timeout(stage: int, stream: Optional[int] = None) -> None:
+    _check(lib().opw_attn_stage_probe_timeout(stage, stream), "opw_attn_stage_probe_timeout")
 
 
 def opw_attn_stage_poll_error(stage: int, stream: Optional[int] = None) -> int:

@@ -485,6 +485,15 @@ opw_status_t opw_decode_step_host(opw_attn_stage_t* st, int32_t layer, int32_t b
   return OPW_OK;
 }
 
+opw_status_t opw_attn_stage_probe_timeout(opw_attn_stage_t* st, void* cuda_stream) {
+  if (!st) return OPW_ERR_INVALID_ARG;
+  opw::wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      reinterpret_cast<uint32_t*>(st->ws + st->lay.status));
+  if (cudaGetLastError() != cudaSuccess) return OPW_ERR_CUDA;
+  st->launches += 1;
+  return OPW_OK;
+}
+
 opw_status_t opw_attn_stage_poll_error(opw_attn_stage_t* st, void* cuda_stream) {
   if (!st) return OPW_ERR_INVALID_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);

@@ -276,6 +276,22 @@ __global__ void advance_kernel(int32_t* positions, int32_t* kv_lens, int32_t n) 
   }
 }
 
+// Self-test of the bounded wait: one warp arms a shared-memory barrier for bytes that no copy
+// will ever deliver, waits for it the way the attention kernel waits for a tile, and must come
+// back after kWaitLimitNs with the time-out recorded in the status word.  Nothing is in
+// flight, so the kernel exits cleanly and the context stays usable.
+__global__ void wait_probe_kernel(uint32_t* status) {
+  __shared__ __align__(8) uint64_t bar;
+  const uint32_t b = smem_u32(&bar);
+  if (threadIdx.x == 0) {
+    mbar_init(b, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    mbar_expect_tx(b, 16);
+  }
+  __syncwarp();
+  if (!mbar_wait_bounded(b, 0) && threadIdx.x == 0) atomicOr(status, kErrTimeout);
+}
+
 // ---------------------------------------------------------------------------------
 // split-KV partial attention
 // ---------------------------------------------------------------------------------

@@ -2,6 +2,8 @@
 same seeded inputs.  Append and page indexing must be bit-exact; attention output must
 satisfy max |err| <= 1e-2 and mean |err| <= 1e-3 (bf16 in, fp32 accumulate, bf16 out),
 plus the tighter checks below (error relative to the output's rms, log-sum-exp)."""
+import time
+
 import numpy as np
 import pytest
 import torch
@@ -454,6 +456,28 @@ def test_overlapped_plan_needs_distinct_outputs_for_consecutive_items():
     assert ei.value.status == B.OPW_ERR_INVALID_ARG
     plan = B.opw_attn_plan_create(st.handle, [item, dict(item, out=x + 4096)], B.OPW_PLAN_OVERLAP)
     B.opw_attn_plan_destroy(plan)
+    st.close()
+
+
+def test_a_wait_that_runs_out_is_reported_and_the_stage_keeps_working():
+    """The bounded wait gives up after 0.1 s on a barrier nothing completes; no fault, no hang."""
+    rng = np.random.default_rng(65)
+    Hq, Hkv, D = 8, 2, 64
+    lens = [100, 3000]
+    pool_np, tab, q, _, _ = make_case(rng, lens, Hq, Hkv, D)
+    pool = dev(pool_np, torch.bfloat16)
+    st = B.Stage(pools=[pool], layer_window=[0], num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, max_batch=2,
+                 max_pages_per_seq=tab.shape[1])
+    t0 = time.perf_counter()
+    B.opw_attn_stage_probe_timeout(st.handle, torch.cuda.current_stream().cuda_stream)
+    assert st.poll_error() == B.OPW_ERR_TIMEOUT
+    assert 0.05 < time.perf_counter() - t0 < 5.0
+    assert st.poll_error() == B.OPW_OK                                   # cleared
+    out = torch.empty(2, Hq, D, dtype=torch.bfloat16, device="cuda")
+    st.decode_attention(0, dev(q, torch.bfloat16), dev(np.asarray(lens, np.int32)), dev(tab), out)
+    assert st.poll_error() == B.OPW_OK
+    ref, _, _ = oracle.decode_attention(pool_np, Hq, Hkv, D, P, q, lens, tab)
+    check_close(out_to_f64(out), ref)
     st.close()
 
 
