@@ -74,7 +74,8 @@ class ClockSampler(threading.Thread):
         except Exception as e:                                   # noqa: BLE001
             self.err = repr(e)
 
-    def run(self):
+    def sample(self):
+        """One reading of the SM clock and the throttle reasons."""
         if not self.ok:
             return
         nv = self.nv
@@ -84,18 +85,21 @@ class ClockSampler(threading.Thread):
             getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
             getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
         }
-        while not self.stop_flag:
+        try:
+            self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
             try:
-                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
-                try:
-                    mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
-                except Exception:                                # noqa: BLE001
-                    mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
-                for bit, name in names.items():
-                    if mask & bit:
-                        self.reasons.add(name)
+                mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
             except Exception:                                    # noqa: BLE001
-                pass
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+            for bit, name in names.items():
+                if mask & bit:
+                    self.reasons.add(name)
+        except Exception:                                        # noqa: BLE001
+            pass
+
+    def run(self):
+        while self.ok and not self.stop_flag:
+            self.sample()
             time.sleep(self.period)
 
     def result(self):
@@ -195,6 +199,7 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
     for s in range(warmup, warmup + steps):
         device_step(s, ev)
     t1.record(stream)
+    sampler.sample()                                # at least one reading while the GPU is still busy
     torch.cuda.synchronize()
     barrier()
     clocks = sampler.result()
