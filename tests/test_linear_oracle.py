@@ -19,8 +19,8 @@ def rand_case(rng, B, Hk, Hv, dk, dv, slots=None):
 
 
 def loops(state, slot, q, k, v, a, beta, scale):
-    B, Hk, dk = q.shape
-    Hv, dv = v.shape[1], v.shape[2]
+    B, Hk, dk = len(q), len(q[0]), len(q[0][0])
+    Hv, dv = len(v[0]), len(v[0][0])
     out = [[[0.0] * dv for _ in range(Hv)] for _ in range(B)]
     st = state.tolist()
     for b in range(B):
