@@ -348,6 +348,53 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
     return res
 
 
+def run_linear_layer(steps, batch=256, Hk=16, Hv=32, dk=128, dv=128, rotate=4):
+    """The recurrent-state (linear attention) decode step: state bytes read + written per second."""
+    import torch
+
+    from paper_2609_14237_b200 import binding
+
+    g = torch.Generator(device="cuda")
+    g.manual_seed(2001)
+    states = [torch.randn(batch, Hv, dk, dv, device="cuda", generator=g) for _ in range(rotate)]
+    q = torch.randn(batch, Hk, dk, device="cuda", generator=g).to(torch.bfloat16)
+    k = torch.nn.functional.normalize(torch.randn(batch, Hk, dk, device="cuda", generator=g), dim=-1).to(torch.bfloat16)
+    v = torch.randn(batch, Hv, dv, device="cuda", generator=g).to(torch.bfloat16)
+    a = torch.rand(batch, Hv, device="cuda", generator=g) * 0.1 + 0.9
+    beta = torch.rand(batch, Hv, device="cuda", generator=g)
+    slot = torch.arange(batch, dtype=torch.int32, device="cuda")
+    out = torch.empty(batch, Hv, dv, dtype=torch.bfloat16, device="cuda")
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        binding.opw_linear_attn_decode_step(batch=batch, num_k_heads=Hk, num_v_heads=Hv, dk=dk, dv=dv,
+                                            state=states[i % rotate].data_ptr(), num_slots=batch, slot=slot.data_ptr(),
+                                            q=q.data_ptr(), k=k.data_ptr(), v=v.data_ptr(), a=a.data_ptr(),
+                                            beta=beta.data_ptr(), out=out.data_ptr(), stream=stream.cuda_stream)
+
+    for i in range(5):
+        step(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(steps):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    nbytes = 2 * batch * Hv * dk * dv * 4
+    peak, kind = measured_peak()
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    return {"value": round(gbs, 1), "unit": "GB/s (state read + write)", "ms_per_step": round(ms, 5),
+            "seq_steps_per_s_per_layer": round(batch / (ms * 1e-3), 1), "state_bytes_per_step": nbytes // 2,
+            "config": {"batch": batch, "num_k_heads": Hk, "num_v_heads": Hv, "dk": dk, "dv": dv,
+                       "l2": f"rotating over {rotate} state sets, {rotate * nbytes / 2e9:.2f} GB between re-reads"},
+            "roofline": {"bound": "hbm", "achieved": round(gbs, 1), "peak": peak, "unit": "GB/s",
+                         "frac": round(gbs / peak, 4), "peak_kind": kind, "kernel": "opw_lin::decode_step_kernel",
+                         "traffic": None},
+            "steps": steps}
+
+
 def cpu_baseline(name, inp=None, budget_s=15.0, device="cpu"):
     """The fp64 oracle as it stands, timed on this machine's host cores over a bounded sample of
     the workload's sequences (layer 0, step 0); value in the metric's unit."""
@@ -505,6 +552,7 @@ def main():
                                                     "pct_of_nominal_8000", "roofline", "steps", "submit", "submit_overlap")
                             if key in r}
             others[name]["kv_bytes_per_step"] = r["config"]["kv_bytes_per_step"]
+        others["linear_state_layer"] = run_linear_layer(max(10, min(steps, 500)))
         res["other_workloads"] = others
     if world > 1:
         import torch.distributed as dist

@@ -38,9 +38,9 @@ extern "C" {
  *   slot       : DEVICE int32 [batch]; state slot of each sequence, < 0 = inactive row (its
  *                state is untouched and its output is 0); two rows must not name the same slot
  *   q, k       : DEVICE bf16 [batch, Hk, dk]
- *   v          : DEVICE bf16 [batch, Hv, dv]
+ *   v          : DEVICE bf16 [batch, Hv, dv], 8-byte aligned
  *   a, beta    : DEVICE float [batch, Hv]
- *   out        : DEVICE bf16 [batch, Hv, dv]
+ *   out        : DEVICE bf16 [batch, Hv, dv], 8-byte aligned
  *   scale      : read-out scale; 0 -> 1/sqrt(dk)
  * dk in {64, 128}, dv in {64, 128, 256} (a multiple of 32), Hv % Hk == 0; otherwise
  * OPW_ERR_UNSUPPORTED.  A slot id >= num_slots is skipped (output 0); no status word here.

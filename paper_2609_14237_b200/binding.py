@@ -15,8 +15,10 @@ from typing import Optional, Sequence
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 LIB_PATH = os.path.join(_HERE, "libopw_attn.so")
-SOURCES = [os.path.join(_HERE, "csrc", "opw_attn.cu"), os.path.join(_HERE, "csrc", "opw_noalloc.cu")]
-HEADERS = [os.path.join(_HERE, "csrc", "opw_kernels.cuh"), os.path.join(_ROOT, "include", "opw_attn.h")]
+SOURCES = [os.path.join(_HERE, "csrc", "opw_attn.cu"), os.path.join(_HERE, "csrc", "opw_noalloc.cu"),
+           os.path.join(_HERE, "csrc", "opw_linear_attn.cu")]
+HEADERS = [os.path.join(_HERE, "csrc", "opw_kernels.cuh"), os.path.join(_ROOT, "include", "opw_attn.h"),
+           os.path.join(_ROOT, "include", "opw_linear_attn.h")]
 
 OPW_FLAG_PDL = 1
 OPW_OK, OPW_ERR_INVALID_ARG, OPW_ERR_UNSUPPORTED, OPW_ERR_CAPACITY, OPW_ERR_CUDA, OPW_ERR_BAD_PAGE, OPW_ERR_TIMEOUT = range(7)
@@ -27,6 +29,7 @@ EXPORTS = [
     "opw_attn_stage_launch_count", "opw_attn_stage_destroy", "opw_status_string", "opw_attn_stage_set_trace",
     "opw_decode_attention_noalloc", "opw_attn_plan_create", "opw_attn_plan_submit", "opw_attn_plan_destroy",
     "opw_decode_step", "opw_attn_stage_host_layout", "opw_attn_stage_probe_timeout",
+    "opw_linear_attn_decode_step", "opw_linear_attn_state_bytes",
 ]
 
 
@@ -127,6 +130,10 @@ def lib() -> ctypes.CDLL:
     L.opw_attn_stage_host_layout.argtypes = [vp] + [ctypes.POINTER(ctypes.c_size_t)] * 5
     L.opw_decode_step_host.restype = ctypes.c_int
     L.opw_decode_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.opw_linear_attn_decode_step.restype = ctypes.c_int
+    L.opw_linear_attn_decode_step.argtypes = [i32, i32, i32, i32, i32, vp, i64, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp]
+    L.opw_linear_attn_state_bytes.restype = ctypes.c_size_t
+    L.opw_linear_attn_state_bytes.argtypes = [i32, i32, i32, i64]
     L.opw_attn_stage_probe_timeout.restype = ctypes.c_int
     L.opw_attn_stage_probe_timeout.argtypes = [vp, vp]
     L.opw_attn_stage_poll_error.restype = ctypes.c_int
@@ -278,6 +285,18 @@ def opw_attn_plan_submit(plan: int, stream: Optional[int] = None) -> None:
 
 def opw_attn_plan_destroy(plan: Optional[int]) -> None:
     _check(lib().opw_attn_plan_destroy(plan), "opw_attn_plan_destroy")
+
+
+def opw_linear_attn_decode_step(*, batch: int, num_k_heads: int, num_v_heads: int, dk: int, dv: int, state: int,
+                                num_slots: int, slot: int, q: int, k: int, v: int, a: int, beta: int, out: int,
+                                scale: float = 0.0, stream: Optional[int] = None) -> None:
+    """One in-place decode step of a recurrent-state layer (all arguments are device addresses)."""
+    _check(lib().opw_linear_attn_decode_step(batch, num_k_heads, num_v_heads, dk, dv, state, num_slots, slot, q, k, v,
+                                             a, beta, scale, out, stream), "opw_linear_attn_decode_step")
+
+
+def opw_linear_attn_state_bytes(num_v_heads: int, dk: int, dv: int, num_slots: int) -> int:
+    return int(lib().opw_linear_attn_state_bytes(num_v_heads, dk, dv, num_slots))
 
 
 def opw_attn_stage_probe_timeout(stage: int, stream: Optional[int] = None) -> None:
