@@ -530,6 +530,15 @@ def main():
             dist.init_process_group(backend)
     steps = args.steps if args.steps is not None else 2000
     warmup = args.warmup if args.warmup is not None else 20
+    if args.workload == "linear_state_layer":       # the recurrent-state layer alone (1 GPU)
+        r = run_linear_layer(max(10, min(steps, 2000)))
+        r.update({"metric": "recurrent-state layer decode: state GB/s (read + write)", "n_gpus": 1, "warmup": 5,
+                  "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+                  "gpu_launches": r["steps"]})
+        r["config"]["workload"] = "linear_state_layer"
+        if rank == 0:
+            print(json.dumps(r), flush=True)
+        return
     tune = dict(tune_warps=args.warps, tune_stages=args.stages, tune_ctas_per_sm=args.ctas,
                 flags=1 if args.pdl else 0)
     res = run_ours(args.workload, steps, max(3, warmup), args.rotate, tune, want_e2e=not args.no_e2e, want_submit=(world == 1), unfused=args.unfused,
