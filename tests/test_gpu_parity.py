@@ -496,6 +496,25 @@ def test_step_calls_validate_arguments_on_the_host():
     st.close()
 
 
+def test_read_sharing_rows_with_the_same_pages_and_query_agree():
+    """Two batch rows may read the same pages (a shared prefix): same table, same q, same result."""
+    rng = np.random.default_rng(66)
+    Hq, Hkv, D = 32, 8, 128
+    lens = [3000, 3000, 50, 3000]
+    pool, tab, q, _, _ = make_case(rng, lens, Hq, Hkv, D)
+    tab[1] = tab[0]
+    tab[3] = tab[0]
+    q[1] = q[0]
+    q[3] = q[0]
+    ref, ref_lse, _ = oracle.decode_attention(pool, Hq, Hkv, D, P, q, lens, tab)
+    out, lse, rc, _ = gpu_attention(pool, tab, q, lens, Hq, Hkv, D)
+    assert rc == B.OPW_OK
+    got = out_to_f64(out)
+    check_close(got, ref, lse, ref_lse)
+    # the rows are split at different places, so they agree to rounding, not bit for bit
+    assert np.abs(got[0] - got[1]).max() <= 2.0 ** -7 and np.abs(got[0] - got[3]).max() <= 2.0 ** -7
+
+
 def test_all_rows_inactive_and_one_key_batches():
     rng = np.random.default_rng(60)
     Hq, Hkv, D = 32, 8, 128
