@@ -57,6 +57,11 @@ WORKLOADS = {
     "c5_hybrid_stack": Workload(
         "c5_hybrid_stack", 128, 32, 8, 128, [4096, 4096, 4096, 0, 4096, 4096, 4096, 0],
         "uniform_8192_65536", 1005),
+    # not one of the five benchmark configurations: a stack shaped like the paper's first evaluated
+    # model (sliding-window : full = 5 : 1, 32 query / 16 KV heads of 128; the window, 1024, is an
+    # assumption -- the paper prints only the ratio), batch 64, contexts U[8192, 32768]
+    "m1_swa5to1_stack": Workload(
+        "m1_swa5to1_stack", 64, 32, 16, 128, [1024, 1024, 1024, 1024, 1024, 0], "uniform_8192_32768", 1101),
 }
 
 
