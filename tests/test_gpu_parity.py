@@ -203,6 +203,41 @@ def test_fused_step_with_a_position_beyond_the_table_appends_nothing_for_that_ro
     st.close()
 
 
+@pytest.mark.parametrize("fused", [True, False])
+def test_programmatic_dependent_launch_keeps_back_to_back_steps_ordered(fused):
+    """With OPW_FLAG_PDL every kernel may start while its predecessor finishes; eight steps enqueued
+    without a host synchronisation in between must still leave the exact pool and the right outputs."""
+    wl = synth.Workload("pdl", 8, 32, 8, 128, [0, 200], "uniform_1024_4096", 80)
+    inp = synth.make_inputs(wl, device="cpu", growth=4, steps=4)
+    pools = [p.cuda() for p in inp.pools]
+    refs = [oracle.as_u16(p).copy() for p in inp.pools]
+    st = B.Stage(pools=pools, layer_window=wl.layer_window, num_q_heads=32, num_kv_heads=8, head_dim=128,
+                 max_batch=8, max_pages_per_seq=inp.max_pages_per_seq, flags=B.OPW_FLAG_PDL)
+    tabs = [t.cuda() for t in inp.page_tables]
+    dq, dk, dv = inp.q.cuda(), inp.k_new.cuda(), inp.v_new.cuda()
+    pos = [dev(inp.positions(s)) for s in range(4)]
+    lens = [dev(inp.kv_lens(s)) for s in range(4)]
+    outs = torch.empty(4, 2, 8, 32, 128, dtype=torch.bfloat16, device="cuda")
+    for step in range(4):
+        for layer in range(2):
+            if fused:
+                st.decode_step(layer, dq[step, layer], dk[step, layer], dv[step, layer], pos[step], tabs[layer], outs[step, layer])
+            else:
+                st.kv_append(layer, dk[step, layer], dv[step, layer], pos[step], tabs[layer])
+                st.decode_attention(layer, dq[step, layer], lens[step], tabs[layer], outs[step, layer])
+    assert st.poll_error() == B.OPW_OK
+    for step in range(4):
+        for layer in range(2):
+            assert oracle.kv_append(refs[layer], 8, 128, P, inp.k_new[step, layer], inp.v_new[step, layer],
+                                    inp.positions(step), inp.page_tables[layer]) == 0
+            ref, _, _ = oracle.decode_attention(refs[layer], 32, 8, 128, P, inp.q[step, layer], inp.kv_lens(step),
+                                                inp.page_tables[layer], window=wl.layer_window[layer])
+            check_close(out_to_f64(outs[step, layer]), ref)
+    for layer in range(2):
+        assert (pools[layer].cpu().view(torch.int16).numpy().view(np.uint16) == refs[layer]).all()
+    st.close()
+
+
 def test_single_key_returns_v_bit_exactly():
     rng = np.random.default_rng(51)
     Hq, Hkv, D = 8, 2, 64
