@@ -50,6 +50,37 @@ opw_status_t opw_linear_attn_decode_step(int32_t batch, int32_t num_k_heads, int
                                          const void *k, const void *v, const float *a, const float *beta, float scale,
                                          void *out, void *cuda_stream);
 
+/*
+ * Mixed plans: one native submission (Section 6.2) for a hybrid stack that interleaves
+ * attention layers with recurrent-state layers.  An op is either one attention item (see
+ * opw_step_item_t in opw_attn.h) or one recurrent-state step with the arguments of
+ * opw_linear_attn_decode_step; ops run in the order given, one after the other.  Flags as for
+ * opw_attn_plan_create, except that OPW_PLAN_OVERLAP is not available (OPW_ERR_UNSUPPORTED);
+ * OPW_PLAN_ADVANCE touches the attention items' positions / kv_lens only.  Submit and destroy
+ * with opw_attn_plan_submit / opw_attn_plan_destroy.
+ */
+typedef struct {
+  int32_t batch, num_k_heads, num_v_heads, dk, dv;
+  float *state;
+  int64_t num_slots;
+  const int32_t *slot;
+  const void *q, *k, *v;
+  const float *a, *beta;
+  float scale;
+  void *out;
+} opw_linear_item_t;
+
+#define OPW_OP_ATTENTION 0
+#define OPW_OP_LINEAR 1
+typedef struct {
+  int32_t kind;                /* OPW_OP_ATTENTION or OPW_OP_LINEAR */
+  opw_step_item_t attention;   /* used when kind == OPW_OP_ATTENTION */
+  opw_linear_item_t linear;    /* used when kind == OPW_OP_LINEAR */
+} opw_plan_op_t;
+
+opw_status_t opw_attn_plan_create_mixed(opw_attn_stage_t *stage, const opw_plan_op_t *ops, int32_t n_ops,
+                                        uint32_t flags, opw_attn_plan_t **out);
+
 /* Host helper: bytes of the state of num_slots sequences. */
 size_t opw_linear_attn_state_bytes(int32_t num_v_heads, int32_t dk, int32_t dv, int64_t num_slots);
 

@@ -29,7 +29,7 @@ EXPORTS = [
     "opw_attn_stage_launch_count", "opw_attn_stage_destroy", "opw_status_string", "opw_attn_stage_set_trace",
     "opw_decode_attention_noalloc", "opw_attn_plan_create", "opw_attn_plan_submit", "opw_attn_plan_destroy",
     "opw_decode_step", "opw_attn_stage_host_layout", "opw_attn_stage_probe_timeout",
-    "opw_linear_attn_decode_step", "opw_linear_attn_state_bytes",
+    "opw_linear_attn_decode_step", "opw_linear_attn_state_bytes", "opw_attn_plan_create_mixed",
 ]
 
 
@@ -73,6 +73,21 @@ class StepItem(ctypes.Structure):
     ]
 
 
+class LinearItem(ctypes.Structure):
+    _fields_ = [
+        ("batch", ctypes.c_int32), ("num_k_heads", ctypes.c_int32), ("num_v_heads", ctypes.c_int32),
+        ("dk", ctypes.c_int32), ("dv", ctypes.c_int32),
+        ("state", ctypes.c_void_p), ("num_slots", ctypes.c_int64), ("slot", ctypes.c_void_p),
+        ("q", ctypes.c_void_p), ("k", ctypes.c_void_p), ("v", ctypes.c_void_p),
+        ("a", ctypes.c_void_p), ("beta", ctypes.c_void_p), ("scale", ctypes.c_float), ("out", ctypes.c_void_p),
+    ]
+
+
+class PlanOp(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int32), ("attention", StepItem), ("linear", LinearItem)]
+
+
+OPW_OP_ATTENTION, OPW_OP_LINEAR = 0, 1
 OPW_PLAN_GRAPH, OPW_PLAN_ADVANCE, OPW_PLAN_OVERLAP = 1, 2, 4
 
 
@@ -145,6 +160,8 @@ def lib() -> ctypes.CDLL:
                                                vp, vp]
     L.opw_attn_plan_create.restype = ctypes.c_int
     L.opw_attn_plan_create.argtypes = [vp, ctypes.POINTER(StepItem), i32, ctypes.c_uint32, ctypes.POINTER(vp)]
+    L.opw_attn_plan_create_mixed.restype = ctypes.c_int
+    L.opw_attn_plan_create_mixed.argtypes = [vp, ctypes.POINTER(PlanOp), i32, ctypes.c_uint32, ctypes.POINTER(vp)]
     L.opw_attn_plan_submit.restype = ctypes.c_int
     L.opw_attn_plan_submit.argtypes = [vp, vp]
     L.opw_attn_plan_destroy.restype = ctypes.c_int
@@ -276,6 +293,28 @@ def opw_attn_plan_create(stage: int, items: Sequence[dict], flags: int = 0) -> i
             setattr(a, k, it.get(k))
     h = ctypes.c_void_p()
     _check(lib().opw_attn_plan_create(stage, arr, len(items), flags, ctypes.byref(h)), "opw_attn_plan_create")
+    return h.value
+
+
+def opw_attn_plan_create_mixed(stage: int, ops: Sequence[dict], flags: int = 0) -> int:
+    """ops: dicts with kind "attention" (fields of an attention item) or "linear" (batch, num_k_heads,
+    num_v_heads, dk, dv, state, num_slots, slot, q, k, v, a, beta, out and optionally scale)."""
+    arr = (PlanOp * len(ops))()
+    for a, op in zip(arr, ops):
+        if op["kind"] == "attention":
+            a.kind = OPW_OP_ATTENTION
+            a.attention.layer, a.attention.batch = op["layer"], op["batch"]
+            for k in ("q", "k_new", "v_new", "positions", "kv_lens", "page_table", "out", "lse"):
+                setattr(a.attention, k, op.get(k))
+        else:
+            a.kind = OPW_OP_LINEAR
+            for k in ("batch", "num_k_heads", "num_v_heads", "dk", "dv", "num_slots"):
+                setattr(a.linear, k, int(op[k]))
+            for k in ("state", "slot", "q", "k", "v", "a", "beta", "out"):
+                setattr(a.linear, k, op[k])
+            a.linear.scale = float(op.get("scale", 0.0))
+    h = ctypes.c_void_p()
+    _check(lib().opw_attn_plan_create_mixed(stage, arr, len(ops), flags, ctypes.byref(h)), "opw_attn_plan_create_mixed")
     return h.value
 
 

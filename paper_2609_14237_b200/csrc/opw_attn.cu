@@ -2,6 +2,7 @@
 // carving, launches.  The library allocates no device memory and never synchronises
 // except in opw_attn_stage_poll_error and (once) in opw_attn_stage_create.
 #include "opw_attn.h"
+#include "opw_linear_attn.h"
 
 #include <cmath>
 #include <cstdlib>
@@ -517,6 +518,8 @@ opw_status_t opw_attn_stage_poll_error(opw_attn_stage_t* st, void* cuda_stream) 
 struct opw_attn_plan {
   opw_attn_stage* stage;
   std::vector<opw_step_item_t> items;
+  std::vector<opw_linear_item_t> linear;    // recurrent-state ops of a mixed plan ...
+  std::vector<int> linear_after;            // ... each runs after attention item linear_after[i] (-1: first)
   uint32_t flags;
   cudaStream_t side;                     // OPW_PLAN_OVERLAP: the combines run here
   std::vector<cudaEvent_t> ev_attn, ev_comb;
@@ -567,7 +570,18 @@ opw_status_t enqueue_plan(opw_attn_plan* pl, cudaStream_t stream, cudaStream_t s
     opw_status_t rc = enqueue_plan_overlapped(pl, stream, side);
     if (rc != OPW_OK) { (void)cudaGetLastError(); return rc; }
   } else
-  for (const opw_step_item_t& it : pl->items) {
+  for (int i = -1; i < (int)pl->items.size(); ++i) {
+    for (size_t j = 0; j < pl->linear.size(); ++j) {       // recurrent-state ops placed after item i
+      if (pl->linear_after[j] != i) continue;
+      const opw_linear_item_t& ln = pl->linear[j];
+      opw_status_t rl = opw_linear_attn_decode_step(ln.batch, ln.num_k_heads, ln.num_v_heads, ln.dk, ln.dv, ln.state,
+                                                    ln.num_slots, ln.slot, ln.q, ln.k, ln.v, ln.a, ln.beta, ln.scale,
+                                                    ln.out, stream);
+      if (rl != OPW_OK) return rl;
+      if (ln.batch > 0) st->launches += 1;
+    }
+    if (i + 1 >= (int)pl->items.size()) break;
+    const opw_step_item_t& it = pl->items[i + 1];
     opw_status_t rc;
     if (it.k_new && !it.kv_lens) {              // one fused launch: append inside the attention kernel
       rc = opw_decode_step(st, it.layer, it.batch, it.q, it.k_new, it.v_new, it.positions, it.page_table, it.out,
@@ -606,10 +620,12 @@ opw_status_t enqueue_plan(opw_attn_plan* pl, cudaStream_t stream, cudaStream_t s
 
 extern "C" {
 
-opw_status_t opw_attn_plan_create(opw_attn_stage_t* st, const opw_step_item_t* items, int32_t n_items, uint32_t flags,
-                                  opw_attn_plan_t** out) {
-  if (!st || !items || n_items < 1 || !out) return OPW_ERR_INVALID_ARG;
+static opw_status_t build_plan(opw_attn_stage_t* st, const opw_step_item_t* items, int32_t n_items,
+                               const opw_linear_item_t* linear, const int* linear_after, int32_t n_linear, uint32_t flags,
+                               opw_attn_plan_t** out) {
+  if (!st || !out || n_items < 0 || n_items + n_linear < 1 || (n_items > 0 && !items)) return OPW_ERR_INVALID_ARG;
   if (flags & ~(uint32_t)(OPW_PLAN_GRAPH | OPW_PLAN_ADVANCE | OPW_PLAN_OVERLAP)) return OPW_ERR_INVALID_ARG;
+  if ((flags & OPW_PLAN_OVERLAP) && n_linear > 0) return OPW_ERR_UNSUPPORTED;
   for (int i = 0; i < n_items; ++i) {
     const opw_step_item_t& it = items[i];
     opw_status_t rc = check_step(st, it.layer, it.batch);
@@ -631,7 +647,11 @@ opw_status_t opw_attn_plan_create(opw_attn_stage_t* st, const opw_step_item_t* i
   opw_attn_plan* pl = new (std::nothrow) opw_attn_plan();
   if (!pl) return OPW_ERR_INVALID_ARG;
   pl->stage = st;
-  pl->items.assign(items, items + n_items);
+  if (n_items > 0) pl->items.assign(items, items + n_items);
+  if (n_linear > 0) {
+    pl->linear.assign(linear, linear + n_linear);
+    pl->linear_after.assign(linear_after, linear_after + n_linear);
+  }
   pl->flags = flags;
   pl->side = nullptr;
   if (flags & OPW_PLAN_OVERLAP) {
@@ -670,6 +690,35 @@ opw_status_t opw_attn_plan_create(opw_attn_stage_t* st, const opw_step_item_t* i
   }
   *out = pl;
   return OPW_OK;
+}
+
+opw_status_t opw_attn_plan_create(opw_attn_stage_t* st, const opw_step_item_t* items, int32_t n_items, uint32_t flags,
+                                  opw_attn_plan_t** out) {
+  if (!items || n_items < 1) return OPW_ERR_INVALID_ARG;
+  return build_plan(st, items, n_items, nullptr, nullptr, 0, flags, out);
+}
+
+opw_status_t opw_attn_plan_create_mixed(opw_attn_stage_t* st, const opw_plan_op_t* ops, int32_t n_ops, uint32_t flags,
+                                        opw_attn_plan_t** out) {
+  if (!st || !ops || n_ops < 1 || !out) return OPW_ERR_INVALID_ARG;
+  std::vector<opw_step_item_t> items;
+  std::vector<opw_linear_item_t> linear;
+  std::vector<int> after;
+  for (int i = 0; i < n_ops; ++i) {
+    if (ops[i].kind == OPW_OP_ATTENTION) {
+      items.push_back(ops[i].attention);
+    } else if (ops[i].kind == OPW_OP_LINEAR) {
+      const opw_linear_item_t& ln = ops[i].linear;
+      if (ln.batch < 0 || !ln.state || !ln.slot || !ln.q || !ln.k || !ln.v || !ln.a || !ln.beta || !ln.out)
+        return OPW_ERR_INVALID_ARG;
+      linear.push_back(ln);
+      after.push_back((int)items.size() - 1);
+    } else {
+      return OPW_ERR_INVALID_ARG;
+    }
+  }
+  return build_plan(st, items.data(), (int32_t)items.size(), linear.data(), after.data(), (int32_t)linear.size(), flags,
+                    out);
 }
 
 opw_status_t opw_attn_plan_submit(opw_attn_plan_t* pl, void* cuda_stream) {

@@ -64,6 +64,83 @@ def test_qwen3_next_like_layer_batch_64():
     run_case(99, 64, 16, 32, 128, 128, slots=70, steps=2)
 
 
+@pytest.mark.parametrize("flags", [0, B.OPW_PLAN_GRAPH | B.OPW_PLAN_ADVANCE])
+def test_mixed_plan_runs_a_hybrid_stack_in_one_submission(flags):
+    """linear, full attention (fused append), linear -- two decode steps, one native call each."""
+    import sys, os
+    sys.path.insert(0, os.path.dirname(__file__))
+    from helpers import P
+    from paper_2609_14237_b200 import synth
+
+    B.build()
+    rng = np.random.default_rng(5)
+    Bn, Hk, Hv, dk, dv = 4, 2, 4, 128, 128
+    wl = synth.Workload("mix", Bn, 16, 2, 128, [0], "uniform_1024_4096", 81)
+    inp = synth.make_inputs(wl, device="cpu", growth=2, steps=2, lengths=np.array([40, 700, 1500, 16], np.int32))
+    pool = inp.pools[0].cuda()
+    ref_pool = oracle.as_u16(inp.pools[0]).copy()
+    st = B.Stage(pools=[pool], layer_window=[0], num_q_heads=16, num_kv_heads=2, head_dim=128, max_batch=Bn,
+                 max_pages_per_seq=inp.max_pages_per_seq)
+    states = [rng.standard_normal((Bn, Hv, dk, dv)).astype(np.float32) for _ in range(2)]
+    d_states = [torch.from_numpy(x.copy()).cuda() for x in states]
+    ref_states = [x.astype(np.float64) for x in states]
+    slot = torch.arange(Bn, dtype=torch.int32, device="cuda")
+    # static buffers
+    lq = [torch.empty(Bn, Hk, dk, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    lk = [torch.empty_like(t) for t in lq]
+    lv = [torch.empty(Bn, Hv, dv, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    la_ = [torch.empty(Bn, Hv, dtype=torch.float32, device="cuda") for _ in range(2)]
+    lb = [torch.empty_like(t) for t in la_]
+    lo = [torch.empty(Bn, Hv, dv, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+    aq = torch.empty(Bn, 16, 128, dtype=torch.bfloat16, device="cuda")
+    ak = torch.empty(Bn, 2, 128, dtype=torch.bfloat16, device="cuda")
+    av = torch.empty_like(ak)
+    ao = torch.empty_like(aq)
+    pos = torch.from_numpy(inp.positions(0)).cuda()
+    tab = inp.page_tables[0].cuda()
+
+    def lin(i):
+        return dict(kind="linear", batch=Bn, num_k_heads=Hk, num_v_heads=Hv, dk=dk, dv=dv, state=d_states[i].data_ptr(),
+                    num_slots=Bn, slot=slot.data_ptr(), q=lq[i].data_ptr(), k=lk[i].data_ptr(), v=lv[i].data_ptr(),
+                    a=la_[i].data_ptr(), beta=lb[i].data_ptr(), out=lo[i].data_ptr())
+
+    ops = [lin(0), dict(kind="attention", layer=0, batch=Bn, q=aq.data_ptr(), k_new=ak.data_ptr(), v_new=av.data_ptr(),
+                        positions=pos.data_ptr(), page_table=tab.data_ptr(), out=ao.data_ptr()), lin(1)]
+    plan = B.opw_attn_plan_create_mixed(st.handle, ops, flags)
+    f = lambda t: oracle.bf16_bits_to_f64(t.cpu().view(torch.int16).numpy().view(np.uint16))   # noqa: E731
+    for step in range(2):
+        host = []
+        for i in range(2):
+            q = rng.standard_normal((Bn, Hk, dk)); k = rng.standard_normal((Bn, Hk, dk))
+            k /= np.linalg.norm(k, axis=-1, keepdims=True)
+            v = rng.standard_normal((Bn, Hv, dv))
+            a = rng.uniform(0.8, 1.0, (Bn, Hv)).astype(np.float32); beta = rng.uniform(0, 1, (Bn, Hv)).astype(np.float32)
+            lq[i].copy_(bits_to_bf16(q)); lk[i].copy_(bits_to_bf16(k)); lv[i].copy_(bits_to_bf16(v))
+            la_[i].copy_(torch.from_numpy(a)); lb[i].copy_(torch.from_numpy(beta))
+            host.append((a, beta))
+        aq.copy_(inp.q[step, 0]); ak.copy_(inp.k_new[step, 0]); av.copy_(inp.v_new[step, 0])
+        if not flags & B.OPW_PLAN_ADVANCE:
+            pos.copy_(torch.from_numpy(inp.positions(step)))
+        B.opw_attn_plan_submit(plan, torch.cuda.current_stream().cuda_stream)
+        assert st.poll_error() == B.OPW_OK
+        for i in range(2):
+            a, beta = host[i]
+            ref = la.decode_step(ref_states[i], np.arange(Bn), f(lq[i]), f(lk[i]), f(lv[i]), a.astype(np.float64),
+                                 beta.astype(np.float64))
+            got = f(lo[i])
+            assert (np.abs(got - ref) <= 2.0 ** -8 * np.abs(ref) + 2e-3).all()
+            gs = d_states[i].cpu().numpy().astype(np.float64)
+            assert (np.abs(gs - ref_states[i]) <= 2e-5 * (1 + np.abs(ref_states[i]))).all()
+            ref_states[i] = gs
+        assert oracle.kv_append(ref_pool, 2, 128, P, inp.k_new[step, 0], inp.v_new[step, 0], inp.positions(step),
+                                inp.page_tables[0]) == 0
+        assert (pool.cpu().view(torch.int16).numpy().view(np.uint16) == ref_pool).all()
+        ref, _, _ = oracle.decode_attention(ref_pool, 16, 2, 128, P, inp.q[step, 0], inp.kv_lens(step), inp.page_tables[0])
+        assert np.abs(f(ao) - ref).max() <= 1e-2
+    B.opw_attn_plan_destroy(plan)
+    st.close()
+
+
 def test_argument_checks():
     B.build()
     L = B.lib()
