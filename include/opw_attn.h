@@ -114,6 +114,15 @@ size_t opw_attn_stage_workspace_bytes(const opw_attn_stage_config_t *cfg);
 opw_status_t opw_attn_stage_create(const opw_attn_stage_config_t *cfg, opw_attn_stage_t **out);
 
 /*
+ * Reads back the static shape a stage was bound with (Section 6: the shapes are fixed at
+ * bind time): device ordinal, layer count, Hq, Hkv, D and max_batch.  Any out pointer may be
+ * NULL.  For code layered on a stage that has only the opaque handle.
+ */
+opw_status_t opw_attn_stage_shape(const opw_attn_stage_t *stage, int32_t *device, int32_t *num_layers,
+                                  int32_t *num_q_heads, int32_t *num_kv_heads, int32_t *head_dim,
+                                  int32_t *max_batch);
+
+/*
  * KV append (Section 6: KV-cache contents and metadata change every iteration).  For
  * every b < batch with positions[b] >= 0, copies k_new[b] and v_new[b] bit for bit into
  * slot positions[b] % page_size of page page_table[b][positions[b] / page_size] of the

@@ -16,9 +16,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 LIB_PATH = os.path.join(_HERE, "libopw_attn.so")
 SOURCES = [os.path.join(_HERE, "csrc", "opw_attn.cu"), os.path.join(_HERE, "csrc", "opw_noalloc.cu"),
-           os.path.join(_HERE, "csrc", "opw_linear_attn.cu")]
+           os.path.join(_HERE, "csrc", "opw_linear_attn.cu"), os.path.join(_HERE, "csrc", "opw_afd.cu")]
 HEADERS = [os.path.join(_HERE, "csrc", "opw_kernels.cuh"), os.path.join(_ROOT, "include", "opw_attn.h"),
-           os.path.join(_ROOT, "include", "opw_linear_attn.h")]
+           os.path.join(_ROOT, "include", "opw_linear_attn.h"), os.path.join(_ROOT, "include", "opw_afd.h")]
 
 OPW_FLAG_PDL = 1
 OPW_OK, OPW_ERR_INVALID_ARG, OPW_ERR_UNSUPPORTED, OPW_ERR_CAPACITY, OPW_ERR_CUDA, OPW_ERR_BAD_PAGE, OPW_ERR_TIMEOUT = range(7)
@@ -30,6 +30,8 @@ EXPORTS = [
     "opw_decode_attention_noalloc", "opw_attn_plan_create", "opw_attn_plan_submit", "opw_attn_plan_destroy",
     "opw_decode_step", "opw_attn_stage_host_layout", "opw_attn_stage_probe_timeout",
     "opw_linear_attn_decode_step", "opw_linear_attn_state_bytes", "opw_attn_plan_create_mixed",
+    "opw_attn_stage_shape", "opw_afd_module_workspace_bytes", "opw_afd_module_create", "opw_afd_module_step",
+    "opw_afd_module_intermediates", "opw_afd_module_destroy",
 ]
 
 
@@ -101,6 +103,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [
         "nvcc", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
         "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(_ROOT, "include"), "-o", tmp, *srcs,
+        "-lcublasLt",
     ]
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
@@ -166,6 +169,18 @@ def lib() -> ctypes.CDLL:
     L.opw_attn_plan_submit.argtypes = [vp, vp]
     L.opw_attn_plan_destroy.restype = ctypes.c_int
     L.opw_attn_plan_destroy.argtypes = [vp]
+    L.opw_attn_stage_shape.restype = ctypes.c_int
+    L.opw_attn_stage_shape.argtypes = [vp] + [ctypes.POINTER(i32)] * 6
+    L.opw_afd_module_workspace_bytes.restype = ctypes.c_size_t
+    L.opw_afd_module_workspace_bytes.argtypes = [i32, i32, i32, i32]
+    L.opw_afd_module_create.restype = ctypes.c_int
+    L.opw_afd_module_create.argtypes = [vp, i32, i32, vp, vp, ctypes.c_float, vp, ctypes.c_size_t, ctypes.POINTER(vp)]
+    L.opw_afd_module_step.restype = ctypes.c_int
+    L.opw_afd_module_step.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+    L.opw_afd_module_intermediates.restype = ctypes.c_int
+    L.opw_afd_module_intermediates.argtypes = [vp] + [ctypes.POINTER(vp)] * 4
+    L.opw_afd_module_destroy.restype = ctypes.c_int
+    L.opw_afd_module_destroy.argtypes = [vp]
     L.opw_attn_stage_launch_count.restype = i64
     L.opw_attn_stage_launch_count.argtypes = [vp]
     L.opw_attn_stage_destroy.restype = ctypes.c_int
@@ -357,6 +372,42 @@ def opw_attn_stage_launch_count(stage: int) -> int:
     return int(lib().opw_attn_stage_launch_count(stage))
 
 
+def opw_attn_stage_shape(stage: int) -> dict:
+    """The static shape the stage was bound with."""
+    names = ("device", "num_layers", "num_q_heads", "num_kv_heads", "head_dim", "max_batch")
+    vals = [ctypes.c_int32(0) for _ in names]
+    _check(lib().opw_attn_stage_shape(stage, *[ctypes.byref(v) for v in vals]), "opw_attn_stage_shape")
+    return {n: int(v.value) for n, v in zip(names, vals)}
+
+
+def opw_afd_module_workspace_bytes(num_q_heads: int, num_kv_heads: int, head_dim: int, max_batch: int) -> int:
+    return int(lib().opw_afd_module_workspace_bytes(num_q_heads, num_kv_heads, head_dim, max_batch))
+
+
+def opw_afd_module_create(stage: int, layer: int, hidden: int, w_qkv: int, w_o: int, rope_theta: float,
+                          workspace: int, workspace_bytes: int) -> int:
+    h = ctypes.c_void_p()
+    _check(lib().opw_afd_module_create(stage, layer, hidden, w_qkv, w_o, rope_theta, workspace, workspace_bytes,
+                                       ctypes.byref(h)), "opw_afd_module_create")
+    return h.value
+
+
+def opw_afd_module_step(module: int, batch: int, x: int, positions: int, page_table: int, y: int,
+                        stream: Optional[int] = None) -> None:
+    _check(lib().opw_afd_module_step(module, batch, x, positions, page_table, y, stream), "opw_afd_module_step")
+
+
+def opw_afd_module_intermediates(module: int):
+    """Device addresses (q, k_new, v_new, attn_out) of the last step's intermediates."""
+    ptrs = [ctypes.c_void_p() for _ in range(4)]
+    _check(lib().opw_afd_module_intermediates(module, *[ctypes.byref(p) for p in ptrs]), "opw_afd_module_intermediates")
+    return tuple(p.value for p in ptrs)
+
+
+def opw_afd_module_destroy(module: Optional[int]) -> None:
+    _check(lib().opw_afd_module_destroy(module), "opw_afd_module_destroy")
+
+
 def opw_attn_stage_destroy(stage: Optional[int]) -> None:
     _check(lib().opw_attn_stage_destroy(stage), "opw_attn_stage_destroy")
 
@@ -454,6 +505,56 @@ class Stage:
     def close(self):
         if getattr(self, "handle", None):
             opw_attn_stage_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class AfdModule:
+    """Owner of one complete-attention-module handle (projections + rotary encoding + the stage's
+    core attention) over torch tensors; forwards to the opw_afd_module_* entry points."""
+
+    def __init__(self, stage: Stage, layer: int, w_qkv, w_o, rope_theta: float = 10000.0):
+        import torch
+
+        shp = opw_attn_stage_shape(stage.handle)
+        self.stage, self.w_qkv, self.w_o = stage, w_qkv, w_o
+        self.hidden = int(w_qkv.shape[1])
+        n_qkv = (shp["num_q_heads"] + 2 * shp["num_kv_heads"]) * shp["head_dim"]
+        if tuple(w_qkv.shape) != (n_qkv, self.hidden) or tuple(w_o.shape) != (self.hidden, shp["num_q_heads"] * shp["head_dim"]):
+            raise ValueError("weight shapes do not match the stage")
+        if w_qkv.dtype != torch.bfloat16 or w_o.dtype != torch.bfloat16 or not (w_qkv.is_contiguous() and w_o.is_contiguous()):
+            raise ValueError("weights must be contiguous bf16")
+        nbytes = opw_afd_module_workspace_bytes(shp["num_q_heads"], shp["num_kv_heads"], shp["head_dim"], shp["max_batch"])
+        self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=stage.device)
+        base = (self.workspace.data_ptr() + 255) // 256 * 256
+        self.shape = shp
+        self.handle = opw_afd_module_create(stage.handle, layer, self.hidden, w_qkv.data_ptr(), w_o.data_ptr(),
+                                            rope_theta, base, nbytes)
+
+    def step(self, x, positions, page_table, y):
+        opw_afd_module_step(self.handle, positions.shape[0], x.data_ptr(), positions.data_ptr(), page_table.data_ptr(),
+                            y.data_ptr(), Stage._stream())
+
+    def intermediates(self, batch: int):
+        """Copies of the last step's q, k_new, v_new and attention output as torch tensors."""
+        import torch
+
+        Hq, Hkv, D = self.shape["num_q_heads"], self.shape["num_kv_heads"], self.shape["head_dim"]
+        base = self.workspace.data_ptr()
+        out = []
+        for ptr, heads in zip(opw_afd_module_intermediates(self.handle), (Hq, Hkv, Hkv, Hq)):
+            off = ptr - base
+            out.append(self.workspace[off:off + batch * heads * D * 2].view(torch.bfloat16).view(batch, heads, D).clone())
+        return tuple(out)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            opw_afd_module_destroy(self.handle)
             self.handle = None
 
     def __del__(self):

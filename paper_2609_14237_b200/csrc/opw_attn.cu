@@ -429,6 +429,18 @@ opw_status_t opw_decode_step(opw_attn_stage_t* st, int32_t layer, int32_t batch,
   return enqueue_attention(st, layer, batch, q, nullptr, k_new, v_new, positions, page_table, out, lse, cuda_stream);
 }
 
+opw_status_t opw_attn_stage_shape(const opw_attn_stage_t* st, int32_t* device, int32_t* num_layers, int32_t* Hq,
+                                  int32_t* Hkv, int32_t* D, int32_t* max_batch) {
+  if (!st) return OPW_ERR_INVALID_ARG;
+  if (device) *device = st->cfg.device;
+  if (num_layers) *num_layers = st->cfg.num_layers;
+  if (Hq) *Hq = st->cfg.num_q_heads;
+  if (Hkv) *Hkv = st->cfg.num_kv_heads;
+  if (D) *D = st->cfg.head_dim;
+  if (max_batch) *max_batch = st->cfg.max_batch;
+  return OPW_OK;
+}
+
 opw_status_t opw_attn_stage_host_layout(const opw_attn_stage_t* st, size_t* q_off, size_t* k_off, size_t* v_off,
                                         size_t* pos_off, size_t* total_bytes) {
   if (!st || !q_off || !k_off || !v_off || !pos_off || !total_bytes) return OPW_ERR_INVALID_ARG;

@@ -1,0 +1,170 @@
+"""GPU parity of the complete attention module (projections + rotary encoding + core attention)
+against its fp64 oracle, through the C ABI.
+
+The module is checked stage by stage, each stage fed with the GPU's own previous result so that a
+one-ulp rounding flip upstream is not counted again downstream, and once end to end:
+  q, k, v   : both sides round the GEMM result to bf16, rotate, and round again; fp32 against fp64
+              accumulation can flip either rounding by one ulp (<= 2^-7 relative).  A flipped input
+              pair (x0, x1) moves the rotated value by <= 2^-7 (|x0| + |x1|) <= 2^-7 sqrt(2) (|ref| +
+              |partner|), partner being the other element of the rotated pair, and the second flip adds
+              2^-7 |ref|: |err| <= 2.5 * 2^-7 * (|ref| + |partner|).
+              v is not rotated: |err| <= 2^-7 |ref| (one flip)
+  append    : the pool afterwards holds the GPU's k, v rows bit for bit
+  attention : the stated core-attention tolerance, oracle run on the GPU's q and that pool
+  y         : a K-term fp32 dot product rounded to bf16: |err| <= 2^-8 |ref| + 2^-10 * rms(y)
+  end to end: independent roundings of relative size 2^-9 (attention output, probabilities, q/k/v)
+              pass through a projection that averages them: max |err| <= 2^-5 rms(y) + 2^-8 |ref|,
+              mean |err| <= 2^-7 rms(y)
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import P, make_case
+from oracle import afd
+from paper_2609_14237_b200 import binding as B
+
+pytestmark = pytest.mark.gpu
+THETA = 10000.0
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    B.build()
+    assert torch.cuda.is_available()
+
+
+def to_dev_bf16(bits):
+    return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).view(torch.bfloat16).cuda()
+
+
+def f64(t):
+    return oracle.bf16_bits_to_f64(t.cpu().contiguous().view(torch.int16).numpy().view(np.uint16))
+
+
+def tobits(t):
+    return t.cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def run_module(seed, lens, Hq, Hkv, D, hidden, steps=2, inactive=(), window=0, batches=None):
+    rng = np.random.default_rng(seed)
+    Bn = len(lens)
+    lens = np.asarray(lens, np.int32)
+    pool_np, tab, _, _, _ = make_case(rng, [int(n) + steps for n in lens], Hq, Hkv, D)
+    n_qkv = (Hq + 2 * Hkv) * D
+    w_qkv_bits = oracle.f32_to_bf16_bits((rng.standard_normal((n_qkv, hidden)) / np.sqrt(hidden)).astype(np.float32))
+    w_o_bits = oracle.f32_to_bf16_bits((rng.standard_normal((hidden, Hq * D)) / np.sqrt(Hq * D)).astype(np.float32))
+    w_qkv, w_o = oracle.bf16_bits_to_f64(w_qkv_bits), oracle.bf16_bits_to_f64(w_o_bits)
+
+    pool = to_dev_bf16(pool_np)
+    d_tab = torch.from_numpy(tab).cuda()
+    stage = B.Stage(pools=[pool], layer_window=[window], num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D,
+                    max_batch=Bn, max_pages_per_seq=tab.shape[1])
+    mod = B.AfdModule(stage, 0, to_dev_bf16(w_qkv_bits), to_dev_bf16(w_o_bits), THETA)
+    ref_pool = pool_np.copy()                      # the oracle's own pool, end to end
+    worst = {}
+    for step in range(steps):
+        nb = Bn if batches is None else batches[step]
+        pos = (lens[:nb] + step).astype(np.int32)
+        for i in inactive:
+            if i < nb:
+                pos[i] = -1
+        x_bits = oracle.f32_to_bf16_bits(rng.standard_normal((nb, hidden)).astype(np.float32))
+        x = oracle.bf16_bits_to_f64(x_bits)
+        d_x, d_pos = to_dev_bf16(x_bits), torch.from_numpy(pos).cuda()
+        y = torch.full((nb, hidden), float("nan"), dtype=torch.bfloat16, device="cuda")
+        before = tobits(pool).copy()
+        mod.step(d_x, d_pos, d_tab[:nb].contiguous(), y)
+        torch.cuda.synchronize()
+        assert stage.poll_error() == B.OPW_OK
+        gq, gk, gv, gattn = mod.intermediates(nb)
+        act = pos >= 0
+
+        # q, k, v against the oracle's projections
+        rq, rk, rv = afd.project_qkv(x, w_qkv, pos, Hq, Hkv, D, THETA)
+        for name, got, ref in (("q", f64(gq), rq), ("k", f64(gk), rk)):
+            partner = np.concatenate([ref[..., D // 2:], ref[..., :D // 2]], axis=-1)
+            err = np.abs(got - ref)[act]
+            assert (err <= 2.5 * 2.0 ** -7 * (np.abs(ref) + np.abs(partner))[act] + 1e-6).all(), (name, err.max())
+            worst[name] = max(worst.get(name, 0.0), float(err.max()))
+        assert (np.abs(f64(gv) - rv)[act] <= 2.0 ** -7 * np.abs(rv)[act] + 1e-6).all()
+
+        # append: exactly the GPU's k, v rows, nothing else changed
+        expect = before.copy()
+        assert oracle.kv_append(expect, Hkv, D, P, tobits(gk), tobits(gv), pos, tab[:nb]) == 0
+        after = tobits(pool)
+        assert (after == expect).all()
+
+        # attention on the GPU's q and that pool
+        kv_lens = np.where(act, pos + 1, 0).astype(np.int32)
+        ref_attn, _, rc = oracle.decode_attention(expect, Hq, Hkv, D, P, tobits(gq), kv_lens, tab[:nb], window=window)
+        assert rc == 0
+        err = np.abs(f64(gattn) - ref_attn)
+        assert err.max() <= 1e-2 and err.mean() <= 1e-3, (err.max(), err.mean())
+        assert (f64(gattn)[~act] == 0).all()
+
+        # output projection of the GPU's attention output
+        got_y = f64(y)
+        assert np.isfinite(got_y).all()
+        ref_y = f64(gattn).reshape(nb, Hq * D) @ w_o.T
+        rms = float(np.sqrt(np.mean(ref_y[act] ** 2)))
+        assert (np.abs(got_y - ref_y) <= 2.0 ** -8 * np.abs(ref_y) + 2.0 ** -10 * rms).all(), np.abs(got_y - ref_y).max()
+        assert (got_y[~act] == 0).all()
+
+        # end to end against the oracle's own module step on its own pool
+        e2e_y, _, _, _ = afd.module_step(ref_pool, x, w_qkv, w_o, pos, tab[:nb], Hq, Hkv, D, THETA, window=window)
+        err = np.abs(got_y - e2e_y)
+        rms = float(np.sqrt(np.mean(e2e_y[act] ** 2)))
+        assert (err <= 2.0 ** -5 * rms + 2.0 ** -8 * np.abs(e2e_y)).all(), (err.max(), rms)
+        assert err[act].mean() <= 2.0 ** -7 * rms, (err[act].mean(), rms)
+        worst["y_rel"] = max(worst.get("y_rel", 0.0), float(err.max() / rms))
+    mod.close()
+    stage.close()
+    return worst
+
+
+@pytest.mark.parametrize("Hq,Hkv,D,hidden", [(8, 2, 64, 256), (16, 2, 128, 512), (8, 2, 256, 384)])
+def test_module_matches_the_oracle_stage_by_stage_and_end_to_end(Hq, Hkv, D, hidden):
+    run_module(11 + D, [1, 15, 16, 700, 3000], Hq, Hkv, D, hidden, steps=2, inactive=(2,))
+
+
+def test_module_on_a_sliding_window_layer():
+    run_module(5, [30, 100, 2000], 8, 2, 64, 256, steps=2, window=64)
+
+
+def test_llama8b_layer_shape_and_a_batch_that_changes_between_steps():
+    run_module(21, [17, 900, 33, 2047, 512, 64, 5, 1200], 32, 8, 128, 4096, steps=3, batches=[8, 3, 8])
+
+
+def test_create_and_step_validate_arguments():
+    pool = torch.zeros(4 * 2 * 2 * P * 64, dtype=torch.bfloat16, device="cuda")
+    stage = B.Stage(pools=[pool], layer_window=[0], num_q_heads=8, num_kv_heads=2, head_dim=64, max_batch=2,
+                    max_pages_per_seq=2)
+    assert B.opw_attn_stage_shape(stage.handle) == dict(device=0, num_layers=1, num_q_heads=8, num_kv_heads=2,
+                                                        head_dim=64, max_batch=2)
+    w_qkv = torch.zeros(12 * 64, 256, dtype=torch.bfloat16, device="cuda")
+    w_o = torch.zeros(256, 8 * 64, dtype=torch.bfloat16, device="cuda")
+    nbytes = B.opw_afd_module_workspace_bytes(8, 2, 64, 2)
+    assert nbytes > 32 << 20 and B.opw_afd_module_workspace_bytes(8, 3, 64, 2) == 0
+    ws = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
+    base = (ws.data_ptr() + 255) // 256 * 256
+    for kw, status in ((dict(layer=1), B.OPW_ERR_INVALID_ARG), (dict(hidden=12), B.OPW_ERR_INVALID_ARG),
+                       (dict(rope_theta=0.0), B.OPW_ERR_INVALID_ARG), (dict(workspace=base + 8), B.OPW_ERR_INVALID_ARG),
+                       (dict(workspace_bytes=nbytes - 1), B.OPW_ERR_CAPACITY)):
+        args = dict(stage=stage.handle, layer=0, hidden=256, w_qkv=w_qkv.data_ptr(), w_o=w_o.data_ptr(),
+                    rope_theta=1e4, workspace=base, workspace_bytes=nbytes)
+        args.update(kw)
+        with pytest.raises(B.OpwError) as e:
+            B.opw_afd_module_create(**args)
+        assert e.value.status == status
+    mod = B.AfdModule(stage, 0, w_qkv, w_o)
+    x = torch.zeros(3, 256, dtype=torch.bfloat16, device="cuda")
+    pos = torch.zeros(3, dtype=torch.int32, device="cuda")
+    tab = torch.zeros(3, 2, dtype=torch.int32, device="cuda")
+    with pytest.raises(B.OpwError) as e:
+        mod.step(x, pos, tab, x.clone())
+    assert e.value.status == B.OPW_ERR_CAPACITY
+    mod.close()
+    B.opw_afd_module_destroy(None)
+    stage.close()
