@@ -8,7 +8,9 @@ one-ulp rounding flip upstream is not counted again downstream, and once end to 
               pair (x0, x1) moves the rotated value by <= 2^-7 (|x0| + |x1|) <= 2^-7 sqrt(2) (|ref| +
               |partner|), partner being the other element of the rotated pair, and the second flip adds
               2^-7 |ref|: |err| <= 2.5 * 2^-7 * (|ref| + |partner|).
-              v is not rotated: |err| <= 2^-7 |ref| (one flip)
+              v is not rotated: |err| <= 2^-7 |ref| (one flip).
+              Near zero the fp32 accumulation itself shows: tensor-core accumulators may truncate, so
+              its error can grow linearly, hidden * 2^-24 * rms -- added to all three bounds.
   append    : the pool afterwards holds the GPU's k, v rows bit for bit
   attention : the stated core-attention tolerance, oracle run on the GPU's q and that pool
   y         : a K-term fp32 dot product rounded to bf16: |err| <= 2^-8 |ref| + 2^-10 * rms(y)
@@ -83,12 +85,14 @@ def run_module(seed, lens, Hq, Hkv, D, hidden, steps=2, inactive=(), window=0, b
 
         # q, k, v against the oracle's projections
         rq, rk, rv = afd.project_qkv(x, w_qkv, pos, Hq, Hkv, D, THETA)
+        acc = hidden * 2.0 ** -24 * float(np.sqrt(np.mean(rv[act] ** 2))) + 1e-6
         for name, got, ref in (("q", f64(gq), rq), ("k", f64(gk), rk)):
             partner = np.concatenate([ref[..., D // 2:], ref[..., :D // 2]], axis=-1)
             err = np.abs(got - ref)[act]
-            assert (err <= 2.5 * 2.0 ** -7 * (np.abs(ref) + np.abs(partner))[act] + 1e-6).all(), (name, err.max())
+            assert (err <= 2.5 * 2.0 ** -7 * (np.abs(ref) + np.abs(partner))[act] + 2 * acc).all(), (name, err.max())
             worst[name] = max(worst.get(name, 0.0), float(err.max()))
-        assert (np.abs(f64(gv) - rv)[act] <= 2.0 ** -7 * np.abs(rv)[act] + 1e-6).all()
+        verr = np.abs(f64(gv) - rv)[act]
+        assert (verr <= 2.0 ** -7 * np.abs(rv)[act] + acc).all(), float((verr - 2.0 ** -7 * np.abs(rv)[act]).max())
 
         # append: exactly the GPU's k, v rows, nothing else changed
         expect = before.copy()
