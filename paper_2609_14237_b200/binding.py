@@ -17,7 +17,7 @@ _ROOT = os.path.dirname(_HERE)
 LIB_PATH = os.path.join(_HERE, "libopw_attn.so")
 SOURCES = [os.path.join(_HERE, "csrc", "opw_attn.cu"), os.path.join(_HERE, "csrc", "opw_noalloc.cu"),
            os.path.join(_HERE, "csrc", "opw_linear_attn.cu"), os.path.join(_HERE, "csrc", "opw_afd.cu")]
-HEADERS = [os.path.join(_HERE, "csrc", "opw_kernels.cuh"), os.path.join(_ROOT, "include", "opw_attn.h"),
+HEADERS = [os.path.join(_HERE, "csrc", "opw_kernels.cuh"), os.path.join(_HERE, "csrc", "opw_afd_gemm.cuh"), os.path.join(_ROOT, "include", "opw_attn.h"),
            os.path.join(_ROOT, "include", "opw_linear_attn.h"), os.path.join(_ROOT, "include", "opw_afd.h")]
 
 OPW_FLAG_PDL = 1
@@ -31,7 +31,8 @@ EXPORTS = [
     "opw_decode_step", "opw_attn_stage_host_layout", "opw_attn_stage_probe_timeout",
     "opw_linear_attn_decode_step", "opw_linear_attn_state_bytes", "opw_attn_plan_create_mixed",
     "opw_attn_stage_shape", "opw_afd_module_workspace_bytes", "opw_afd_module_create", "opw_afd_module_step",
-    "opw_afd_module_intermediates", "opw_afd_module_destroy",
+    "opw_afd_module_intermediates", "opw_afd_module_destroy", "opw_afd_module_poll_error",
+    "opw_afd_module_launch_count", "opw_afd_module_set_trace",
 ]
 
 
@@ -91,6 +92,7 @@ class PlanOp(ctypes.Structure):
 
 OPW_OP_ATTENTION, OPW_OP_LINEAR = 0, 1
 OPW_PLAN_GRAPH, OPW_PLAN_ADVANCE, OPW_PLAN_OVERLAP = 1, 2, 4
+OPW_AFD_LIBRARY_GEMM = 1
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
@@ -172,9 +174,16 @@ def lib() -> ctypes.CDLL:
     L.opw_attn_stage_shape.restype = ctypes.c_int
     L.opw_attn_stage_shape.argtypes = [vp] + [ctypes.POINTER(i32)] * 6
     L.opw_afd_module_workspace_bytes.restype = ctypes.c_size_t
-    L.opw_afd_module_workspace_bytes.argtypes = [i32, i32, i32, i32]
+    L.opw_afd_module_workspace_bytes.argtypes = [i32, i32, i32, i32, i32]
     L.opw_afd_module_create.restype = ctypes.c_int
-    L.opw_afd_module_create.argtypes = [vp, i32, i32, vp, vp, ctypes.c_float, vp, ctypes.c_size_t, ctypes.POINTER(vp)]
+    L.opw_afd_module_create.argtypes = [vp, i32, i32, vp, vp, ctypes.c_float, ctypes.c_uint32, vp, ctypes.c_size_t,
+                                        ctypes.POINTER(vp)]
+    L.opw_afd_module_poll_error.restype = ctypes.c_int
+    L.opw_afd_module_poll_error.argtypes = [vp, vp]
+    L.opw_afd_module_set_trace.restype = ctypes.c_int
+    L.opw_afd_module_set_trace.argtypes = [vp, vp, ctypes.c_size_t]
+    L.opw_afd_module_launch_count.restype = i64
+    L.opw_afd_module_launch_count.argtypes = [vp]
     L.opw_afd_module_step.restype = ctypes.c_int
     L.opw_afd_module_step.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     L.opw_afd_module_intermediates.restype = ctypes.c_int
@@ -380,16 +389,29 @@ def opw_attn_stage_shape(stage: int) -> dict:
     return {n: int(v.value) for n, v in zip(names, vals)}
 
 
-def opw_afd_module_workspace_bytes(num_q_heads: int, num_kv_heads: int, head_dim: int, max_batch: int) -> int:
-    return int(lib().opw_afd_module_workspace_bytes(num_q_heads, num_kv_heads, head_dim, max_batch))
+def opw_afd_module_workspace_bytes(num_q_heads: int, num_kv_heads: int, head_dim: int, max_batch: int,
+                                   hidden: int) -> int:
+    return int(lib().opw_afd_module_workspace_bytes(num_q_heads, num_kv_heads, head_dim, max_batch, hidden))
 
 
 def opw_afd_module_create(stage: int, layer: int, hidden: int, w_qkv: int, w_o: int, rope_theta: float,
-                          workspace: int, workspace_bytes: int) -> int:
+                          workspace: int, workspace_bytes: int, flags: int = 0) -> int:
     h = ctypes.c_void_p()
-    _check(lib().opw_afd_module_create(stage, layer, hidden, w_qkv, w_o, rope_theta, workspace, workspace_bytes,
-                                       ctypes.byref(h)), "opw_afd_module_create")
+    _check(lib().opw_afd_module_create(stage, layer, hidden, w_qkv, w_o, rope_theta, flags, workspace,
+                                       workspace_bytes, ctypes.byref(h)), "opw_afd_module_create")
     return h.value
+
+
+def opw_afd_module_poll_error(module: int, stream: Optional[int] = None) -> int:
+    return int(lib().opw_afd_module_poll_error(module, stream))
+
+
+def opw_afd_module_set_trace(module: int, trace: Optional[int], trace_bytes: int = 0) -> None:
+    _check(lib().opw_afd_module_set_trace(module, trace, trace_bytes), "opw_afd_module_set_trace")
+
+
+def opw_afd_module_launch_count(module: int) -> int:
+    return int(lib().opw_afd_module_launch_count(module))
 
 
 def opw_afd_module_step(module: int, batch: int, x: int, positions: int, page_table: int, y: int,
@@ -518,7 +540,7 @@ class AfdModule:
     """Owner of one complete-attention-module handle (projections + rotary encoding + the stage's
     core attention) over torch tensors; forwards to the opw_afd_module_* entry points."""
 
-    def __init__(self, stage: Stage, layer: int, w_qkv, w_o, rope_theta: float = 10000.0):
+    def __init__(self, stage: Stage, layer: int, w_qkv, w_o, rope_theta: float = 10000.0, flags: int = 0):
         import torch
 
         shp = opw_attn_stage_shape(stage.handle)
@@ -529,12 +551,28 @@ class AfdModule:
             raise ValueError("weight shapes do not match the stage")
         if w_qkv.dtype != torch.bfloat16 or w_o.dtype != torch.bfloat16 or not (w_qkv.is_contiguous() and w_o.is_contiguous()):
             raise ValueError("weights must be contiguous bf16")
-        nbytes = opw_afd_module_workspace_bytes(shp["num_q_heads"], shp["num_kv_heads"], shp["head_dim"], shp["max_batch"])
+        nbytes = opw_afd_module_workspace_bytes(shp["num_q_heads"], shp["num_kv_heads"], shp["head_dim"], shp["max_batch"],
+                                                self.hidden)
         self.workspace = torch.empty(nbytes + 256, dtype=torch.uint8, device=stage.device)
         base = (self.workspace.data_ptr() + 255) // 256 * 256
         self.shape = shp
         self.handle = opw_afd_module_create(stage.handle, layer, self.hidden, w_qkv.data_ptr(), w_o.data_ptr(),
-                                            rope_theta, base, nbytes)
+                                            rope_theta, base, nbytes, flags)
+
+    def poll_error(self) -> int:
+        return opw_afd_module_poll_error(self.handle, Stage._stream())
+
+    def launch_count(self) -> int:
+        return opw_afd_module_launch_count(self.handle)
+
+    def enable_trace(self):
+        """Allocate the trace buffer and switch tracing on; returns the int64 tensor [2, 1024, 8]
+        (region 0: output projection, region 1: QKV projection)."""
+        import torch
+
+        self.trace = torch.zeros(2, 1024, 8, dtype=torch.int64, device=self.stage.device)
+        opw_afd_module_set_trace(self.handle, self.trace.data_ptr(), self.trace.numel() * 8)
+        return self.trace
 
     def step(self, x, positions, page_table, y):
         opw_afd_module_step(self.handle, positions.shape[0], x.data_ptr(), positions.data_ptr(), page_table.data_ptr(),

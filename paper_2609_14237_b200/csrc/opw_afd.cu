@@ -1,7 +1,10 @@
-// The complete attention module as one stage (AFD partition): QKV projection (cuBLASLt),
-// rotary encoding fused with the split into q / k_new / v_new (own kernel), core attention
-// (opw_decode_step), output projection (cuBLASLt).  See include/opw_afd.h.
+// The complete attention module as one stage (AFD partition): QKV projection with the rotary
+// encoding and the split into q / k_new / v_new in its epilogue, core attention
+// (opw_decode_step), output projection.  The projections run on the tcgen05 kernel of
+// opw_afd_gemm.cuh; cuBLASLt plus a separate rotary kernel is the alternative path
+// (OPW_AFD_LIBRARY_GEMM, and head_dim 256).  See include/opw_afd.h.
 #include "opw_afd.h"
+#include "opw_afd_gemm.cuh"
 
 #include <cmath>
 #include <cstdint>
@@ -100,6 +103,10 @@ bool run_plan(cublasLtHandle_t lt, const GemmPlan& p, const void* w, const void*
 
 }  // namespace
 
+typedef CUresult (*TensorMapEncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                      const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                      CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
 struct opw_afd_module {
   opw_attn_stage_t* stage;
   int32_t layer, hidden, Hq, Hkv, D, max_batch;
@@ -107,50 +114,137 @@ struct opw_afd_module {
   const void* w_o;
   double log_theta;
   unsigned char* ws;
-  size_t off_qkv, off_q, off_k, off_v, off_out, off_gemm;
+  size_t off_qkv, off_q, off_k, off_v, off_out, off_gemm, off_partials, off_tickets, off_status;
+  // tensor-core path
+  bool tc_qkv, tc_o;
+  int sms;
+  TensorMapEncodeFn encode;
+  CUtensorMap map_wqkv, map_wo;
+  int64_t launches;
+  unsigned long long* trace;
+  // library path: plans are keyed by the batch size; decode loops repeat a handful of sizes, so the
+  // last one of each projection is kept and rebuilt when the batch changes.
   cublasLtHandle_t lt;
-  // Plans are keyed by the batch size; decode loops repeat a handful of sizes, so the last one
-  // of each projection is kept and rebuilt when the batch changes.
   int32_t plan_batch;
   GemmPlan plan_qkv, plan_o;
 };
 
 namespace {
 
-struct Carve { size_t qkv, q, k, v, out, gemm, total; };
+constexpr int kSmsBound = 160;             // split-K sizing assumes no more SMs than this
+// Above this batch the skinny kernel stops paying: every CTA streams the whole activation matrix
+// beside its 128 weight rows, so at 256 rows two thirds of its traffic is activations re-read from
+// L2 by every CTA, and a square-tiled library GEMM wins (measured: ahead up to 32 rows, level at
+// 64 and 96, behind at 128).
+constexpr int kTcMaxBatch = 96;
+constexpr size_t kGemmSmemBudget = 226 * 1024;
 
-Carve carve(int Hq, int Hkv, int D, int max_batch) {
+inline int round16(int x) { return (x + 15) / 16 * 16; }
+inline int tiles_of(int n_out) { return (n_out + opw_afd::kTileM - 1) / opw_afd::kTileM; }
+inline int ksplit_of(int n_out, int k, int sms) {
+  int ks = sms / tiles_of(n_out);
+  if (ks > opw_afd::kMaxSplit) ks = opw_afd::kMaxSplit;
+  const int kblocks = (k + opw_afd::kBlockK - 1) / opw_afd::kBlockK;
+  if (ks > kblocks) ks = kblocks;
+  return ks < 1 ? 1 : ks;
+}
+inline size_t partial_bytes(int n_out, int k, int nb) {
+  return (size_t)tiles_of(n_out) * ksplit_of(n_out, k, kSmsBound) * nb * opw_afd::kTileM * sizeof(float);
+}
+
+struct Carve { size_t qkv, q, k, v, out, gemm, partials, tickets, status, total; };
+
+Carve carve(int Hq, int Hkv, int D, int max_batch, int hidden) {
   Carve c;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
-  c.qkv = take((size_t)max_batch * (Hq + 2 * Hkv) * D * 2);
-  c.q = take((size_t)max_batch * Hq * D * 2);
+  const int n_qkv = (Hq + 2 * Hkv) * D, n_attn = Hq * D;
+  const int nb = max_batch < 256 ? round16(max_batch) : 256;
+  c.qkv = take((size_t)max_batch * n_qkv * 2);
+  c.q = take((size_t)max_batch * n_attn * 2);
   c.k = take((size_t)max_batch * Hkv * D * 2);
   c.v = take((size_t)max_batch * Hkv * D * 2);
-  c.out = take((size_t)max_batch * Hq * D * 2);
+  c.out = take((size_t)max_batch * n_attn * 2);
   c.gemm = take(kGemmWorkspace);
+  const size_t p1 = partial_bytes(n_qkv, hidden, nb), p2 = partial_bytes(hidden, n_attn, nb);
+  c.partials = take(p1 > p2 ? p1 : p2);
+  const int t1 = tiles_of(n_qkv), t2 = tiles_of(hidden);
+  c.tickets = take((size_t)(t1 > t2 ? t1 : t2) * sizeof(uint32_t));
+  c.status = take(sizeof(uint32_t));
   c.total = off;
   return c;
 }
 
-bool dims_ok(int Hq, int Hkv, int D, int max_batch) {
-  return Hq >= 1 && Hkv >= 1 && Hq % Hkv == 0 && (D == 64 || D == 128 || D == 256) && max_batch >= 1;
+bool dims_ok(int Hq, int Hkv, int D, int max_batch, int hidden) {
+  return Hq >= 1 && Hkv >= 1 && Hq % Hkv == 0 && (D == 64 || D == 128 || D == 256) && max_batch >= 1 && hidden >= 8 &&
+         hidden % 8 == 0;
+}
+
+// Row-major bf16 [rows, k] seen by TMA as a 2-D tensor, boxes of 64 x box_rows elements, 128-byte swizzle,
+// zero fill outside the tensor (so ragged rows and a ragged K tail contribute nothing).
+bool encode_map(TensorMapEncodeFn fn, CUtensorMap* map, const void* base, uint64_t rows, uint64_t k, uint32_t box_rows) {
+  const cuuint64_t dims[2] = {k, rows};
+  const cuuint64_t strides[1] = {k * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)opw_afd::kBlockK, box_rows};
+  const cuuint32_t elem[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, elem,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// One projection on the tensor-core kernel; batches beyond 256 rows go in blocks of 256.
+opw_status_t run_tc_gemm(opw_afd_module* m, const CUtensorMap& map_w, const void* x, int batch, int n_out, int k, int mode,
+                         const int32_t* positions, __nv_bfloat16* out, __nv_bfloat16* q, __nv_bfloat16* kn, __nv_bfloat16* vn, cudaStream_t stream) {
+  for (int b0 = 0; b0 < batch; b0 += 256) {
+    const int nbatch = batch - b0 < 256 ? batch - b0 : 256;
+    opw_afd::GemmParams p;
+    p.n_out = n_out; p.k = k; p.batch = nbatch; p.nb = round16(nbatch);
+    const size_t stage_bytes = opw_afd::kTileABytes + (size_t)p.nb * 128;
+    // mode 1 keeps the step's angle table behind the ring: (cos, sin) per row and pair, then D/2 doubles
+    const size_t angle_bytes = mode == 1 ? (size_t)nbatch * (m->D / 2) * sizeof(float2) + (size_t)(m->D / 2) * sizeof(double) : 0;
+    int stages = (int)((kGemmSmemBudget - 1024 - angle_bytes) / stage_bytes);
+    if (stages > opw_afd::kMaxStages) stages = opw_afd::kMaxStages;
+    p.stages = stages;
+    p.ksplit = ksplit_of(n_out, k, m->sms < kSmsBound ? m->sms : kSmsBound);
+    p.mode = mode;
+    p.out = out ? out + (size_t)b0 * n_out : nullptr;
+    p.q = q ? q + (size_t)b0 * m->Hq * m->D : nullptr;
+    p.kn = kn ? kn + (size_t)b0 * m->Hkv * m->D : nullptr;
+    p.vn = vn ? vn + (size_t)b0 * m->Hkv * m->D : nullptr;
+    p.positions = positions ? positions + b0 : nullptr;
+    p.log_theta = m->log_theta;
+    p.Hq = m->Hq; p.Hkv = m->Hkv; p.D = m->D;
+    p.partials = reinterpret_cast<float*>(m->ws + m->off_partials);
+    p.tickets = reinterpret_cast<uint32_t*>(m->ws + m->off_tickets);
+    p.status = reinterpret_cast<uint32_t*>(m->ws + m->off_status);
+    // region 0: output projection, region 1: QKV projection (the last column block of a step stays)
+    p.trace = m->trace ? m->trace + (size_t)mode * opw_afd::kTraceMaxCtas * opw_afd::kTraceWords : nullptr;
+    CUtensorMap map_x;
+    const unsigned char* xb = static_cast<const unsigned char*>(x) + (size_t)b0 * k * 2;
+    if (!encode_map(m->encode, &map_x, xb, (uint64_t)nbatch, (uint64_t)k, (uint32_t)p.nb)) return OPW_ERR_CUDA;
+    const size_t smem = 1024 + (size_t)stages * stage_bytes + angle_bytes;
+    const dim3 grid(tiles_of(n_out), p.ksplit);
+    opw_afd::skinny_gemm_kernel<<<grid, opw_afd::kGemmThreads, smem, stream>>>(map_w, map_x, p);
+    if (cudaGetLastError() != cudaSuccess) return OPW_ERR_CUDA;
+    ++m->launches;
+  }
+  return OPW_OK;
 }
 
 }  // namespace
 
 extern "C" {
 
-size_t opw_afd_module_workspace_bytes(int32_t Hq, int32_t Hkv, int32_t D, int32_t max_batch) {
-  if (!dims_ok(Hq, Hkv, D, max_batch)) return 0;
-  return carve(Hq, Hkv, D, max_batch).total;
+size_t opw_afd_module_workspace_bytes(int32_t Hq, int32_t Hkv, int32_t D, int32_t max_batch, int32_t hidden) {
+  if (!dims_ok(Hq, Hkv, D, max_batch, hidden)) return 0;
+  return carve(Hq, Hkv, D, max_batch, hidden).total;
 }
 
 opw_status_t opw_afd_module_create(opw_attn_stage_t* stage, int32_t layer, int32_t hidden, const void* w_qkv,
-                                   const void* w_o, float rope_theta, void* workspace, size_t workspace_bytes,
-                                   opw_afd_module_t** out) {
+                                   const void* w_o, float rope_theta, uint32_t flags, void* workspace,
+                                   size_t workspace_bytes, opw_afd_module_t** out) {
   if (!stage || !w_qkv || !w_o || !workspace || !out) return OPW_ERR_INVALID_ARG;
-  if (hidden < 8 || hidden % 8 != 0 || !(rope_theta > 0.f)) return OPW_ERR_INVALID_ARG;
+  if (hidden < 8 || hidden % 8 != 0 || !(rope_theta > 0.f) || (flags & ~OPW_AFD_LIBRARY_GEMM)) return OPW_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255) || (reinterpret_cast<uintptr_t>(w_qkv) & 15) ||
       (reinterpret_cast<uintptr_t>(w_o) & 15))
     return OPW_ERR_INVALID_ARG;
@@ -158,7 +252,7 @@ opw_status_t opw_afd_module_create(opw_attn_stage_t* stage, int32_t layer, int32
   opw_status_t rc = opw_attn_stage_shape(stage, &device, &layers, &Hq, &Hkv, &D, &max_batch);
   if (rc != OPW_OK) return rc;
   if (layer < 0 || layer >= layers) return OPW_ERR_INVALID_ARG;
-  const Carve c = carve(Hq, Hkv, D, max_batch);
+  const Carve c = carve(Hq, Hkv, D, max_batch, hidden);
   if (workspace_bytes < c.total) return OPW_ERR_CAPACITY;
   if (cudaSetDevice(device) != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
   opw_afd_module* m = new (std::nothrow) opw_afd_module();
@@ -169,8 +263,40 @@ opw_status_t opw_afd_module_create(opw_attn_stage_t* stage, int32_t layer, int32
   m->log_theta = std::log((double)rope_theta);
   m->ws = static_cast<unsigned char*>(workspace);
   m->off_qkv = c.qkv; m->off_q = c.q; m->off_k = c.k; m->off_v = c.v; m->off_out = c.out; m->off_gemm = c.gemm;
+  m->off_partials = c.partials; m->off_tickets = c.tickets; m->off_status = c.status;
   m->plan_batch = 0;
-  if (cublasLtCreate(&m->lt) != CUBLAS_STATUS_SUCCESS) { delete m; return OPW_ERR_CUDA; }
+  m->launches = 0;
+  m->trace = nullptr;
+  m->lt = nullptr;
+  m->encode = nullptr;
+  const bool library = (flags & OPW_AFD_LIBRARY_GEMM) != 0;
+  m->tc_qkv = !library && D <= 128;         // the rotary epilogue needs a rotated pair inside one 128-row tile
+  m->tc_o = !library;
+  bool ok = true;
+  if (m->tc_qkv || m->tc_o) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    ok = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+         qres == cudaDriverEntryPointSuccess && fn != nullptr;
+    m->encode = reinterpret_cast<TensorMapEncodeFn>(fn);
+    int sms = 0;
+    ok = ok && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) == cudaSuccess && sms > 0;
+    m->sms = sms;
+    ok = ok && cudaFuncSetAttribute(opw_afd::skinny_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    (int)kGemmSmemBudget) == cudaSuccess;
+    const int n_qkv = (Hq + 2 * Hkv) * D, n_attn = Hq * D;
+    ok = ok && encode_map(m->encode, &m->map_wqkv, w_qkv, (uint64_t)n_qkv, (uint64_t)hidden, opw_afd::kTileM);
+    ok = ok && encode_map(m->encode, &m->map_wo, w_o, (uint64_t)hidden, (uint64_t)n_attn, opw_afd::kTileM);
+  }
+  // tickets and the status word start at zero (synchronously, on the default stream, as the stage does)
+  ok = ok && cudaMemset(m->ws + c.tickets, 0, c.total - c.tickets) == cudaSuccess;
+  if (ok) ok = cublasLtCreate(&m->lt) == CUBLAS_STATUS_SUCCESS;   // also serves batches beyond kTcMaxBatch
+  if (!ok) {
+    (void)cudaGetLastError();
+    if (m->lt) cublasLtDestroy(m->lt);
+    delete m;
+    return OPW_ERR_CUDA;
+  }
   *out = m;
   return OPW_OK;
 }
@@ -178,14 +304,15 @@ opw_status_t opw_afd_module_create(opw_attn_stage_t* stage, int32_t layer, int32
 opw_status_t opw_afd_module_step(opw_afd_module_t* m, int32_t batch, const void* x, const int32_t* positions,
                                  const int32_t* page_table, void* y, void* cuda_stream) {
   if (!m || !x || !positions || !page_table || !y) return OPW_ERR_INVALID_ARG;
-  if (batch < 1) return OPW_ERR_INVALID_ARG;
+  if (batch < 1 || (reinterpret_cast<uintptr_t>(x) & 15) || (reinterpret_cast<uintptr_t>(y) & 15)) return OPW_ERR_INVALID_ARG;
   if (batch > m->max_batch) return OPW_ERR_CAPACITY;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const int n_qkv = (m->Hq + 2 * m->Hkv) * m->D, n_attn = m->Hq * m->D;
-  if (m->plan_batch != batch) {
+  const bool tc_qkv = m->tc_qkv && batch <= kTcMaxBatch, tc_o = m->tc_o && batch <= kTcMaxBatch;
+  if ((!tc_qkv || !tc_o) && m->plan_batch != batch) {
     m->plan_batch = 0;
-    if (!make_plan(m->lt, m->plan_qkv, batch, n_qkv, m->hidden)) return OPW_ERR_CUDA;
-    if (!make_plan(m->lt, m->plan_o, batch, m->hidden, n_attn)) return OPW_ERR_CUDA;
+    if (!tc_qkv && !make_plan(m->lt, m->plan_qkv, batch, n_qkv, m->hidden)) return OPW_ERR_CUDA;
+    if (!tc_o && !make_plan(m->lt, m->plan_o, batch, m->hidden, n_attn)) return OPW_ERR_CUDA;
     m->plan_batch = batch;
   }
   __nv_bfloat16* qkv = reinterpret_cast<__nv_bfloat16*>(m->ws + m->off_qkv);
@@ -194,14 +321,27 @@ opw_status_t opw_afd_module_step(opw_afd_module_t* m, int32_t batch, const void*
   __nv_bfloat16* v = reinterpret_cast<__nv_bfloat16*>(m->ws + m->off_v);
   __nv_bfloat16* attn = reinterpret_cast<__nv_bfloat16*>(m->ws + m->off_out);
   void* gemm_ws = m->ws + m->off_gemm;
+  opw_status_t rc;
 
-  if (!run_plan(m->lt, m->plan_qkv, m->w_qkv, x, qkv, gemm_ws, stream)) return OPW_ERR_CUDA;
-  rope_split_kernel<<<batch, 256, (size_t)m->D * sizeof(float), stream>>>(qkv, positions, q, k, v, m->Hq, m->Hkv, m->D,
-                                                                         m->log_theta);
-  if (cudaGetLastError() != cudaSuccess) return OPW_ERR_CUDA;
-  opw_status_t rc = opw_decode_step(m->stage, m->layer, batch, q, k, v, positions, page_table, attn, nullptr, cuda_stream);
+  if (tc_qkv) {
+    rc = run_tc_gemm(m, m->map_wqkv, x, batch, n_qkv, m->hidden, 1, positions, nullptr, q, k, v, stream);
+    if (rc != OPW_OK) return rc;
+  } else {
+    if (!run_plan(m->lt, m->plan_qkv, m->w_qkv, x, qkv, gemm_ws, stream)) return OPW_ERR_CUDA;
+    rope_split_kernel<<<batch, 256, (size_t)m->D * sizeof(float), stream>>>(qkv, positions, q, k, v, m->Hq, m->Hkv, m->D,
+                                                                           m->log_theta);
+    if (cudaGetLastError() != cudaSuccess) return OPW_ERR_CUDA;
+    ++m->launches;
+  }
+  rc = opw_decode_step(m->stage, m->layer, batch, q, k, v, positions, page_table, attn, nullptr, cuda_stream);
   if (rc != OPW_OK) return rc;
-  if (!run_plan(m->lt, m->plan_o, m->w_o, attn, y, gemm_ws, stream)) return OPW_ERR_CUDA;
+  if (tc_o) {
+    rc = run_tc_gemm(m, m->map_wo, attn, batch, m->hidden, n_attn, 0, nullptr, static_cast<__nv_bfloat16*>(y), nullptr,
+                     nullptr, nullptr, stream);
+    if (rc != OPW_OK) return rc;
+  } else if (!run_plan(m->lt, m->plan_o, m->w_o, attn, y, gemm_ws, stream)) {
+    return OPW_ERR_CUDA;
+  }
   return OPW_OK;
 }
 
@@ -214,11 +354,35 @@ opw_status_t opw_afd_module_intermediates(opw_afd_module_t* m, void** q, void** 
   return OPW_OK;
 }
 
+opw_status_t opw_afd_module_poll_error(opw_afd_module_t* m, void* cuda_stream) {
+  if (!m) return OPW_ERR_INVALID_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  uint32_t word = 0;
+  uint32_t* d = reinterpret_cast<uint32_t*>(m->ws + m->off_status);
+  if (cudaMemcpyAsync(&word, d, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaMemsetAsync(d, 0, 4, stream) != cudaSuccess || cudaStreamSynchronize(stream) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return OPW_ERR_CUDA;
+  }
+  return (word & opw_afd::kGemmErrTimeout) ? OPW_ERR_TIMEOUT : OPW_OK;
+}
+
+opw_status_t opw_afd_module_set_trace(opw_afd_module_t* m, void* trace, size_t trace_bytes) {
+  if (!m) return OPW_ERR_INVALID_ARG;
+  if (!trace) { m->trace = nullptr; return OPW_OK; }
+  if (reinterpret_cast<uintptr_t>(trace) & 7) return OPW_ERR_INVALID_ARG;
+  if (trace_bytes < (size_t)2 * opw_afd::kTraceMaxCtas * opw_afd::kTraceWords * 8) return OPW_ERR_CAPACITY;
+  m->trace = static_cast<unsigned long long*>(trace);
+  return OPW_OK;
+}
+
+int64_t opw_afd_module_launch_count(const opw_afd_module_t* m) { return m ? m->launches : 0; }
+
 opw_status_t opw_afd_module_destroy(opw_afd_module_t* m) {
   if (!m) return OPW_OK;
   destroy_plan(m->plan_qkv);
   destroy_plan(m->plan_o);
-  cublasLtDestroy(m->lt);
+  if (m->lt) cublasLtDestroy(m->lt);
   delete m;
   return OPW_OK;
 }

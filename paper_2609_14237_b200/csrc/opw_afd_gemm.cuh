@@ -1,0 +1,404 @@
+// Skinny projection GEMM of the decode step on the 5th-generation tensor cores (sm_100a).
+//
+//   C[b, n] = sum_k x[b, k] * W[n, k]          x: [batch <= 256, K] bf16, W: [N, K] bf16, fp32 accumulate
+//
+// A decode step has few rows (the batch) and a large weight matrix that is read once, so the
+// kernel is built around streaming W: the WEIGHT rows take the tensor core's M dimension (one
+// CTA = 128 weight rows = 128 TMEM lanes), the batch takes its N dimension (16..256 columns of
+// fp32 accumulators in TMEM), and K is cut into 64-element blocks (128 bytes = one swizzle row)
+// that TMA brings into a shared-memory ring.  One thread issues the copies, one thread issues
+// tcgen05.mma (4 per block, K = 16 each) and releases ring slots with tcgen05.commit, and after
+// the last block sixteen warps read the accumulators back with tcgen05.ld (four lane quadrants x
+// four column groups) -- the epilogue is a chain of L2 round trips, so it wants many threads.
+//
+// With N/128 tiles alone a 6144 x 4096 projection would occupy 48 of 148 SMs, too few to pull
+// the weights at HBM speed, so K is also split over `ksplit` CTAs per tile; each writes its fp32
+// partial tile to a workspace and the last to arrive (an atomic ticket per tile) adds them in
+// split order -- deterministic -- and runs the epilogue.
+//
+// Epilogues: plain (bf16 C[b, n]) and rotary (the QKV projection of the attention module: the
+// result is rounded to bf16 as a library GEMM would, pairs (d, d + D/2) of the q and k heads
+// are rotated by angles that the warps idle in the main loop compute meanwhile, v is passed
+// through, and the three outputs go to separate [batch, heads, D] buffers).  The rotary form needs both elements of a pair in one
+// 128-row tile: D in {64, 128}.
+//
+// Every wait is bounded by the global timer (kGemmWaitNs); a wait that runs out records
+// kGemmErrTimeout in the status word, the CTA skips its epilogue, frees its TMEM and exits.
+#pragma once
+
+#include <cstdint>
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+namespace opw_afd {
+
+constexpr int kTileM = 128;               // weight rows per CTA
+constexpr int kBlockK = 64;               // bf16 elements per k-block (128 bytes)
+constexpr int kGemmThreads = 512;        // 16 warps: 2 single-thread roles in the main loop, all of them in the epilogue
+constexpr int kColPhases = kGemmThreads / 64;   // epilogue: thread = 2 adjacent rows x every kColPhases-th batch column
+constexpr int kMaxStages = 12;
+constexpr int kMaxSplit = 4;
+constexpr uint32_t kTileABytes = kTileM * kBlockK * 2;
+constexpr uint64_t kGemmWaitNs = 200ull * 1000 * 1000;
+constexpr uint32_t kGemmErrTimeout = 2u;  // same bit as the attention kernels' timeout
+
+struct GemmParams {
+  int n_out, k, batch;
+  int nb;                 // MMA N: batch rounded up to a multiple of 16 (16..256)
+  int stages;
+  int ksplit;
+  int mode;               // 0: plain, 1: rotary + split into q / k / v
+  __nv_bfloat16* out;     // mode 0: [batch, n_out]
+  __nv_bfloat16* q;       // mode 1: [batch, Hq, D]
+  __nv_bfloat16* kn;      //         [batch, Hkv, D]
+  __nv_bfloat16* vn;      //         [batch, Hkv, D]
+  const int32_t* positions;  // mode 1: [batch]; the rotation angle of pair i is position * theta^(-2i/D)
+  double log_theta;
+  int Hq, Hkv, D;
+  float* partials;        // [tiles, ksplit, nb, 128] fp32, used when ksplit > 1
+  uint32_t* tickets;      // [tiles], zero between launches
+  uint32_t* status;
+  unsigned long long* trace;   // optional: [grid][8] global-timer stamps of each CTA's phases (see kTrace*)
+};
+
+// Trace record of one CTA: begin, ring and TMEM ready, accumulator complete, accumulator in shared
+// memory, partial tile published (ticket taken), partial tiles reduced, end; then the SM id.
+constexpr int kTraceWords = 8;
+constexpr int kTraceMaxCtas = 1024;
+__device__ __forceinline__ void g_stamp(const GemmParams& p, int cta, int slot) {
+  if (p.trace && cta < kTraceMaxCtas && threadIdx.x == 0) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    p.trace[(size_t)cta * kTraceWords + slot] = t;
+  }
+}
+
+// ---- PTX wrappers ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t g_smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void g_mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void g_mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ uint32_t g_mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+__device__ __forceinline__ bool g_mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+  if (g_mbar_try_wait(bar, parity)) return true;
+  uint64_t t0, t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
+  for (;;) {
+    for (int i = 0; i < 64; ++i)
+      if (g_mbar_try_wait(bar, parity)) return true;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    if (t - t0 > kGemmWaitNs) return false;
+  }
+}
+// 2-D tiled TMA load (no multicast): box of the tensor map at element coordinates (c0 = k, c1 = row).
+__device__ __forceinline__ void g_tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+               "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void g_tmem_alloc(uint32_t slot_smem, uint32_t ncols) {
+  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(ncols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void g_tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void g_tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void g_tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 in, fp32 out, M = 128, N from the instruction descriptor, K = 16.
+__device__ __forceinline__ void g_umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// Arrives on the mbarrier once every tcgen05.mma issued so far by this thread has finished.
+__device__ __forceinline__ void g_umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 16 consecutive fp32 columns of this thread's TMEM lane.
+__device__ __forceinline__ void g_tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr));
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes, stored as TMA's
+// 128-byte swizzle leaves them: 8-row groups 1024 bytes apart (stride byte offset), leading
+// byte offset unused (1), descriptor version 1, layout type 2 = 128-byte swizzle.  Addresses and
+// offsets are in 16-byte units.
+__device__ __forceinline__ uint64_t g_smem_desc(uint32_t smem_addr) {
+  return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor of kind::f16: fp32 accumulator (bits 4-5 = 1), A and B bf16 (bits 7-9
+// and 10-12 = 1), both K-major (bits 15, 16 = 0), N / 8 in bits 17-22, M / 16 in bits 24-28.
+__device__ __forceinline__ uint32_t g_instr_desc(int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
+}
+
+__device__ __forceinline__ float g_round_bf16(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
+
+// grid = (ceil(n_out / 128), ksplit), 512 threads, 1 CTA per SM.
+// Dynamic shared memory: 1024 (alignment slack) + stages * (16384 + nb * 128) bytes, then in mode 1
+// the angle table, batch * D/2 (cos, sin) pairs of 8 bytes.
+__global__ void __launch_bounds__(kGemmThreads, 1)
+skinny_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const GemmParams p) {
+  extern __shared__ unsigned char g_smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[kMaxStages];
+  __shared__ __align__(8) uint64_t empty_bar[kMaxStages];
+  __shared__ __align__(8) uint64_t acc_bar;
+  __shared__ uint32_t tmem_slot;
+  __shared__ volatile int s_fail;
+  __shared__ int s_last;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tile = blockIdx.x, split = blockIdx.y;
+  const uint32_t raw = g_smem_u32(g_smem_raw);
+  const uint32_t ring = (raw + 1023u) & ~1023u;             // swizzled tiles need 1024-byte alignment
+  float* stage_f = reinterpret_cast<float*>(g_smem_raw + (ring - raw));   // the ring again, after the last MMA: [nb][128] fp32
+  const uint32_t stage_bytes = kTileABytes + (uint32_t)p.nb * 128u;
+  float2* angles = reinterpret_cast<float2*>(g_smem_raw + (ring - raw) + (size_t)p.stages * stage_bytes);   // [batch][D/2]
+  const int kblocks = (p.k + kBlockK - 1) / kBlockK;
+  const int kb0 = (int)((int64_t)kblocks * split / p.ksplit);
+  const int kb1 = (int)((int64_t)kblocks * (split + 1) / p.ksplit);
+  const int nkb = kb1 - kb0;
+  uint32_t ncols = 32;
+  while (ncols < (uint32_t)p.nb) ncols <<= 1;
+  const int cta = blockIdx.y * gridDim.x + blockIdx.x;
+  g_stamp(p, cta, 0);
+  if (p.trace && cta < kTraceMaxCtas && tid == 0) {
+    uint32_t sm;
+    asm volatile("mov.u32 %0, %smid;" : "=r"(sm));
+    p.trace[(size_t)cta * kTraceWords + 7] = sm;
+  }
+
+  auto issue = [&](int i) {                                  // both tiles of k-block i into slot i % stages
+    const int s = i % p.stages;
+    const uint32_t fb = g_smem_u32(&full_bar[s]);
+    const uint32_t a = ring + (uint32_t)s * stage_bytes;
+    g_mbar_expect_tx(fb, stage_bytes);
+    g_tma_load_2d(a, &map_w, (kb0 + i) * kBlockK, tile * kTileM, fb);
+    g_tma_load_2d(a + kTileABytes, &map_x, (kb0 + i) * kBlockK, 0, fb);
+  };
+
+  if (tid == 0) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_w)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&map_x)) : "memory");
+    for (int s = 0; s < p.stages; ++s) {
+      g_mbar_init(g_smem_u32(&full_bar[s]), 1);
+      g_mbar_init(g_smem_u32(&empty_bar[s]), 1);
+    }
+    g_mbar_init(g_smem_u32(&acc_bar), 1);
+    s_fail = 0;
+    s_last = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    // the first round of the ring needs no free-slot wait: start the stream before the TMEM allocation
+    for (int i = 0; i < nkb && i < p.stages; ++i) issue(i);
+  }
+  if (warp == 1) g_tmem_alloc(g_smem_u32(&tmem_slot), ncols);
+  g_tc_fence_before();
+  __syncthreads();
+  g_tc_fence_after();
+  const uint32_t tmem_d = tmem_slot;
+  g_stamp(p, cta, 1);
+
+  if (tid == 0) {
+    // ---- producer: one TMA load of the weight tile and one of the activation tile per k-block ----
+    for (int i = p.stages; i < nkb; ++i) {
+      if (!g_mbar_wait_bounded(g_smem_u32(&empty_bar[i % p.stages]), (uint32_t)((i / p.stages) - 1) & 1u)) {
+        s_fail = 1;
+        atomicOr(p.status, kGemmErrTimeout);
+        break;
+      }
+      issue(i);
+    }
+  } else if (tid == 32) {
+    // ---- MMA issuer ----
+    const uint32_t idesc = g_instr_desc(p.nb);
+    bool ok = true;
+    for (int i = 0; i < nkb; ++i) {
+      const int s = i % p.stages;
+      if (!g_mbar_wait_bounded(g_smem_u32(&full_bar[s]), (uint32_t)(i / p.stages) & 1u)) {
+        s_fail = 1;
+        atomicOr(p.status, kGemmErrTimeout);
+        ok = false;
+        break;
+      }
+      g_tc_fence_after();
+      const uint32_t a = ring + (uint32_t)s * stage_bytes;
+      const uint64_t adesc = g_smem_desc(a), bdesc = g_smem_desc(a + kTileABytes);
+#pragma unroll
+      for (int k4 = 0; k4 < kBlockK / 16; ++k4)         // 32 bytes along K per MMA: +2 in 16-byte units
+        g_umma_bf16(tmem_d, adesc + 2u * k4, bdesc + 2u * k4, idesc, (uint32_t)((i | k4) != 0));
+      g_umma_commit(g_smem_u32(&empty_bar[s]));         // the slot is free once these MMAs have read it
+    }
+    if (ok) g_umma_commit(g_smem_u32(&acc_bar));        // the accumulator is complete
+  } else if (tid >= 64 && p.mode == 1 && (tile * kTileM) / p.D < p.Hq + p.Hkv) {
+    // ---- warps 2..15, idle in the main loop: (cos, sin) of position * theta^(-2i/D) for every
+    // sequence and pair i, in double (a float angle is off by 1e-7 * position radians) ----
+    const int half = p.D >> 1, t = tid - 64;
+    double* inv_freq = reinterpret_cast<double*>(angles + (size_t)p.batch * half);
+    for (int i = t; i < half; i += kGemmThreads - 64) inv_freq[i] = exp(-2.0 * i / p.D * p.log_theta);
+    asm volatile("bar.sync 1, %0;" ::"n"(kGemmThreads - 64) : "memory");
+    for (int idx = t; idx < p.batch * half; idx += kGemmThreads - 64) {
+      const int b = idx / half, i = idx - b * half;
+      int32_t pos = __ldg(p.positions + b);
+      if (pos < 0) pos = 0;                             // inactive row: any finite value, the row is never appended
+      double sn, cn;
+      sincos((double)pos * inv_freq[i], &sn, &cn);
+      angles[idx] = make_float2((float)cn, (float)sn);
+    }
+  }
+  __syncwarp();
+
+  // ---- accumulators: TMEM -> registers -> shared memory, transposed to [column b][row] ----
+  // warp = (lane quadrant it may read, column group): quadrant = warp % 4, columns 16 * (warp / 4) + 64 j
+  const bool arrived = g_mbar_wait_bounded(g_smem_u32(&acc_bar), 0);
+  if (!arrived && tid == 0) atomicOr(p.status, kGemmErrTimeout);
+  const bool good = __syncthreads_and(arrived ? 1 : 0) && s_fail == 0;
+  g_stamp(p, cta, 2);
+  if (good) {
+    g_tc_fence_after();
+    const int quad = warp & 3, row = quad * 32 + lane;
+    for (int c0 = 16 * (warp >> 2); c0 < p.nb; c0 += 64) {
+      uint32_t r[16];
+      g_tmem_ld16(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, r);
+#pragma unroll
+      for (int j = 0; j < 16; ++j) stage_f[(c0 + j) * kTileM + row] = __uint_as_float(r[j]);
+    }
+    g_tc_fence_before();
+  }
+  __syncthreads();
+  if (warp == 1) g_tmem_dealloc(tmem_d, ncols);
+  g_stamp(p, cta, 3);
+
+  // ---- split-K: the last CTA of the tile to arrive adds the partial tiles in split order ----
+  // Ordering: every thread's partial stores happen before the CTA barrier, thread 0's ticket is an
+  // acq_rel atomic at gpu scope after it (release is cumulative over the barrier), and the last
+  // CTA's threads read only after a second barrier behind that atomic.
+  bool finish = good;
+  if (p.ksplit > 1) {
+    const int n4 = p.batch * kTileM / 4;
+    const size_t split_stride = (size_t)p.nb * kTileM / 4;
+    float4* part = reinterpret_cast<float4*>(p.partials + ((size_t)tile * p.ksplit * p.nb) * kTileM);
+    if (good)
+      for (int i = tid; i < n4; i += kGemmThreads) part[split * split_stride + i] = reinterpret_cast<const float4*>(stage_f)[i];
+    __syncthreads();
+    if (tid == 0) {
+      uint32_t prev;                                           // taken on failure too, so the count always completes
+      asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(p.tickets + tile) : "memory");
+      s_last = prev == (uint32_t)p.ksplit - 1u;
+      if (s_last) p.tickets[tile] = 0;                         // ready for the next launch
+    }
+    __syncthreads();
+    g_stamp(p, cta, 4);
+    finish = good && s_last != 0;
+  }
+  if (!finish) {
+    g_stamp(p, cta, 6);
+    return;
+  }
+
+  // ---- epilogue set-up (before the reduction, so that its loads overlap the reduction's) ----
+  const int r0 = 2 * (tid & 63), n0 = tile * kTileM + r0;
+  const bool live = n0 < p.n_out;
+  const int half = p.D >> 1;
+  int head = 0, d = 0, hh = 0, H = 1;
+  __nv_bfloat16* base = nullptr;
+  bool rotate = false;
+  if (p.mode == 1 && live) {
+    head = n0 / p.D;
+    d = n0 - head * p.D;
+    if (head < p.Hq) { base = p.q; hh = head; H = p.Hq; }
+    else if (head < p.Hq + p.Hkv) { base = p.kn; hh = head - p.Hq; H = p.Hkv; }
+    else { base = p.vn; hh = head - p.Hq - p.Hkv; H = p.Hkv; }
+    rotate = head < p.Hq + p.Hkv;
+  }
+  const int pr = r0 ^ half, i0 = d & (half - 1);
+  const float sgn = d < half ? -1.f : 1.f;      // out_i = x_i c - x_{i+half} s ; out_{i+half} = x_{i+half} c + x_i s
+  const float4* angles4 = reinterpret_cast<const float4*>(angles);   // (cos, sin) of pairs i0 and i0 + 1: 16 bytes
+
+  if (p.ksplit > 1) {
+    // Every other split's values are fetched at once (the reduction would otherwise be a chain of
+    // L2 round trips); this CTA's own are already in shared memory.  Summed in split order, so the
+    // result does not depend on which CTA came last.
+    const int n4 = p.batch * kTileM / 4;
+    const size_t split_stride = (size_t)p.nb * kTileM / 4;
+    const float4* part = reinterpret_cast<const float4*>(p.partials + ((size_t)tile * p.ksplit * p.nb) * kTileM);
+    constexpr int R = 4;
+    for (int ib = tid; ib < n4; ib += R * kGemmThreads) {
+      float4 v[R][kMaxSplit];
+#pragma unroll
+      for (int r = 0; r < R; ++r)
+#pragma unroll
+        for (int s = 0; s < kMaxSplit; ++s) {
+          const int i = ib + r * kGemmThreads;
+          if (i < n4 && s < p.ksplit && s != split) v[r][s] = __ldcg(part + s * split_stride + i);
+        }
+#pragma unroll
+      for (int r = 0; r < R; ++r) {
+        const int i = ib + r * kGemmThreads;
+        if (i >= n4) break;
+        const float4 own = reinterpret_cast<const float4*>(stage_f)[i];
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int s = 0; s < kMaxSplit; ++s)
+          if (s < p.ksplit) {
+            const float4 t = s == split ? own : v[r][s];
+            acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+          }
+        reinterpret_cast<float4*>(stage_f)[i] = acc;
+      }
+    }
+    __syncthreads();
+    g_stamp(p, cta, 5);
+  }
+
+  // ---- epilogue: thread = two adjacent weight rows, every kColPhases-th batch column ----
+  if (live) {
+    if (p.mode == 0) {
+      for (int b = tid >> 6; b < p.batch; b += kColPhases) {
+        const float2 v = *reinterpret_cast<const float2*>(&stage_f[b * kTileM + r0]);
+        *reinterpret_cast<__nv_bfloat162*>(&p.out[(size_t)b * p.n_out + n0]) = __floats2bfloat162_rn(v.x, v.y);
+      }
+    } else {
+      for (int b = tid >> 6; b < p.batch; b += kColPhases) {
+        float2 v = *reinterpret_cast<const float2*>(&stage_f[b * kTileM + r0]);
+        v.x = g_round_bf16(v.x);                 // the projection's own bf16 output, as a library GEMM rounds it
+        v.y = g_round_bf16(v.y);
+        if (rotate) {
+          float2 w = *reinterpret_cast<const float2*>(&stage_f[b * kTileM + pr]);
+          w.x = g_round_bf16(w.x);
+          w.y = g_round_bf16(w.y);
+          const float4 cs = angles4[(b * half + i0) >> 1];
+          v = make_float2(v.x * cs.x + sgn * (w.x * cs.y), v.y * cs.z + sgn * (w.y * cs.w));
+        }
+        *reinterpret_cast<__nv_bfloat162*>(&base[((size_t)b * H + hh) * p.D + d]) = __floats2bfloat162_rn(v.x, v.y);
+      }
+    }
+  }
+  g_stamp(p, cta, 6);
+}
+
+}  // namespace opw_afd
