@@ -395,6 +395,77 @@ def run_linear_layer(steps, batch=256, Hk=16, Hv=32, dk=128, dv=128, rotate=4):
             "steps": steps}
 
 
+def run_afd_module(steps, name="c2_llama8b", hidden=4096, layers=4):
+    """The complete attention module (QKV projection + rotary encoding + core attention + output
+    projection) on the workload's shape: time per module step with the projections on the
+    tensor-core kernel and on the library path, back to back over `layers` layers with their own
+    weights and KV pools (so neither stays in L2), beside the core-attention step alone."""
+    import numpy as np
+    import torch
+
+    from paper_2609_14237_b200 import binding, synth
+
+    wl = dataclasses.replace(synth.WORKLOADS[name], layer_window=[0] * layers)
+    total = steps + 8
+    inp = synth.make_inputs(wl, device="cuda", growth=3 * (total // layers + 2), steps=1)
+    Hq, Hkv, D, Bn = wl.num_q_heads, wl.num_kv_heads, wl.head_dim, wl.batch
+    stage = binding.Stage(pools=inp.pools, layer_window=wl.layer_window, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D,
+                          max_batch=Bn, max_pages_per_seq=inp.max_pages_per_seq)
+    g = torch.Generator(device="cuda")
+    g.manual_seed(3001)
+    w_qkv = [(torch.randn((Hq + 2 * Hkv) * D, hidden, device="cuda", generator=g) / hidden ** 0.5).to(torch.bfloat16)
+             for _ in range(layers)]
+    w_o = [(torch.randn(hidden, Hq * D, device="cuda", generator=g) / (Hq * D) ** 0.5).to(torch.bfloat16)
+           for _ in range(layers)]
+    x = torch.randn(Bn, hidden, device="cuda", generator=g).to(torch.bfloat16)
+    y = torch.empty_like(x)
+    out = torch.empty(Bn, Hq, D, dtype=torch.bfloat16, device="cuda")
+    pos0 = torch.from_numpy(inp.lengths.astype(np.int32)).cuda()
+    stream = torch.cuda.current_stream()
+
+    def timed(fn):
+        pos = pos0.clone()
+        for i in range(8):
+            fn(i % layers, pos)
+            if i % layers == layers - 1:
+                pos.add_(1)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for i in range(steps):
+            fn(i % layers, pos)
+            if i % layers == layers - 1:
+                pos.add_(1)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    stage_pdl = binding.Stage(pools=inp.pools, layer_window=wl.layer_window, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D,
+                              max_batch=Bn, max_pages_per_seq=inp.max_pages_per_seq, flags=binding.OPW_FLAG_PDL)
+    res = {}
+    for label, st, flags in (("tcgen05", stage, 0), ("library", stage, binding.OPW_AFD_LIBRARY_GEMM),
+                             ("tcgen05_pdl", stage_pdl, binding.OPW_AFD_PDL)):
+        mods = [binding.AfdModule(st, l, w_qkv[l], w_o[l], 10000.0, flags) for l in range(layers)]
+        res[label] = timed(lambda l, pos: mods[l].step(x, pos, inp.page_tables[l], y))
+        assert all(m.poll_error() == 0 for m in mods) and st.poll_error() == 0
+        for m in mods:
+            m.close()
+    stage_pdl.close()
+    q, k, v = inp.q[0, 0], inp.k_new[0, 0], inp.v_new[0, 0]
+    res["attention"] = timed(lambda l, pos: stage.decode_step(l, q, k, v, pos, inp.page_tables[l], out))
+    stage.close()
+    weight_bytes = 2 * ((Hq + 2 * Hkv) * D * hidden + hidden * Hq * D)
+    return {"value": round(Bn / (res["tcgen05"] * 1e-3), 1), "unit": "sequence-steps/s per layer (whole attention module)",
+            "ms_per_step": round(res["tcgen05"], 5), "ms_per_step_library_gemm": round(res["library"], 5),
+            "ms_per_step_programmatic_dependent_launch": round(res["tcgen05_pdl"], 5),
+            "ms_per_step_core_attention_alone": round(res["attention"], 5),
+            "projection_weight_bytes_per_step": weight_bytes, "kv_bytes_per_step": int(inp.kv_bytes(0, 0)),
+            "config": {"shape_of": name, "batch": Bn, "hidden": hidden, "num_q_heads": Hq, "num_kv_heads": Hkv, "head_dim": D,
+                       "l2": f"{layers} layers with their own weights ({layers * weight_bytes / 1e6:.0f} MB) and KV pools, back to back"},
+            "kernels": "skinny_gemm_kernel (tcgen05, rotary epilogue) x2 + attn_splitkv_kernel + combine_kernel per step",
+            "steps": steps}
+
+
 def cpu_baseline(name, inp=None, budget_s=15.0, device="cpu"):
     """The fp64 oracle as it stands, timed on this machine's host cores over a bounded sample of
     the workload's sequences (layer 0, step 0); value in the metric's unit."""
@@ -530,6 +601,15 @@ def main():
             dist.init_process_group(backend)
     steps = args.steps if args.steps is not None else 2000
     warmup = args.warmup if args.warmup is not None else 20
+    if args.workload == "attention_module":         # the AFD partition's stage alone (1 GPU)
+        r = run_afd_module(max(8, min(steps, 2000)))
+        r.update({"metric": "attention module decode: sequence-steps/s per layer", "n_gpus": 1, "warmup": 8,
+                  "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+                  "gpu_launches": r["steps"] * 4})
+        r["config"]["workload"] = "attention_module"
+        if rank == 0:
+            print(json.dumps(r), flush=True)
+        return
     if args.workload == "linear_state_layer":       # the recurrent-state layer alone (1 GPU)
         r = run_linear_layer(max(10, min(steps, 2000)))
         r.update({"metric": "recurrent-state layer decode: state GB/s (read + write)", "n_gpus": 1, "warmup": 5,
@@ -562,6 +642,7 @@ def main():
                             if key in r}
             others[name]["kv_bytes_per_step"] = r["config"]["kv_bytes_per_step"]
         others["linear_state_layer"] = run_linear_layer(max(10, min(steps, 500)))
+        others["attention_module_llama8b_layer"] = run_afd_module(max(8, min(steps, 400)))
         res["other_workloads"] = others
     if world > 1:
         import torch.distributed as dist

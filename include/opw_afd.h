@@ -39,6 +39,9 @@ extern "C" {
 typedef struct opw_afd_module opw_afd_module_t;
 
 #define OPW_AFD_LIBRARY_GEMM 1u /* projections by cuBLASLt + separate rotary kernel */
+#define OPW_AFD_PDL 2u          /* launch the tensor-core projections with programmatic dependent launch: their
+                                   set-up and the first weight tiles overlap the tail of the previous kernel in
+                                   the stream (pairs with OPW_FLAG_PDL of the stage) */
 
 /* Scratch bytes of one module: qkv, q, k_new, v_new and attention-output buffers for
  * max_batch rows, split-K partial tiles, 32 MiB of library GEMM workspace.  0 on invalid
@@ -52,7 +55,7 @@ size_t opw_afd_module_workspace_bytes(int32_t num_q_heads, int32_t num_kv_heads,
  *   w_o   : DEVICE bf16 [hidden, Hq * D]
  *   workspace : DEVICE, 256-byte aligned, >= opw_afd_module_workspace_bytes(...)
  * hidden must be a multiple of 8, the weights 16-byte aligned; rope_theta > 0 (e.g. 10000);
- * flags: 0 or OPW_AFD_LIBRARY_GEMM.  Clears the module's counters in the workspace
+ * flags: OPW_AFD_* or 0.  Clears the module's counters in the workspace
  * (synchronously).  The stage and the weights must outlive the module.
  */
 opw_status_t opw_afd_module_create(opw_attn_stage_t *stage, int32_t layer, int32_t hidden, const void *w_qkv,

@@ -116,7 +116,7 @@ struct opw_afd_module {
   unsigned char* ws;
   size_t off_qkv, off_q, off_k, off_v, off_out, off_gemm, off_partials, off_tickets, off_status;
   // tensor-core path
-  bool tc_qkv, tc_o;
+  bool tc_qkv, tc_o, pdl;
   int sms;
   TensorMapEncodeFn encode;
   CUtensorMap map_wqkv, map_wo;
@@ -224,8 +224,20 @@ opw_status_t run_tc_gemm(opw_afd_module* m, const CUtensorMap& map_w, const void
     if (!encode_map(m->encode, &map_x, xb, (uint64_t)nbatch, (uint64_t)k, (uint32_t)p.nb)) return OPW_ERR_CUDA;
     const size_t smem = 1024 + (size_t)stages * stage_bytes + angle_bytes;
     const dim3 grid(tiles_of(n_out), p.ksplit);
-    opw_afd::skinny_gemm_kernel<<<grid, opw_afd::kGemmThreads, smem, stream>>>(map_w, map_x, p);
-    if (cudaGetLastError() != cudaSuccess) return OPW_ERR_CUDA;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(opw_afd::kGemmThreads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = m->pdl ? 1 : 0;
+    if (cudaLaunchKernelEx(&cfg, opw_afd::skinny_gemm_kernel, map_w, map_x, p) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return OPW_ERR_CUDA;
+    }
     ++m->launches;
   }
   return OPW_OK;
@@ -244,7 +256,7 @@ opw_status_t opw_afd_module_create(opw_attn_stage_t* stage, int32_t layer, int32
                                    const void* w_o, float rope_theta, uint32_t flags, void* workspace,
                                    size_t workspace_bytes, opw_afd_module_t** out) {
   if (!stage || !w_qkv || !w_o || !workspace || !out) return OPW_ERR_INVALID_ARG;
-  if (hidden < 8 || hidden % 8 != 0 || !(rope_theta > 0.f) || (flags & ~OPW_AFD_LIBRARY_GEMM)) return OPW_ERR_INVALID_ARG;
+  if (hidden < 8 || hidden % 8 != 0 || !(rope_theta > 0.f) || (flags & ~(OPW_AFD_LIBRARY_GEMM | OPW_AFD_PDL))) return OPW_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255) || (reinterpret_cast<uintptr_t>(w_qkv) & 15) ||
       (reinterpret_cast<uintptr_t>(w_o) & 15))
     return OPW_ERR_INVALID_ARG;
@@ -272,6 +284,7 @@ opw_status_t opw_afd_module_create(opw_attn_stage_t* stage, int32_t layer, int32
   const bool library = (flags & OPW_AFD_LIBRARY_GEMM) != 0;
   m->tc_qkv = !library && D <= 128;         // the rotary epilogue needs a rotated pair inside one 128-row tile
   m->tc_o = !library;
+  m->pdl = (flags & OPW_AFD_PDL) != 0;
   bool ok = true;
   if (m->tc_qkv || m->tc_o) {
     void* fn = nullptr;

@@ -192,13 +192,16 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     p.trace[(size_t)cta * kTraceWords + 7] = sm;
   }
 
-  auto issue = [&](int i) {                                  // both tiles of k-block i into slot i % stages
+  // Slot i % stages takes the weight tile and the activation tile of k-block i; both count on one barrier.
+  auto issue_w = [&](int i) {
     const int s = i % p.stages;
     const uint32_t fb = g_smem_u32(&full_bar[s]);
-    const uint32_t a = ring + (uint32_t)s * stage_bytes;
     g_mbar_expect_tx(fb, stage_bytes);
-    g_tma_load_2d(a, &map_w, (kb0 + i) * kBlockK, tile * kTileM, fb);
-    g_tma_load_2d(a + kTileABytes, &map_x, (kb0 + i) * kBlockK, 0, fb);
+    g_tma_load_2d(ring + (uint32_t)s * stage_bytes, &map_w, (kb0 + i) * kBlockK, tile * kTileM, fb);
+  };
+  auto issue_x = [&](int i) {
+    const int s = i % p.stages;
+    g_tma_load_2d(ring + (uint32_t)s * stage_bytes + kTileABytes, &map_x, (kb0 + i) * kBlockK, 0, g_smem_u32(&full_bar[s]));
   };
 
   if (tid == 0) {
@@ -213,25 +216,34 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     s_last = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    // the first round of the ring needs no free-slot wait: start the stream before the TMEM allocation
-    for (int i = 0; i < nkb && i < p.stages; ++i) issue(i);
+    // The weights depend on nothing earlier in the stream and the first round of the ring needs no
+    // free-slot wait: their stream starts before the TMEM allocation and, under programmatic
+    // dependent launch, while the previous kernel is still draining.
+    for (int i = 0; i < nkb && i < p.stages; ++i) issue_w(i);
   }
   if (warp == 1) g_tmem_alloc(g_smem_u32(&tmem_slot), ncols);
   g_tc_fence_before();
   __syncthreads();
   g_tc_fence_after();
   const uint32_t tmem_d = tmem_slot;
+  // Programmatic dependent launch (no-ops without the launch attribute): the next kernel may queue
+  // up now; from here on this one touches what earlier kernels wrote (activations, positions,
+  // partial tiles, tickets), so it waits for them to be complete.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   g_stamp(p, cta, 1);
 
   if (tid == 0) {
     // ---- producer: one TMA load of the weight tile and one of the activation tile per k-block ----
+    for (int i = 0; i < nkb && i < p.stages; ++i) issue_x(i);
     for (int i = p.stages; i < nkb; ++i) {
       if (!g_mbar_wait_bounded(g_smem_u32(&empty_bar[i % p.stages]), (uint32_t)((i / p.stages) - 1) & 1u)) {
         s_fail = 1;
         atomicOr(p.status, kGemmErrTimeout);
         break;
       }
-      issue(i);
+      issue_w(i);
+      issue_x(i);
     }
   } else if (tid == 32) {
     // ---- MMA issuer ----

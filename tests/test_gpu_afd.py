@@ -144,16 +144,24 @@ def test_module_on_a_sliding_window_layer():
     run_module(5, [30, 100, 2000], 8, 2, 64, 256, steps=2, window=64)
 
 
+def test_module_with_programmatic_dependent_launch_over_back_to_back_steps():
+    """Projections launched with the attribute: the appended rows, q and y of every step are checked
+    after steps were enqueued without a host synchronisation in between."""
+    run_module(17, [40, 900, 33, 2047], 16, 4, 128, 1024, steps=3, flags=B.OPW_AFD_PDL)
+
+
 @BOTH
 def test_llama8b_layer_shape_and_a_batch_that_changes_between_steps(flags):
     run_module(21, [17, 900, 33, 2047, 512, 64, 5, 1200], 32, 8, 128, 4096, steps=3, batches=[8, 3, 8], flags=flags)
 
 
-def test_batches_of_one_row_and_of_more_than_256_rows():
-    """One row uses the narrowest accumulator (16 columns); 300 rows run as two column blocks."""
+def test_batches_of_one_row_and_around_the_switch_to_the_library_path():
+    """One row uses the narrowest accumulator (16 columns), 96 rows the widest the tensor-core path
+    takes (six column chunks), 97 and 300 rows go to the library path inside the same module."""
     run_module(31, [77], 8, 2, 128, 512, steps=2)
     rng = np.random.default_rng(32)
-    run_module(33, list(rng.integers(1, 60, 300)), 8, 2, 64, 256, steps=1, inactive=(0, 299))
+    for n in (96, 97, 300):
+        run_module(33 + n, list(rng.integers(1, 60, n)), 8, 2, 64, 256, steps=1, inactive=(0, n - 1))
 
 
 def test_the_two_projection_paths_agree():
@@ -205,7 +213,7 @@ def test_create_and_step_validate_arguments():
     base = (ws.data_ptr() + 255) // 256 * 256
     for kw, status in ((dict(layer=1), B.OPW_ERR_INVALID_ARG), (dict(hidden=12), B.OPW_ERR_INVALID_ARG),
                        (dict(rope_theta=0.0), B.OPW_ERR_INVALID_ARG), (dict(workspace=base + 8), B.OPW_ERR_INVALID_ARG),
-                       (dict(flags=2), B.OPW_ERR_INVALID_ARG),
+                       (dict(flags=4), B.OPW_ERR_INVALID_ARG),
                        (dict(workspace_bytes=nbytes - 1), B.OPW_ERR_CAPACITY)):
         args = dict(stage=stage.handle, layer=0, hidden=256, w_qkv=w_qkv.data_ptr(), w_o=w_o.data_ptr(),
                     rope_theta=1e4, workspace=base, workspace_bytes=nbytes)
