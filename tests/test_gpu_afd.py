@@ -135,7 +135,7 @@ BOTH = pytest.mark.parametrize("flags", [0, B.OPW_AFD_LIBRARY_GEMM], ids=["tcgen
 
 
 @BOTH
-@pytest.mark.parametrize("Hq,Hkv,D,hidden", [(8, 2, 64, 256), (16, 2, 128, 512), (8, 2, 256, 384), (6, 3, 64, 200)])
+@pytest.mark.parametrize("Hq,Hkv,D,hidden", [(8, 2, 64, 256), (16, 2, 128, 512), (8, 2, 256, 384), (6, 3, 64, 200), (4, 1, 64, 8)])
 def test_module_matches_the_oracle_stage_by_stage_and_end_to_end(Hq, Hkv, D, hidden, flags):
     run_module(11 + D, [1, 15, 16, 700, 3000], Hq, Hkv, D, hidden, steps=2, inactive=(2,), flags=flags)
 
