@@ -112,6 +112,37 @@ class ClockSampler(threading.Thread):
                 "samples": len(self.samples)}
 
 
+def measure_read_ceiling(gib=4, passes=10):
+    """Read-only streaming rate of this GPU in this run: the library's read probe (16-byte evict-first
+    loads, every word once) over a buffer far larger than L2, CUDA events, best of `passes`."""
+    import torch
+
+    from paper_2609_14237_b200 import binding
+
+    free = torch.cuda.mem_get_info()[0]
+    nbytes = min(gib << 30, (free // 4) & ~0xFFFFF)
+    if nbytes < (1 << 30):
+        return None
+    buf = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    buf.fill_(1)
+    sink = torch.zeros(4096, dtype=torch.float32, device="cuda")
+    stream = torch.cuda.current_stream()
+    best = None
+    for i in range(passes + 2):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        binding.opw_hbm_read_probe(buf.data_ptr(), nbytes, sink.data_ptr(), stream.cuda_stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        if i >= 2:
+            ms = e0.elapsed_time(e1)
+            best = ms if best is None else min(best, ms)
+    del buf
+    torch.cuda.empty_cache()
+    return {"value": round(nbytes / (best * 1e-3) / 1e9, 1), "unit": "GB/s", "bytes": int(nbytes), "passes": passes,
+            "kernel": "read_probe_kernel (opw_hbm_read_probe), best pass"}
+
+
 def build_stage(wl, rotate, total_rounds, device, tune):
     """R identical copies of a one-layer workload (or the workload's own layer stack)."""
     import torch
@@ -623,6 +654,11 @@ def main():
                 flags=1 if args.pdl else 0)
     res = run_ours(args.workload, steps, max(3, warmup), args.rotate, tune, want_e2e=not args.no_e2e, want_submit=(world == 1), unfused=args.unfused,
                    want_cpu=(world == 1 and rank == 0 and not args.no_cpu), world=world, rank=rank)
+    if world == 1 and rank == 0:
+        ceil = measure_read_ceiling()
+        if ceil is not None:
+            res["roofline"]["read_ceiling"] = ceil
+            res["roofline"]["frac_of_read_ceiling"] = round(res["roofline"]["achieved"] / ceil["value"], 4)
     if world == 1 and args.others:
         others = {}
         for name in args.others.split(","):

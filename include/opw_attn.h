@@ -333,6 +333,17 @@ opw_status_t opw_decode_attention_noalloc(int32_t num_q_heads, int32_t num_kv_he
                                           int32_t max_pages_per_seq, const void *q, const int32_t *kv_lens,
                                           const int32_t *page_table, void *out, float *lse, void *cuda_stream);
 
+/*
+ * Read-bandwidth probe: the ceiling the attention stage is measured against, next to the
+ * nominal and the copy figures (Section 3.1 models attention time as memory traffic over
+ * memory bandwidth; a decode step reads and writes almost nothing back, so the bandwidth that
+ * counts is the read-only one).  Enqueues one kernel that reads `bytes` (a multiple of 16, the
+ * buffer 16-byte aligned) of DEVICE memory once with 16-byte loads marked evict-first, sums
+ * them and writes one float per thread block to `sink` (DEVICE, >= 4096 floats) so that the
+ * loads cannot be dropped.  The caller times it (events) over a buffer larger than L2.
+ */
+opw_status_t opw_hbm_read_probe(const void *buffer, size_t bytes, float *sink, void *cuda_stream);
+
 /* Frees the host-side handle.  Does not touch device memory.  NULL is accepted. */
 opw_status_t opw_attn_stage_destroy(opw_attn_stage_t *stage);
 

@@ -32,7 +32,7 @@ EXPORTS = [
     "opw_linear_attn_decode_step", "opw_linear_attn_state_bytes", "opw_attn_plan_create_mixed",
     "opw_attn_stage_shape", "opw_afd_module_workspace_bytes", "opw_afd_module_create", "opw_afd_module_step",
     "opw_afd_module_intermediates", "opw_afd_module_destroy", "opw_afd_module_poll_error",
-    "opw_afd_module_launch_count", "opw_afd_module_set_trace",
+    "opw_afd_module_launch_count", "opw_afd_module_set_trace", "opw_hbm_read_probe",
 ]
 
 
@@ -171,6 +171,8 @@ def lib() -> ctypes.CDLL:
     L.opw_attn_plan_submit.argtypes = [vp, vp]
     L.opw_attn_plan_destroy.restype = ctypes.c_int
     L.opw_attn_plan_destroy.argtypes = [vp]
+    L.opw_hbm_read_probe.restype = ctypes.c_int
+    L.opw_hbm_read_probe.argtypes = [vp, ctypes.c_size_t, vp, vp]
     L.opw_attn_stage_shape.restype = ctypes.c_int
     L.opw_attn_stage_shape.argtypes = [vp] + [ctypes.POINTER(i32)] * 6
     L.opw_afd_module_workspace_bytes.restype = ctypes.c_size_t
@@ -379,6 +381,11 @@ def opw_attn_stage_set_trace(stage: int, trace: Optional[int], trace_bytes: int 
 
 def opw_attn_stage_launch_count(stage: int) -> int:
     return int(lib().opw_attn_stage_launch_count(stage))
+
+
+def opw_hbm_read_probe(buffer: int, nbytes: int, sink: int, stream: Optional[int] = None) -> None:
+    """Enqueue one pass of 16-byte evict-first loads over [buffer, buffer + nbytes) (device addresses)."""
+    _check(lib().opw_hbm_read_probe(buffer, nbytes, sink, stream), "opw_hbm_read_probe")
 
 
 def opw_attn_stage_shape(stage: int) -> dict:

@@ -159,7 +159,7 @@ Carve carve(int Hq, int Hkv, int D, int max_batch, int hidden) {
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   const int n_qkv = (Hq + 2 * Hkv) * D, n_attn = Hq * D;
-  const int nb = max_batch < 256 ? round16(max_batch) : 256;
+  const int nb = round16(max_batch < kTcMaxBatch ? max_batch : kTcMaxBatch);
   c.qkv = take((size_t)max_batch * n_qkv * 2);
   c.q = take((size_t)max_batch * n_attn * 2);
   c.k = take((size_t)max_batch * Hkv * D * 2);
@@ -192,54 +192,47 @@ bool encode_map(TensorMapEncodeFn fn, CUtensorMap* map, const void* base, uint64
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// One projection on the tensor-core kernel; batches beyond 256 rows go in blocks of 256.
+// One projection on the tensor-core kernel (batch <= kTcMaxBatch).
 opw_status_t run_tc_gemm(opw_afd_module* m, const CUtensorMap& map_w, const void* x, int batch, int n_out, int k, int mode,
-                         const int32_t* positions, __nv_bfloat16* out, __nv_bfloat16* q, __nv_bfloat16* kn, __nv_bfloat16* vn, cudaStream_t stream) {
-  for (int b0 = 0; b0 < batch; b0 += 256) {
-    const int nbatch = batch - b0 < 256 ? batch - b0 : 256;
-    opw_afd::GemmParams p;
-    p.n_out = n_out; p.k = k; p.batch = nbatch; p.nb = round16(nbatch);
-    const size_t stage_bytes = opw_afd::kTileABytes + (size_t)p.nb * 128;
-    // mode 1 keeps the step's angle table behind the ring: (cos, sin) per row and pair, then D/2 doubles
-    const size_t angle_bytes = mode == 1 ? (size_t)nbatch * (m->D / 2) * sizeof(float2) + (size_t)(m->D / 2) * sizeof(double) : 0;
-    int stages = (int)((kGemmSmemBudget - 1024 - angle_bytes) / stage_bytes);
-    if (stages > opw_afd::kMaxStages) stages = opw_afd::kMaxStages;
-    p.stages = stages;
-    p.ksplit = ksplit_of(n_out, k, m->sms < kSmsBound ? m->sms : kSmsBound);
-    p.mode = mode;
-    p.out = out ? out + (size_t)b0 * n_out : nullptr;
-    p.q = q ? q + (size_t)b0 * m->Hq * m->D : nullptr;
-    p.kn = kn ? kn + (size_t)b0 * m->Hkv * m->D : nullptr;
-    p.vn = vn ? vn + (size_t)b0 * m->Hkv * m->D : nullptr;
-    p.positions = positions ? positions + b0 : nullptr;
-    p.log_theta = m->log_theta;
-    p.Hq = m->Hq; p.Hkv = m->Hkv; p.D = m->D;
-    p.partials = reinterpret_cast<float*>(m->ws + m->off_partials);
-    p.tickets = reinterpret_cast<uint32_t*>(m->ws + m->off_tickets);
-    p.status = reinterpret_cast<uint32_t*>(m->ws + m->off_status);
-    // region 0: output projection, region 1: QKV projection (the last column block of a step stays)
-    p.trace = m->trace ? m->trace + (size_t)mode * opw_afd::kTraceMaxCtas * opw_afd::kTraceWords : nullptr;
-    CUtensorMap map_x;
-    const unsigned char* xb = static_cast<const unsigned char*>(x) + (size_t)b0 * k * 2;
-    if (!encode_map(m->encode, &map_x, xb, (uint64_t)nbatch, (uint64_t)k, (uint32_t)p.nb)) return OPW_ERR_CUDA;
-    const size_t smem = 1024 + (size_t)stages * stage_bytes + angle_bytes;
-    const dim3 grid(tiles_of(n_out), p.ksplit);
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid;
-    cfg.blockDim = dim3(opw_afd::kGemmThreads);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = m->pdl ? 1 : 0;
-    if (cudaLaunchKernelEx(&cfg, opw_afd::skinny_gemm_kernel, map_w, map_x, p) != cudaSuccess) {
-      (void)cudaGetLastError();
-      return OPW_ERR_CUDA;
-    }
-    ++m->launches;
+                         const int32_t* positions, __nv_bfloat16* out, __nv_bfloat16* q, __nv_bfloat16* kn,
+                         __nv_bfloat16* vn, cudaStream_t stream) {
+  opw_afd::GemmParams p;
+  p.n_out = n_out; p.k = k; p.batch = batch; p.nb = round16(batch);
+  const size_t stage_bytes = opw_afd::kTileABytes + (size_t)p.nb * 128;
+  // mode 1 keeps the step's angle table behind the ring: (cos, sin) per row and pair, then D/2 doubles
+  const size_t angle_bytes = mode == 1 ? (size_t)batch * (m->D / 2) * sizeof(float2) + (size_t)(m->D / 2) * sizeof(double) : 0;
+  int stages = (int)((kGemmSmemBudget - 1024 - angle_bytes) / stage_bytes);
+  if (stages > opw_afd::kMaxStages) stages = opw_afd::kMaxStages;
+  if ((size_t)stages * stage_bytes < (size_t)p.nb * opw_afd::kTileM * sizeof(float)) return OPW_ERR_UNSUPPORTED;   // the epilogue reuses the ring
+  p.stages = stages;
+  p.ksplit = ksplit_of(n_out, k, m->sms < kSmsBound ? m->sms : kSmsBound);
+  p.mode = mode;
+  p.out = out; p.q = q; p.kn = kn; p.vn = vn;
+  p.positions = positions;
+  p.log_theta = m->log_theta;
+  p.Hq = m->Hq; p.Hkv = m->Hkv; p.D = m->D;
+  p.partials = reinterpret_cast<float*>(m->ws + m->off_partials);
+  p.tickets = reinterpret_cast<uint32_t*>(m->ws + m->off_tickets);
+  p.status = reinterpret_cast<uint32_t*>(m->ws + m->off_status);
+  // trace region 0: output projection, region 1: QKV projection
+  p.trace = m->trace ? m->trace + (size_t)mode * opw_afd::kTraceMaxCtas * opw_afd::kTraceWords : nullptr;
+  CUtensorMap map_x;       // the activation pointer and the batch change from call to call: encoded per launch, on the host
+  if (!encode_map(m->encode, &map_x, x, (uint64_t)batch, (uint64_t)k, (uint32_t)p.nb)) return OPW_ERR_CUDA;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(tiles_of(n_out), p.ksplit);
+  cfg.blockDim = dim3(opw_afd::kGemmThreads);
+  cfg.dynamicSmemBytes = 1024 + (size_t)stages * stage_bytes + angle_bytes;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = m->pdl ? 1 : 0;
+  if (cudaLaunchKernelEx(&cfg, opw_afd::skinny_gemm_kernel, map_w, map_x, p) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return OPW_ERR_CUDA;
   }
+  ++m->launches;
   return OPW_OK;
 }
 

@@ -1,6 +1,7 @@
 // Skinny projection GEMM of the decode step on the 5th-generation tensor cores (sm_100a).
 //
-//   C[b, n] = sum_k x[b, k] * W[n, k]          x: [batch <= 256, K] bf16, W: [N, K] bf16, fp32 accumulate
+//   C[b, n] = sum_k x[b, k] * W[n, k]          x: [batch, K] bf16 (batch <= 256; the module stops at 96), W: [N, K] bf16,
+//                                               fp32 accumulate
 //
 // A decode step has few rows (the batch) and a large weight matrix that is read once, so the
 // kernel is built around streaming W: the WEIGHT rows take the tensor core's M dimension (one

@@ -498,6 +498,18 @@ opw_status_t opw_decode_step_host(opw_attn_stage_t* st, int32_t layer, int32_t b
   return OPW_OK;
 }
 
+opw_status_t opw_hbm_read_probe(const void* buffer, size_t bytes, float* sink, void* cuda_stream) {
+  if (!buffer || !sink || bytes == 0 || (bytes & 15) || (reinterpret_cast<uintptr_t>(buffer) & 15)) return OPW_ERR_INVALID_ARG;
+  int device = 0;
+  if (cudaGetDevice(&device) != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
+  int blocks = query_sms(device) * 8;                     // 8 blocks of 256 threads per SM, grid-stride
+  if (blocks > 4096) blocks = 4096;
+  opw::read_probe_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(cuda_stream)>>>(
+      static_cast<const uint4*>(buffer), (int64_t)(bytes / 16), sink);
+  if (cudaGetLastError() != cudaSuccess) return OPW_ERR_CUDA;
+  return OPW_OK;
+}
+
 opw_status_t opw_attn_stage_probe_timeout(opw_attn_stage_t* st, void* cuda_stream) {
   if (!st) return OPW_ERR_INVALID_ARG;
   opw::wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(cuda_stream)>>>(

@@ -293,6 +293,41 @@ __global__ void wait_probe_kernel(uint32_t* status) {
 }
 
 // ---------------------------------------------------------------------------------
+// read-bandwidth probe: every 16-byte word of a buffer once, evict-first, eight loads in flight
+// per thread; the per-block sums keep the loads alive
+// ---------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) read_probe_kernel(const uint4* __restrict__ buf, int64_t n16, float* __restrict__ sink) {
+  const uint64_t pol = l2_evict_first_policy();
+  const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+  uint32_t acc = 0;
+  int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  for (; i + 7 * stride < n16; i += 8 * stride) {
+    uint4 v[8];
+#pragma unroll
+    for (int u = 0; u < 8; ++u)
+      asm volatile("ld.global.nc.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                   : "=r"(v[u].x), "=r"(v[u].y), "=r"(v[u].z), "=r"(v[u].w)
+                   : "l"(buf + i + u * stride), "l"(pol));
+#pragma unroll
+    for (int u = 0; u < 8; ++u) acc ^= v[u].x ^ v[u].y ^ v[u].z ^ v[u].w;
+  }
+  for (; i < n16; i += stride) {
+    const uint4 v = __ldg(buf + i);
+    acc ^= v.x ^ v.y ^ v.z ^ v.w;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) acc ^= __shfl_xor_sync(0xffffffffu, acc, o);
+  __shared__ uint32_t part[8];
+  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = acc;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    uint32_t t = 0;
+    for (int w = 0; w < 8; ++w) t ^= part[w];
+    sink[blockIdx.x] = __uint_as_float(t & 0x3fffffffu);   // any value: it only has to depend on every load
+  }
+}
+
+// ---------------------------------------------------------------------------------
 // split-KV partial attention
 // ---------------------------------------------------------------------------------
 // Dynamic shared memory: [ring: warps*stages tiles][mbarriers: warps*stages x 8 B]

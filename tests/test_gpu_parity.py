@@ -701,3 +701,27 @@ def test_config5_hybrid_stack_sampled_rows_one_window_and_one_full_layer():
     if free < 70 * (1 << 30):
         pytest.skip("needs ~55 GB of device memory")
     run_full_config("c5_hybrid_stack", sample=1, layers=[2, 3])
+
+
+def test_read_probe_touches_every_word_and_validates_arguments():
+    """The bandwidth probe's sink must depend on every 16-byte word (xor of all words, per block),
+    otherwise the compiler or the hardware could drop loads and the ceiling would be fiction."""
+    n = (1 << 20) + 48                       # not a multiple of the unrolled stride: exercises the tail loop
+    buf = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    sink = torch.zeros(4096, dtype=torch.float32, device="cuda")
+    s = torch.cuda.current_stream().cuda_stream
+    B.opw_hbm_read_probe(buf.data_ptr(), n, sink.data_ptr(), s)
+    torch.cuda.synchronize()
+    base = sink.view(torch.int32).clone()
+    assert int(base.abs().sum()) == 0
+    for off in (0, 4096 + 16, n - 16):       # flip one bit in the first, a middle and the last word
+        buf.zero_()
+        buf[off] = 1
+        sink.zero_()
+        B.opw_hbm_read_probe(buf.data_ptr(), n, sink.data_ptr(), s)
+        torch.cuda.synchronize()
+        assert int((sink.view(torch.int32) != 0).sum()) == 1
+    for args in ((0, n), (buf.data_ptr(), 0), (buf.data_ptr(), n - 8), (buf.data_ptr() + 8, n - 16)):
+        with pytest.raises(B.OpwError) as e:
+            B.opw_hbm_read_probe(args[0], args[1], sink.data_ptr(), s)
+        assert e.value.status == B.OPW_ERR_INVALID_ARG
