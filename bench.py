@@ -176,8 +176,9 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
     e2e_steps = max(3, min(steps, 200)) if want_e2e else 0
     n_timed = warmup + steps + (e2e_steps + 3 if want_e2e else 0)
     n_used = n_timed                                 # steps the call-by-call and host-buffer loops take
-    n_timed += 2 * (steps + 8) if want_submit else 0  # room in the page tables for the plans' submissions
-    rounds = n_timed if stack else (n_timed + R - 1) // R
+    # a plan submission advances every layer by one token; two plans run, each 3 warm-up submissions + n_sub timed
+    n_sub = (steps if stack else max(steps // R, 10)) if want_submit else 0
+    rounds = (n_used if stack else (n_used + R - 1) // R) + (2 * (3 + n_sub) + 2 if want_submit else 0)
     wl_r, inp, st, pos_all, len_all = build_stage(wl, R, rounds, dev, tune)
     B, Hq, Hkv, D = wl.batch, wl.num_q_heads, wl.num_kv_heads, wl.head_dim
     out = torch.empty(B, Hq, D, dtype=torch.bfloat16, device=dev)
@@ -331,8 +332,8 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
         gpos = pos_all[t_now].clone()
         glen = len_all[t_now].clone()
         room = int(pos_all.shape[0] - 1 - t_now)                 # decode steps the page tables still cover
+        assert room >= 2 * (3 + n_sub), (room, n_sub)
         outs = [torch.empty_like(out) for _ in range(R)]        # one output buffer per item
-        n_sub = max(2, min(room // 2 - 3, max(steps // R, 10) if not stack else steps))
         for mode, extra in (("plan: CUDA graph + on-device advance", 0),
                             ("plan: CUDA graph + on-device advance + combine beside the next attention",
                              binding.OPW_PLAN_OVERLAP)):
