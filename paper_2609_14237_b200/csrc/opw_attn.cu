@@ -364,7 +364,8 @@ static opw_status_t launch_attention(opw_attn_stage_t* st, const StepArgs& a, in
 
 // The log-sum-exp combine of the same step.  `small` picks the 128-thread instance, which
 // fits on an SM beside a split-KV block.
-static opw_status_t launch_combine(opw_attn_stage_t* st, const StepArgs& a, int ws_set, cudaStream_t stream, bool small) {
+static opw_status_t launch_combine(opw_attn_stage_t* st, const StepArgs& a, int ws_set, cudaStream_t stream, bool small,
+                                   bool side_stream = false) {
   const int D = st->cfg.head_dim, Hq = st->cfg.num_q_heads, Hkv = st->cfg.num_kv_heads, G = Hq / Hkv;
   opw::CombineParams c;
   c.ticket = reinterpret_cast<int32_t*>(st->ws + st->lay.status + 16 + 16 * ws_set);
@@ -391,9 +392,9 @@ static opw_status_t launch_combine(opw_attn_stage_t* st, const StepArgs& a, int 
   if (splits > opw::kCombineBatch) splits = opw::kCombineBatch;
   if (splits > kCombineScratchSlots / rows) splits = kCombineScratchSlots / rows;
   if (splits < 1) splits = 1;
-  const bool pdl = (st->cfg.flags & OPW_FLAG_PDL) != 0 && !small;
+  const bool pdl = (st->cfg.flags & OPW_FLAG_PDL) != 0 && !side_stream;
   cudaError_t e = small ? launch(opw::combine_kernel<opw::kCombineThreadsSmall>, dim3(rows, splits),
-                                 dim3(opw::kCombineThreadsSmall), 0, stream, false, c)
+                                 dim3(opw::kCombineThreadsSmall), 0, stream, pdl, c)
                         : launch(opw::combine_kernel<opw::kCombineThreads>, dim3(rows, splits),
                                  dim3(opw::kCombineThreads), 0, stream, pdl, c);
   if (e != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
@@ -412,7 +413,10 @@ static opw_status_t enqueue_attention(opw_attn_stage_t* st, int32_t layer, int32
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   rc = launch_attention(st, a, 0, stream);
   if (rc != OPW_OK) return rc;
-  return launch_combine(st, a, 0, stream, false);
+  // With many rows the 128-thread instance wins (twice as many rows resident per SM hide the
+  // chain of L2 round trips a row's merge is); with few long rows the 256-thread one does.
+  const bool small = a.batch * st->cfg.num_kv_heads >= 2 * st->sms;
+  return launch_combine(st, a, 0, stream, small);
 }
 
 opw_status_t opw_decode_attention(opw_attn_stage_t* st, int32_t layer, int32_t batch, const void* q,
@@ -579,7 +583,7 @@ opw_status_t enqueue_plan_overlapped(opw_attn_plan* pl, cudaStream_t stream, cud
     if (rc != OPW_OK) return rc;
     if (cudaEventRecord(pl->ev_attn[i], stream) != cudaSuccess || cudaStreamWaitEvent(side, pl->ev_attn[i], 0) != cudaSuccess)
       return OPW_ERR_CUDA;
-    rc = launch_combine(st, a, set, side, true);
+    rc = launch_combine(st, a, set, side, true, true);
     if (rc != OPW_OK) return rc;
     if (cudaEventRecord(pl->ev_comb[i], side) != cudaSuccess) return OPW_ERR_CUDA;
     last = i;
