@@ -145,3 +145,28 @@ def test_without_a_device_create_fails_loudly_instead_of_falling_back():
     with pytest.raises(RuntimeError):
         B.Stage(pools=[torch.zeros(2 * 2 * 16 * 64 * 4, dtype=torch.bfloat16)], layer_window=[0], num_q_heads=8,
                 num_kv_heads=2, head_dim=64, max_batch=4, max_pages_per_seq=4)
+
+
+def test_attention_module_workspace_and_null_arguments_need_no_device():
+    """Host-only parts of the attention-module ABI: the workspace formula and the argument checks
+    that come before any CUDA call."""
+    base = B.opw_afd_module_workspace_bytes(32, 8, 128, 64, 4096)
+    # qkv + q + k + v + attention output buffers, split-K partial tiles, 32 MiB for the library GEMM
+    acts = 64 * (48 + 32 + 8 + 8 + 32) * 128 * 2
+    assert base >= acts + (32 << 20) and base % 256 == 0
+    assert B.opw_afd_module_workspace_bytes(32, 8, 128, 128, 4096) > base          # grows with the batch
+    assert B.opw_afd_module_workspace_bytes(32, 8, 128, 4096, 4096) - B.opw_afd_module_workspace_bytes(32, 8, 128, 2048, 4096) \
+        == 2048 * (48 + 32 + 8 + 8 + 32) * 128 * 2                                 # partial tiles stop growing at 96 rows
+    for bad in ((32, 7, 128, 64, 4096), (32, 8, 96, 64, 4096), (32, 8, 128, 0, 4096), (32, 8, 128, 64, 4100), (0, 8, 128, 64, 4096)):
+        assert B.opw_afd_module_workspace_bytes(*bad) == 0
+    L = B.lib()
+    h = ctypes.c_void_p()
+    assert L.opw_afd_module_create(None, 0, 4096, 16, 16, 1e4, 0, 256, 1 << 30, ctypes.byref(h)) == B.OPW_ERR_INVALID_ARG
+    assert L.opw_afd_module_step(None, 1, 16, 16, 16, 16, None) == B.OPW_ERR_INVALID_ARG
+    assert L.opw_afd_module_poll_error(None, None) == B.OPW_ERR_INVALID_ARG
+    assert L.opw_afd_module_set_trace(None, None, 0) == B.OPW_ERR_INVALID_ARG
+    assert L.opw_afd_module_launch_count(None) == 0
+    assert L.opw_afd_module_destroy(None) == B.OPW_OK
+    assert L.opw_attn_stage_shape(None, None, None, None, None, None, None) == B.OPW_ERR_INVALID_ARG
+    for buf, n in ((0, 1024), (4096, 0), (4096, 1000), (4104, 1024)):             # null, empty, ragged, misaligned
+        assert L.opw_hbm_read_probe(buf, n, 4096, None) == B.OPW_ERR_INVALID_ARG
