@@ -354,7 +354,6 @@ __global__ void __maxnreg__(D > 128 ? 255 : 200) attn_splitkv_kernel(AttnParams 
   constexpr int TILE = AttnSmem<D>::kTileBytes;
   extern __shared__ __align__(128) unsigned char smem[];
 
-  pdl_launch_dependents();                    // lets the combine kernel queue up behind this grid
   const int warps = blockDim.x >> 5;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int stages = p.stages;
@@ -787,6 +786,9 @@ __global__ void __maxnreg__(D > 128 ? 255 : 200) attn_splitkv_kernel(AttnParams 
   wb = describe(wbase + 32 + lane, u1);
   }
 
+  // The first warp of a block to run out of work lets the combine kernel queue up behind this grid:
+  // late enough that its blocks do not sit on the SMs while the stream is still running.
+  pdl_launch_dependents();
   if (tr && lane == 0) {
     tr[0] = (uint64_t)sm_id() | ((uint64_t)units_done << 32);
     tr[3] = global_timer_ns();
