@@ -231,3 +231,43 @@ def test_create_and_step_validate_arguments():
     mod.close()
     B.opw_afd_module_destroy(None)
     stage.close()
+
+
+@BOTH
+def test_module_at_config_2_full_size_the_shape_the_benchmark_times(flags):
+    """Llama-3-8B layer, batch 64, contexts U[1024, 4096], hidden 4096, the seeded pool and page tables
+    of the benchmark's workload: every row end to end against the oracle, the whole pool bitwise."""
+    from paper_2609_14237_b200 import synth
+
+    wl = synth.WORKLOADS["c2_llama8b"]
+    inp = synth.make_inputs(wl, device="cuda", growth=1, steps=1)
+    Hq, Hkv, D, Bn, hidden = wl.num_q_heads, wl.num_kv_heads, wl.head_dim, wl.batch, 4096
+    rng = np.random.default_rng(77)
+    w_qkv_bits = oracle.f32_to_bf16_bits((rng.standard_normal(((Hq + 2 * Hkv) * D, hidden)) / np.sqrt(hidden)).astype(np.float32))
+    w_o_bits = oracle.f32_to_bf16_bits((rng.standard_normal((hidden, Hq * D)) / np.sqrt(Hq * D)).astype(np.float32))
+    x_bits = oracle.f32_to_bf16_bits(rng.standard_normal((Bn, hidden)).astype(np.float32))
+    w_qkv, w_o, x = (oracle.bf16_bits_to_f64(a) for a in (w_qkv_bits, w_o_bits, x_bits))
+    pool, tab = inp.pools[0], inp.page_tables[0]
+    ref_pool = oracle.as_u16(pool.cpu()).copy()
+    before = ref_pool.copy()
+    pos = inp.positions(0)
+    stage = B.Stage(pools=[pool], layer_window=[0], num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, max_batch=Bn,
+                    max_pages_per_seq=inp.max_pages_per_seq)
+    mod = B.AfdModule(stage, 0, to_dev_bf16(w_qkv_bits), to_dev_bf16(w_o_bits), THETA, flags)
+    y = torch.full((Bn, hidden), float("nan"), dtype=torch.bfloat16, device="cuda")
+    mod.step(to_dev_bf16(x_bits), torch.from_numpy(pos).cuda(), tab, y)
+    torch.cuda.synchronize()
+    assert stage.poll_error() == B.OPW_OK and mod.poll_error() == B.OPW_OK
+    _, gk, gv, _ = mod.intermediates(Bn)
+    tab_np = tab.cpu().numpy()
+    assert oracle.kv_append(before, Hkv, D, P, tobits(gk), tobits(gv), pos, tab_np) == 0
+    assert (oracle.as_u16(pool.cpu()) == before).all()
+    ref_y, _, _, _ = afd.module_step(ref_pool, x, w_qkv, w_o, pos, tab_np, Hq, Hkv, D, THETA)
+    got = f64(y)
+    err = np.abs(got - ref_y)
+    rms = float(np.sqrt(np.mean(ref_y ** 2)))
+    assert np.isfinite(got).all()
+    assert (err <= 2.0 ** -5 * rms + 2.0 ** -8 * np.abs(ref_y)).all(), (err.max(), rms)
+    assert err.mean() <= 2.0 ** -7 * rms, (err.mean(), rms)
+    mod.close()
+    stage.close()
