@@ -78,7 +78,8 @@ typedef struct {
   size_t workspace_bytes;         /* >= opw_attn_stage_workspace_bytes(cfg) */
   float softmax_scale;            /* 0 -> 1/sqrt(head_dim) */
   uint32_t flags;                 /* OPW_FLAG_* */
-  int32_t tune_warps;             /* 0 = default (8; 6 at head_dim 256); warps per thread block (1..8) */
+  int32_t tune_warps;             /* 0 = default (8; 6 at head_dim 256, 12 at head_dim 64); warps per thread block
+                                     (1..16; what does not fit the register file is refused with OPW_ERR_CAPACITY) */
   int32_t tune_stages;            /* 0 = default; shared-memory ring depth per warp (2..16) */
   int32_t tune_ctas_per_sm;       /* 0 = default; resident thread blocks per SM (1..4) */
   int32_t reserved;               /* must be 0 */

@@ -38,7 +38,9 @@ bool shape_ok(const opw_attn_stage_config_t* c) {
 
 opw_status_t resolve_shape(const opw_attn_stage_config_t* c, Shape* s) {
   // head_dim 256 doubles the tile: six warps x two stages x 16 KB fill an SM's shared memory
-  s->warps = c->tune_warps ? c->tune_warps : (c->head_dim > 128 ? 6 : kDefaultWarps);
+  // and at head_dim 64 a unit is only 4 KB, its fixed cost (wait, loads of the matrix fragments, softmax)
+  // weighs more, and the smaller register footprint leaves room for twelve warps to hide it
+  s->warps = c->tune_warps ? c->tune_warps : (c->head_dim > 128 ? 6 : c->head_dim == 64 ? 12 : kDefaultWarps);
   s->stages = c->tune_stages ? c->tune_stages : kDefaultStages;
   s->ctas_per_sm = c->tune_ctas_per_sm ? c->tune_ctas_per_sm : kDefaultCtasPerSm;
   if (s->warps < 1 || s->warps > opw::kMaxWarps || s->stages < 2 || s->stages > 16 || s->ctas_per_sm < 1 ||
@@ -203,6 +205,23 @@ opw_status_t opw_attn_stage_create(const opw_attn_stage_config_t* cfg, opw_attn_
     e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_i);
   }
   if (e != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
+  {
+    // Registers decide how many warps a block may have (eight at head_dim 128, twelve at 64): ask the
+    // runtime now, so that a tuning that cannot launch is refused here and not at the first step.
+    const int G = cfg->num_q_heads / cfg->num_kv_heads;
+    int resident = 0;
+    const int threads = s.warps * 32;
+    if (cfg->head_dim == 64)
+      e = G > 8 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, opw::attn_splitkv_kernel<64, true>, threads, smem)
+                : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, opw::attn_splitkv_kernel<64, false>, threads, smem);
+    else if (cfg->head_dim == 128)
+      e = G > 8 ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, opw::attn_splitkv_kernel<128, true>, threads, smem)
+                : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, opw::attn_splitkv_kernel<128, false>, threads, smem);
+    else
+      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&resident, opw::attn_splitkv_kernel<256, false>, threads, smem);
+    if (e != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
+    if (resident < s.ctas_per_sm) return OPW_ERR_CAPACITY;
+  }
   if (cudaMemset(cfg->workspace, 0, 256) != cudaSuccess ||
       cudaMemset(static_cast<unsigned char*>(cfg->workspace) + lay.row_count, 0,
                  (size_t)cfg->max_batch * cfg->num_kv_heads * 4) != cudaSuccess) {

@@ -31,7 +31,7 @@ namespace OPW_NAMESPACE {
 constexpr int kPage = 16;               // tokens per page
 constexpr uint32_t kErrBadPage = 1u;    // bits of the device status word
 constexpr uint32_t kErrTimeout = 2u;
-constexpr int kMaxWarps = 8;
+constexpr int kMaxWarps = 16;
 constexpr uint64_t kWaitLimitNs = 100ull * 1000 * 1000;   // bound of a wait on a shared-memory copy: 0.1 s
 
 struct AttnParams {

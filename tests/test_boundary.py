@@ -95,7 +95,7 @@ def test_workspace_bytes_needs_a_valid_shape():
     (dict(layer_kv_pool=[0x10010]), B.OPW_ERR_INVALID_ARG),
     (dict(layer_num_pages=[0]), B.OPW_ERR_INVALID_ARG),
     (dict(layer_window=[-1]), B.OPW_ERR_INVALID_ARG),
-    (dict(tune_warps=9), B.OPW_ERR_INVALID_ARG),
+    (dict(tune_warps=17), B.OPW_ERR_INVALID_ARG),
     (dict(tune_stages=1), B.OPW_ERR_INVALID_ARG),
     (dict(softmax_scale=-1.0), B.OPW_ERR_INVALID_ARG),
     (dict(head_dim=128, tune_warps=8, tune_stages=4), B.OPW_ERR_CAPACITY),

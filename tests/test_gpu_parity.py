@@ -725,3 +725,26 @@ def test_read_probe_touches_every_word_and_validates_arguments():
         with pytest.raises(B.OpwError) as e:
             B.opw_hbm_read_probe(args[0], args[1], sink.data_ptr(), s)
         assert e.value.status == B.OPW_ERR_INVALID_ARG
+
+
+def test_a_warp_count_the_register_file_cannot_hold_is_refused_at_create():
+    pool = torch.zeros(4 * 8 * 2 * P * 128, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(B.OpwError) as e:
+        B.Stage(pools=[pool], layer_window=[0], num_q_heads=32, num_kv_heads=8, head_dim=128, max_batch=2,
+                max_pages_per_seq=2, tune_warps=12)
+    assert e.value.status == B.OPW_ERR_CAPACITY
+    pool64 = torch.zeros(4 * 8 * 2 * P * 64, dtype=torch.bfloat16, device="cuda")
+    B.Stage(pools=[pool64], layer_window=[0], num_q_heads=32, num_kv_heads=8, head_dim=64, max_batch=2,
+            max_pages_per_seq=2, tune_warps=12).close()
+
+
+def test_head_dim_64_at_scale_default_twelve_warps():
+    """Long rows at head_dim 64 with the default tuning (twelve warps per block): sampled rows against the oracle."""
+    rng = np.random.default_rng(64)
+    lens = [9000, 33, 20000, 4097, 16]
+    pool, tab, q, _, _ = make_case(rng, lens, 32, 8, 64)
+    ref, ref_lse, rc = oracle.decode_attention(pool, 32, 8, 64, P, q, lens, tab)
+    assert rc == 0
+    out, lse, rc, _ = gpu_attention(pool, tab, q, lens, 32, 8, 64)
+    assert rc == B.OPW_OK
+    check_close(out_to_f64(out), ref, lse, ref_lse)
