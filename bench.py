@@ -439,7 +439,7 @@ def run_afd_module(steps, name="c2_llama8b", hidden=4096, layers=4):
 
     wl = dataclasses.replace(synth.WORKLOADS[name], layer_window=[0] * layers)
     total = steps + 8
-    inp = synth.make_inputs(wl, device="cuda", growth=3 * (total // layers + 2), steps=1)
+    inp = synth.make_inputs(wl, device="cuda", growth=4 * (total // layers + 4), steps=1)
     Hq, Hkv, D, Bn = wl.num_q_heads, wl.num_kv_heads, wl.head_dim, wl.batch
     stage = binding.Stage(pools=inp.pools, layer_window=wl.layer_window, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D,
                           max_batch=Bn, max_pages_per_seq=inp.max_pages_per_seq)
@@ -480,6 +480,25 @@ def run_afd_module(steps, name="c2_llama8b", hidden=4096, layers=4):
         mods = [binding.AfdModule(st, l, w_qkv[l], w_o[l], 10000.0, flags) for l in range(layers)]
         res[label] = timed(lambda l, pos: mods[l].step(x, pos, inp.page_tables[l], y))
         assert all(m.poll_error() == 0 for m in mods) and st.poll_error() == 0
+        if label == "tcgen05_pdl":
+            # the same steps as one plan: all layers' module steps in one CUDA graph, positions advanced on the device
+            pos = pos0.clone()
+            ops = [dict(kind="afd_module", module=mods[l].handle, batch=Bn, x=x.data_ptr(), positions=pos.data_ptr(),
+                        page_table=inp.page_tables[l].data_ptr(), y=y.data_ptr()) for l in range(layers)]
+            plan = binding.opw_attn_plan_create_mixed(st.handle, ops, binding.OPW_PLAN_GRAPH | binding.OPW_PLAN_ADVANCE)
+            n_sub = max(2, steps // layers)
+            for _ in range(2):
+                binding.opw_attn_plan_submit(plan, stream.cuda_stream)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(n_sub):
+                binding.opw_attn_plan_submit(plan, stream.cuda_stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            res["plan"] = e0.elapsed_time(e1) / (n_sub * layers)
+            assert all(m.poll_error() == 0 for m in mods) and st.poll_error() == 0
+            binding.opw_attn_plan_destroy(plan)
         for m in mods:
             m.close()
     stage_pdl.close()
@@ -490,6 +509,7 @@ def run_afd_module(steps, name="c2_llama8b", hidden=4096, layers=4):
     return {"value": round(Bn / (res["tcgen05"] * 1e-3), 1), "unit": "sequence-steps/s per layer (whole attention module)",
             "ms_per_step": round(res["tcgen05"], 5), "ms_per_step_library_gemm": round(res["library"], 5),
             "ms_per_step_programmatic_dependent_launch": round(res["tcgen05_pdl"], 5),
+            "ms_per_step_plan": round(res["plan"], 5),
             "ms_per_step_core_attention_alone": round(res["attention"], 5),
             "projection_weight_bytes_per_step": weight_bytes, "kv_bytes_per_step": int(inp.kv_bytes(0, 0)),
             "config": {"shape_of": name, "batch": Bn, "hidden": hidden, "num_q_heads": Hq, "num_kv_heads": Hkv, "head_dim": D,

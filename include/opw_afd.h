@@ -95,6 +95,21 @@ int64_t opw_afd_module_launch_count(const opw_afd_module_t *module);
 
 opw_status_t opw_afd_module_destroy(opw_afd_module_t *module); /* NULL is accepted */
 
+/*
+ * One module step as an op of a mixed plan (opw_attn_plan_create_mixed in opw_linear_attn.h, kind
+ * OPW_OP_AFD_MODULE): the single native submission of Section 6.2 for a stage that holds complete
+ * attention modules.  Arguments as for opw_afd_module_step; `positions` is advanced by one per
+ * submission under OPW_PLAN_ADVANCE.  The module must belong to the plan's stage and outlive the plan.
+ */
+typedef struct {
+  opw_afd_module_t *module;
+  int32_t batch;
+  const void *x;             /* DEVICE bf16 [batch, hidden] */
+  int32_t *positions;        /* DEVICE int32 [batch] */
+  const int32_t *page_table; /* DEVICE int32 [batch, max_pages_per_seq] */
+  void *y;                   /* DEVICE bf16 [batch, hidden] */
+} opw_afd_item_t;
+
 #ifdef __cplusplus
 }
 #endif

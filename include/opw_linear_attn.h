@@ -26,6 +26,7 @@
 #ifndef OPW_LINEAR_ATTN_H_
 #define OPW_LINEAR_ATTN_H_
 
+#include "opw_afd.h"
 #include "opw_attn.h"
 
 #ifdef __cplusplus
@@ -52,11 +53,12 @@ opw_status_t opw_linear_attn_decode_step(int32_t batch, int32_t num_k_heads, int
 
 /*
  * Mixed plans: one native submission (Section 6.2) for a hybrid stack that interleaves
- * attention layers with recurrent-state layers.  An op is either one attention item (see
- * opw_step_item_t in opw_attn.h) or one recurrent-state step with the arguments of
- * opw_linear_attn_decode_step; ops run in the order given, one after the other.  Flags as for
+ * attention layers with recurrent-state layers, or for a stage that holds whole attention
+ * modules.  An op is one attention item (see opw_step_item_t in opw_attn.h), one recurrent-state
+ * step with the arguments of opw_linear_attn_decode_step, or one attention-module step
+ * (opw_afd_item_t in opw_afd.h); ops run in the order given, one after the other.  Flags as for
  * opw_attn_plan_create, except that OPW_PLAN_OVERLAP is not available (OPW_ERR_UNSUPPORTED);
- * OPW_PLAN_ADVANCE touches the attention items' positions / kv_lens only.  Submit and destroy
+ * OPW_PLAN_ADVANCE touches the positions / kv_lens of attention items and module steps only.  Submit and destroy
  * with opw_attn_plan_submit / opw_attn_plan_destroy.
  */
 typedef struct {
@@ -72,10 +74,12 @@ typedef struct {
 
 #define OPW_OP_ATTENTION 0
 #define OPW_OP_LINEAR 1
+#define OPW_OP_AFD_MODULE 2
 typedef struct {
-  int32_t kind;                /* OPW_OP_ATTENTION or OPW_OP_LINEAR */
+  int32_t kind;                /* OPW_OP_ATTENTION, OPW_OP_LINEAR or OPW_OP_AFD_MODULE */
   opw_step_item_t attention;   /* used when kind == OPW_OP_ATTENTION */
   opw_linear_item_t linear;    /* used when kind == OPW_OP_LINEAR */
+  opw_afd_item_t afd;          /* used when kind == OPW_OP_AFD_MODULE (see opw_afd.h) */
 } opw_plan_op_t;
 
 opw_status_t opw_attn_plan_create_mixed(opw_attn_stage_t *stage, const opw_plan_op_t *ops, int32_t n_ops,

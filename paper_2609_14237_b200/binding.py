@@ -86,11 +86,16 @@ class LinearItem(ctypes.Structure):
     ]
 
 
+class AfdItem(ctypes.Structure):
+    _fields_ = [("module", ctypes.c_void_p), ("batch", ctypes.c_int32), ("x", ctypes.c_void_p),
+                ("positions", ctypes.c_void_p), ("page_table", ctypes.c_void_p), ("y", ctypes.c_void_p)]
+
+
 class PlanOp(ctypes.Structure):
-    _fields_ = [("kind", ctypes.c_int32), ("attention", StepItem), ("linear", LinearItem)]
+    _fields_ = [("kind", ctypes.c_int32), ("attention", StepItem), ("linear", LinearItem), ("afd", AfdItem)]
 
 
-OPW_OP_ATTENTION, OPW_OP_LINEAR = 0, 1
+OPW_OP_ATTENTION, OPW_OP_LINEAR, OPW_OP_AFD_MODULE = 0, 1, 2
 OPW_PLAN_GRAPH, OPW_PLAN_ADVANCE, OPW_PLAN_OVERLAP = 1, 2, 4
 OPW_AFD_LIBRARY_GEMM, OPW_AFD_PDL = 1, 2
 
@@ -323,8 +328,9 @@ def opw_attn_plan_create(stage: int, items: Sequence[dict], flags: int = 0) -> i
 
 
 def opw_attn_plan_create_mixed(stage: int, ops: Sequence[dict], flags: int = 0) -> int:
-    """ops: dicts with kind "attention" (fields of an attention item) or "linear" (batch, num_k_heads,
-    num_v_heads, dk, dv, state, num_slots, slot, q, k, v, a, beta, out and optionally scale)."""
+    """ops: dicts with kind "attention" (fields of an attention item), "linear" (batch, num_k_heads,
+    num_v_heads, dk, dv, state, num_slots, slot, q, k, v, a, beta, out and optionally scale) or
+    "afd_module" (module, batch, x, positions, page_table, y)."""
     arr = (PlanOp * len(ops))()
     for a, op in zip(arr, ops):
         if op["kind"] == "attention":
@@ -332,6 +338,11 @@ def opw_attn_plan_create_mixed(stage: int, ops: Sequence[dict], flags: int = 0) 
             a.attention.layer, a.attention.batch = op["layer"], op["batch"]
             for k in ("q", "k_new", "v_new", "positions", "kv_lens", "page_table", "out", "lse"):
                 setattr(a.attention, k, op.get(k))
+        elif op["kind"] == "afd_module":
+            a.kind = OPW_OP_AFD_MODULE
+            a.afd.batch = int(op["batch"])
+            for k in ("module", "x", "positions", "page_table", "y"):
+                setattr(a.afd, k, op[k])
         else:
             a.kind = OPW_OP_LINEAR
             for k in ("batch", "num_k_heads", "num_v_heads", "dk", "dv", "num_slots"):

@@ -2,6 +2,7 @@
 // carving, launches.  The library allocates no device memory and never synchronises
 // except in opw_attn_stage_poll_error and (once) in opw_attn_stage_create.
 #include "opw_attn.h"
+#include "opw_afd.h"
 #include "opw_linear_attn.h"
 
 #include <cmath>
@@ -565,8 +566,10 @@ opw_status_t opw_attn_stage_poll_error(opw_attn_stage_t* st, void* cuda_stream) 
 struct opw_attn_plan {
   opw_attn_stage* stage;
   std::vector<opw_step_item_t> items;
-  std::vector<opw_linear_item_t> linear;    // recurrent-state ops of a mixed plan ...
-  std::vector<int> linear_after;            // ... each runs after attention item linear_after[i] (-1: first)
+  // the other ops of a mixed plan (recurrent-state steps, whole attention modules), in the order given;
+  // each runs after attention item extra_after[i] (-1: before the first)
+  std::vector<opw_plan_op_t> extra;
+  std::vector<int> extra_after;
   uint32_t flags;
   cudaStream_t side;                     // OPW_PLAN_OVERLAP: the combines run here
   std::vector<cudaEvent_t> ev_attn, ev_comb;
@@ -618,14 +621,20 @@ opw_status_t enqueue_plan(opw_attn_plan* pl, cudaStream_t stream, cudaStream_t s
     if (rc != OPW_OK) { (void)cudaGetLastError(); return rc; }
   } else
   for (int i = -1; i < (int)pl->items.size(); ++i) {
-    for (size_t j = 0; j < pl->linear.size(); ++j) {       // recurrent-state ops placed after item i
-      if (pl->linear_after[j] != i) continue;
-      const opw_linear_item_t& ln = pl->linear[j];
-      opw_status_t rl = opw_linear_attn_decode_step(ln.batch, ln.num_k_heads, ln.num_v_heads, ln.dk, ln.dv, ln.state,
-                                                    ln.num_slots, ln.slot, ln.q, ln.k, ln.v, ln.a, ln.beta, ln.scale,
-                                                    ln.out, stream);
-      if (rl != OPW_OK) return rl;
-      if (ln.batch > 0) st->launches += 1;
+    for (size_t j = 0; j < pl->extra.size(); ++j) {        // the other ops placed after item i
+      if (pl->extra_after[j] != i) continue;
+      if (pl->extra[j].kind == OPW_OP_LINEAR) {
+        const opw_linear_item_t& ln = pl->extra[j].linear;
+        opw_status_t rl = opw_linear_attn_decode_step(ln.batch, ln.num_k_heads, ln.num_v_heads, ln.dk, ln.dv, ln.state,
+                                                      ln.num_slots, ln.slot, ln.q, ln.k, ln.v, ln.a, ln.beta, ln.scale,
+                                                      ln.out, stream);
+        if (rl != OPW_OK) return rl;
+        if (ln.batch > 0) st->launches += 1;
+      } else {
+        const opw_afd_item_t& am = pl->extra[j].afd;     // counts its own launches (and the stage its attention's)
+        opw_status_t ra = opw_afd_module_step(am.module, am.batch, am.x, am.positions, am.page_table, am.y, stream);
+        if (ra != OPW_OK) return ra;
+      }
     }
     if (i + 1 >= (int)pl->items.size()) break;
     const opw_step_item_t& it = pl->items[i + 1];
@@ -644,7 +653,15 @@ opw_status_t enqueue_plan(opw_attn_plan* pl, cudaStream_t stream, cudaStream_t s
   }
   if (pl->flags & OPW_PLAN_ADVANCE) {
     std::vector<const void*> done;
-    for (const opw_step_item_t& it : pl->items) {
+    std::vector<opw_step_item_t> moving(pl->items);
+    for (const opw_plan_op_t& op : pl->extra)
+      if (op.kind == OPW_OP_AFD_MODULE) {
+        opw_step_item_t it = {};
+        it.batch = op.afd.batch;
+        it.positions = op.afd.positions;
+        moving.push_back(it);
+      }
+    for (const opw_step_item_t& it : moving) {
       int32_t* pos = it.positions;
       int32_t* len = it.kv_lens;
       for (const void* d : done) {
@@ -668,11 +685,11 @@ opw_status_t enqueue_plan(opw_attn_plan* pl, cudaStream_t stream, cudaStream_t s
 extern "C" {
 
 static opw_status_t build_plan(opw_attn_stage_t* st, const opw_step_item_t* items, int32_t n_items,
-                               const opw_linear_item_t* linear, const int* linear_after, int32_t n_linear, uint32_t flags,
+                               const opw_plan_op_t* extra, const int* extra_after, int32_t n_extra, uint32_t flags,
                                opw_attn_plan_t** out) {
-  if (!st || !out || n_items < 0 || n_items + n_linear < 1 || (n_items > 0 && !items)) return OPW_ERR_INVALID_ARG;
+  if (!st || !out || n_items < 0 || n_items + n_extra < 1 || (n_items > 0 && !items)) return OPW_ERR_INVALID_ARG;
   if (flags & ~(uint32_t)(OPW_PLAN_GRAPH | OPW_PLAN_ADVANCE | OPW_PLAN_OVERLAP)) return OPW_ERR_INVALID_ARG;
-  if ((flags & OPW_PLAN_OVERLAP) && n_linear > 0) return OPW_ERR_UNSUPPORTED;
+  if ((flags & OPW_PLAN_OVERLAP) && n_extra > 0) return OPW_ERR_UNSUPPORTED;
   for (int i = 0; i < n_items; ++i) {
     const opw_step_item_t& it = items[i];
     opw_status_t rc = check_step(st, it.layer, it.batch);
@@ -695,9 +712,9 @@ static opw_status_t build_plan(opw_attn_stage_t* st, const opw_step_item_t* item
   if (!pl) return OPW_ERR_INVALID_ARG;
   pl->stage = st;
   if (n_items > 0) pl->items.assign(items, items + n_items);
-  if (n_linear > 0) {
-    pl->linear.assign(linear, linear + n_linear);
-    pl->linear_after.assign(linear_after, linear_after + n_linear);
+  if (n_extra > 0) {
+    pl->extra.assign(extra, extra + n_extra);
+    pl->extra_after.assign(extra_after, extra_after + n_extra);
   }
   pl->flags = flags;
   pl->side = nullptr;
@@ -749,23 +766,27 @@ opw_status_t opw_attn_plan_create_mixed(opw_attn_stage_t* st, const opw_plan_op_
                                         opw_attn_plan_t** out) {
   if (!st || !ops || n_ops < 1 || !out) return OPW_ERR_INVALID_ARG;
   std::vector<opw_step_item_t> items;
-  std::vector<opw_linear_item_t> linear;
+  std::vector<opw_plan_op_t> extra;
   std::vector<int> after;
   for (int i = 0; i < n_ops; ++i) {
     if (ops[i].kind == OPW_OP_ATTENTION) {
       items.push_back(ops[i].attention);
-    } else if (ops[i].kind == OPW_OP_LINEAR) {
+      continue;
+    }
+    if (ops[i].kind == OPW_OP_LINEAR) {
       const opw_linear_item_t& ln = ops[i].linear;
       if (ln.batch < 0 || !ln.state || !ln.slot || !ln.q || !ln.k || !ln.v || !ln.a || !ln.beta || !ln.out)
         return OPW_ERR_INVALID_ARG;
-      linear.push_back(ln);
-      after.push_back((int)items.size() - 1);
+    } else if (ops[i].kind == OPW_OP_AFD_MODULE) {
+      const opw_afd_item_t& am = ops[i].afd;
+      if (!am.module || am.batch < 1 || !am.x || !am.positions || !am.page_table || !am.y) return OPW_ERR_INVALID_ARG;
     } else {
       return OPW_ERR_INVALID_ARG;
     }
+    extra.push_back(ops[i]);
+    after.push_back((int)items.size() - 1);
   }
-  return build_plan(st, items.data(), (int32_t)items.size(), linear.data(), after.data(), (int32_t)linear.size(), flags,
-                    out);
+  return build_plan(st, items.data(), (int32_t)items.size(), extra.data(), after.data(), (int32_t)extra.size(), flags, out);
 }
 
 opw_status_t opw_attn_plan_submit(opw_attn_plan_t* pl, void* cuda_stream) {

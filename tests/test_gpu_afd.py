@@ -271,3 +271,60 @@ def test_module_at_config_2_full_size_the_shape_the_benchmark_times(flags):
     assert err.mean() <= 2.0 ** -7 * rms, (err.mean(), rms)
     mod.close()
     stage.close()
+
+
+@pytest.mark.parametrize("plan_flags", [0, B.OPW_PLAN_GRAPH | B.OPW_PLAN_ADVANCE])
+@BOTH
+def test_a_plan_of_module_steps_equals_the_same_steps_called_one_by_one(flags, plan_flags):
+    """Two layers' attention modules as ops of one plan (one native submission per token), three
+    tokens: outputs and both KV pools bit for bit as from opw_afd_module_step calls."""
+    rng = np.random.default_rng(91)
+    Hq, Hkv, D, hidden, lens = 16, 4, 128, 1024, [40, 900, 33, 2047]
+    Bn, steps = len(lens), 3
+    cases = [make_case(rng, [n + steps for n in lens], Hq, Hkv, D) for _ in range(2)]
+    w = [(to_dev_bf16(oracle.f32_to_bf16_bits((rng.standard_normal(((Hq + 2 * Hkv) * D, hidden)) / 32).astype(np.float32))),
+          to_dev_bf16(oracle.f32_to_bf16_bits((rng.standard_normal((hidden, Hq * D)) / 45).astype(np.float32)))) for _ in range(2)]
+    x = to_dev_bf16(oracle.f32_to_bf16_bits(rng.standard_normal((Bn, hidden)).astype(np.float32)))
+    maxp = max(c[1].shape[1] for c in cases)
+    tabs = []
+    for c in cases:
+        t = np.full((Bn, maxp), -1, np.int32)
+        t[:, :c[1].shape[1]] = c[1]
+        tabs.append(torch.from_numpy(t).cuda())
+    results = []
+    for use_plan in (False, True):
+        pools = [to_dev_bf16(c[0]) for c in cases]
+        stage = B.Stage(pools=pools, layer_window=[0, 0], num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, max_batch=Bn,
+                        max_pages_per_seq=maxp)
+        mods = [B.AfdModule(stage, l, w[l][0], w[l][1], THETA, flags) for l in range(2)]
+        pos = torch.tensor(lens, dtype=torch.int32, device="cuda")
+        ys = [torch.zeros(Bn, hidden, dtype=torch.bfloat16, device="cuda") for _ in range(2)]
+        outs = []
+        if use_plan:
+            ops = [dict(kind="afd_module", module=mods[l].handle, batch=Bn, x=(x if l == 0 else ys[0]).data_ptr(),
+                        positions=pos.data_ptr(), page_table=tabs[l].data_ptr(), y=ys[l].data_ptr()) for l in range(2)]
+            plan = B.opw_attn_plan_create_mixed(stage.handle, ops, plan_flags)
+        for _ in range(steps):
+            if use_plan:
+                B.opw_attn_plan_submit(plan, torch.cuda.current_stream().cuda_stream)
+                if not plan_flags & B.OPW_PLAN_ADVANCE:
+                    pos.add_(1)
+            else:
+                mods[0].step(x, pos, tabs[0], ys[0])
+                mods[1].step(ys[0], pos, tabs[1], ys[1])      # layer 1 reads layer 0's output
+                pos.add_(1)
+            torch.cuda.synchronize()
+            outs.append(tobits(ys[1]).copy())
+        assert stage.poll_error() == B.OPW_OK and all(m.poll_error() == B.OPW_OK for m in mods)
+        assert pos.cpu().tolist() == [n + steps for n in lens]
+        results.append((outs, [tobits(p).copy() for p in pools]))
+        if use_plan:
+            B.opw_attn_plan_destroy(plan)
+        for m in mods:
+            m.close()
+        stage.close()
+    for a, b in zip(results[0][0], results[1][0]):
+        assert (a == b).all()
+    for a, b in zip(results[0][1], results[1][1]):
+        assert (a == b).all()
+    assert np.isfinite(oracle.bf16_bits_to_f64(results[1][0][-1])).all() and results[1][0][-1].any()
