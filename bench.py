@@ -26,6 +26,13 @@ import sys
 import threading
 import time
 
+# torchrun gives every rank one OpenMP thread unless the variable is set, which suits N ranks sharing the
+# host; the reference arm runs the CPU oracle on rank 0 alone (the other ranks exit), so it gets the cores
+# this process may use.  Set before anything loads an OpenMP runtime.
+if ("reference" in sys.argv and "TORCHELASTIC_RUN_ID" in os.environ and os.environ.get("OMP_NUM_THREADS") == "1"
+        and hasattr(os, "sched_getaffinity")):
+    os.environ["OMP_NUM_THREADS"] = str(len(os.sched_getaffinity(0)))
+
 import numpy as np
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
