@@ -413,10 +413,16 @@ static opw_status_t launch_combine(opw_attn_stage_t* st, const StepArgs& a, int 
   if (splits > kCombineScratchSlots / rows) splits = kCombineScratchSlots / rows;
   if (splits < 1) splits = 1;
   const bool pdl = (st->cfg.flags & OPW_FLAG_PDL) != 0 && !side_stream;
-  cudaError_t e = small ? launch(opw::combine_kernel<opw::kCombineThreadsSmall>, dim3(rows, splits),
-                                 dim3(opw::kCombineThreadsSmall), 0, stream, pdl, c)
-                        : launch(opw::combine_kernel<opw::kCombineThreads>, dim3(rows, splits),
-                                 dim3(opw::kCombineThreads), 0, stream, pdl, c);
+  const dim3 grid(rows, splits);
+  cudaError_t e;
+#define OPW_LAUNCH_COMBINE(DIM)                                                                                            \
+  e = small ? launch(opw::combine_kernel<opw::kCombineThreadsSmall, DIM>, grid, dim3(opw::kCombineThreadsSmall), 0, stream, \
+                     pdl, c)                                                                                               \
+            : launch(opw::combine_kernel<opw::kCombineThreads, DIM>, grid, dim3(opw::kCombineThreads), 0, stream, pdl, c)
+  if (D == 64) OPW_LAUNCH_COMBINE(64);
+  else if (D == 128) OPW_LAUNCH_COMBINE(128);
+  else OPW_LAUNCH_COMBINE(256);
+#undef OPW_LAUNCH_COMBINE
   if (e != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
   st->launches += 1;
   return OPW_OK;

@@ -873,13 +873,15 @@ __device__ __forceinline__ void combine_accumulate(float* acc, const float* part
 // block (row, y) merges every splits-th batch of the row's partials into one intermediate
 // partial in `scratch`, and the block that finishes last for the row (an atomic counter,
 // nothing waits) merges those `splits` intermediates and writes the output.
-template <int kCT>
-__global__ void __launch_bounds__(kCT) combine_kernel(CombineParams p) {
+// kD: the head dimension as a compile-time constant (0: read it from the parameters); the kernel is
+// bound by integer arithmetic more than by memory, and divisions by D are a good part of it.
+template <int kCT, int kD = 0>
+__global__ void __launch_bounds__(kCT, kCT == 128 ? 6 : 2) combine_kernel(CombineParams p) {
   pdl_launch_dependents();
   const int row = blockIdx.x;
   const int splits = gridDim.y, split = blockIdx.y;
   const int b = row / p.Hkv, g = row - b * p.Hkv;
-  const int D = p.D, G = p.G;
+  const int D = kD ? kD : p.D, G = p.G;
   const int GD = G * D;
   int32_t n = visible_keys(p.kv_lens, p.positions, b);   // an input: may be read before the attention kernel is done
   pdl_wait();                                  // partials, prefix sums and complete rows are final now
