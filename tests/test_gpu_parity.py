@@ -748,3 +748,25 @@ def test_head_dim_64_at_scale_default_twelve_warps():
     out, lse, rc, _ = gpu_attention(pool, tab, q, lens, 32, 8, 64)
     assert rc == B.OPW_OK
     check_close(out_to_f64(out), ref, lse, ref_lse)
+
+
+@pytest.mark.parametrize("lens,Hq,Hkv,D,window", [([1_000_000, 5], 32, 8, 128, 0), ([1_048_576], 16, 2, 256, 0),
+                                                   ([700_001, 33, 1], 8, 8, 64, 100_000)])
+def test_million_token_contexts(lens, Hq, Hkv, D, window):
+    """One sequence of about a million keys (65536 pages, thousands of partials for one row, the
+    two-level combine) beside tiny ones: the fused step against the oracle on the whole output."""
+    wl = synth.Workload("long", len(lens), Hq, Hkv, D, [window], "const_1", 99)
+    inp = synth.make_inputs(wl, device="cuda", growth=2, steps=1, lengths=np.array(lens, np.int32))
+    st = B.Stage(pools=inp.pools, layer_window=[window], num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, max_batch=len(lens),
+                 max_pages_per_seq=inp.max_pages_per_seq)
+    out = torch.empty(len(lens), Hq, D, dtype=torch.bfloat16, device="cuda")
+    lse = torch.empty(len(lens), Hq, dtype=torch.float32, device="cuda")
+    pos = torch.tensor(lens, dtype=torch.int32, device="cuda")
+    q = inp.q[0, 0]
+    st.decode_step(0, q, inp.k_new[0, 0], inp.v_new[0, 0], pos, inp.page_tables[0], out, lse)
+    assert st.poll_error() == B.OPW_OK
+    ref, ref_lse, rc = oracle.decode_attention(oracle.as_u16(inp.pools[0].cpu()), Hq, Hkv, D, P, oracle.as_u16(q.cpu()),
+                                               np.array(lens, np.int32) + 1, inp.page_tables[0].cpu().numpy(), window=window)
+    assert rc == 0
+    check_close(out_to_f64(out), ref, lse.cpu().numpy().astype(np.float64), ref_lse)
+    st.close()
