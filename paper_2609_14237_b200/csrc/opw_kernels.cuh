@@ -904,11 +904,14 @@ __global__ void __launch_bounds__(kCT, kCT == 128 ? 6 : 2) combine_kernel(Combin
   const int64_t uend = ustart + cnt;
   const int64_t wf = worker_of(U, ustart, p.num_workers), wl = worker_of(U, uend - 1, p.num_workers);
   const int64_t stride = (int64_t)G * (D + 2);
+  // segments a share really has in this launch (1 + the number of ticketed chunks, which depends on the
+  // share length only): small launches have fewer than kSegPerShare, and fewer candidates to test
+  const int segs = dyn_chunks(U, p.num_workers) + 1;
   // If the segment that holds the row's first unit also holds its last, that segment's worker
   // has already stored the final result: nothing to merge (every block of the row sees this).
   {
     bool whole = false;
-    if (threadIdx.x < kSegPerShare) {
+    if (threadIdx.x < segs) {
       int64_t a, bnd;
       segment_bounds(U, p.num_workers, wf, (int)threadIdx.x, a, bnd);
       whole = a <= ustart && ustart < bnd && bnd >= uend;
@@ -938,7 +941,7 @@ __global__ void __launch_bounds__(kCT, kCT == 128 ? 6 : 2) combine_kernel(Combin
   // that (tiny launches: most shares are empty), by unit: the share holding unit ustart + j,
   // counted once, at its first unit inside the row.
   const bool by_unit = (wl - wf + 1) > (int64_t)cnt;
-  const int64_t ncand = (by_unit ? (int64_t)cnt : (wl - wf + 1)) * kSegPerShare;
+  const int64_t ncand = (by_unit ? (int64_t)cnt : (wl - wf + 1)) * segs;
 
   // One merge pass over `nseg` listed partials at `base_ptr` (slot stride `stride`): stage
   // (m, l), weights per head, then the weighted sums.
@@ -985,8 +988,8 @@ __global__ void __launch_bounds__(kCT, kCT == 128 ? 6 : 2) combine_kernel(Combin
     bool hit = false;
     int32_t slot = 0;
     if (threadIdx.x < kCombineBatch && i < ncand) {
-      const int64_t j = i / kSegPerShare;
-      const int k = (int)(i % kSegPerShare);
+      const int64_t j = i / segs;
+      const int k = (int)(i - j * segs);
       int64_t w;
       bool counted = true;
       if (by_unit) {
