@@ -406,9 +406,10 @@ static opw_status_t launch_combine(opw_attn_stage_t* st, const StepArgs& a, int 
   c.scratch = reinterpret_cast<float*>(st->ws + st->lay.comb_scratch);
   c.row_count = reinterpret_cast<int32_t*>(st->ws + st->lay.row_count);
   // Few rows can have very many partials each (long contexts at small batch): split each row's
-  // merge over several blocks so that about two blocks per SM are busy.
+  // merge over several blocks so that about one block per SM is busy (two per SM measured slower:
+  // the hand-off between a row's blocks costs more than the extra parallelism gives).
   const int rows = a.batch * Hkv;
-  int splits = (2 * st->sms) / rows;
+  int splits = st->sms / rows;
   if (splits > opw::kCombineBatch) splits = opw::kCombineBatch;
   if (splits > kCombineScratchSlots / rows) splits = kCombineScratchSlots / rows;
   if (splits < 1) splits = 1;
