@@ -11,8 +11,11 @@ The rotary convention (rotate-half: the pair (x_i, x_{i+D/2}) turns by position 
 is a declared reading, so parity against the paper is UNPINNED for it; it is pinned to its own
 mathematics instead (tests/test_afd_oracle.py): position 0 is the identity, norms are preserved,
 <rope(q, m), rope(k, n)> depends on m - n only, and a plain-Python restatement.
-Values that cross the stage's bf16 interfaces (q, k, v, the attention output) are rounded to
-bf16 at the same points as on the GPU, so that rounding is not counted as error twice.
+The only roundings are at the module's declared bf16 interfaces: q, k_new and v_new as they are
+handed to core attention and stored in the cache (the activation interface of Appendix B.3:
+tensors of a stated shape and byte size cross between operators), and the attention output handed
+to the output projection.  Everything between two interfaces is fp64: the projection is not
+rounded before the rotation, and y is returned unrounded.
 """
 from __future__ import annotations
 
@@ -43,12 +46,12 @@ def rope(x: np.ndarray, positions, theta: float) -> np.ndarray:
 def project_qkv(x, w_qkv, positions, Hq, Hkv, D, theta):
     """Returns bf16-rounded (q [B,Hq,D], k [B,Hkv,D], v [B,Hkv,D]) as float64 arrays."""
     B = x.shape[0]
-    qkv = round_bf16(x @ w_qkv.T)                              # the GEMM's bf16 output
+    qkv = x @ w_qkv.T                                          # fp64, not rounded: no interface here
     q = qkv[:, :Hq * D].reshape(B, Hq, D)
     k = qkv[:, Hq * D:(Hq + Hkv) * D].reshape(B, Hkv, D)
     v = qkv[:, (Hq + Hkv) * D:].reshape(B, Hkv, D)
     pos = np.maximum(np.asarray(positions), 0)
-    return round_bf16(rope(q, pos, theta)), round_bf16(rope(k, pos, theta)), v
+    return round_bf16(rope(q, pos, theta)), round_bf16(rope(k, pos, theta)), round_bf16(v)
 
 
 def module_step(pool, x, w_qkv, w_o, positions, page_table, Hq, Hkv, D, theta, window=0, P=16):

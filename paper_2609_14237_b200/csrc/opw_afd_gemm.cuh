@@ -17,10 +17,10 @@
 // partial tile to a workspace and the last to arrive (an atomic ticket per tile) adds them in
 // split order -- deterministic -- and runs the epilogue.
 //
-// Epilogues: plain (bf16 C[b, n]) and rotary (the QKV projection of the attention module: the
-// result is rounded to bf16 as a library GEMM would, pairs (d, d + D/2) of the q and k heads
-// are rotated by angles that the warps idle in the main loop compute meanwhile, v is passed
-// through, and the three outputs go to separate [batch, heads, D] buffers).  The rotary form needs both elements of a pair in one
+// Epilogues: plain (bf16 C[b, n]) and rotary (the QKV projection of the attention module: pairs
+// (d, d + D/2) of the q and k heads are rotated, still as fp32 accumulators, by angles that the
+// warps idle in the main loop compute meanwhile, v is passed through, everything is rounded to
+// bf16 once, and the three outputs go to separate [batch, heads, D] buffers).  The rotary form needs both elements of a pair in one
 // 128-row tile: D in {64, 128}.
 //
 // Every wait is bounded by the global timer (kGemmWaitNs); a wait that runs out records
@@ -156,8 +156,6 @@ __device__ __forceinline__ uint64_t g_smem_desc(uint32_t smem_addr) {
 __device__ __forceinline__ uint32_t g_instr_desc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
 }
-
-__device__ __forceinline__ float g_round_bf16(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
 
 // grid = (ceil(n_out / 128), ksplit), 512 threads, 1 CTA per SM.
 // Dynamic shared memory: 1024 (alignment slack) + stages * (16384 + nb * 128) bytes, then in mode 1
@@ -398,12 +396,8 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     } else {
       for (int b = tid >> 6; b < p.batch; b += kColPhases) {
         float2 v = *reinterpret_cast<const float2*>(&stage_f[b * kTileM + r0]);
-        v.x = g_round_bf16(v.x);                 // the projection's own bf16 output, as a library GEMM rounds it
-        v.y = g_round_bf16(v.y);
-        if (rotate) {
-          float2 w = *reinterpret_cast<const float2*>(&stage_f[b * kTileM + pr]);
-          w.x = g_round_bf16(w.x);
-          w.y = g_round_bf16(w.y);
+        if (rotate) {                            // on the fp32 accumulators: one rounding, at the bf16 output
+          const float2 w = *reinterpret_cast<const float2*>(&stage_f[b * kTileM + pr]);
           const float4 cs = angles4[(b * half + i0) >> 1];
           v = make_float2(v.x * cs.x + sgn * (w.x * cs.y), v.y * cs.z + sgn * (w.y * cs.w));
         }

@@ -8,6 +8,7 @@
 #include <cmath>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -108,6 +109,35 @@ int query_sms(int device) {
   return sms;
 }
 
+// The dynamic shared-memory limit is an attribute of a kernel on a device, not of a stage, and
+// several stages of different sizes may be alive on one device: it is only ever raised.  The
+// largest value set so far is kept per device and head size (both instances of a head size get
+// the same value).
+constexpr int kMaxDevices = 64;
+std::mutex g_smem_mutex;
+int g_smem_set[kMaxDevices][3];
+
+cudaError_t raise_smem_limit(int device, int D, int bytes) {
+  if (device < 0 || device >= kMaxDevices) return cudaErrorInvalidDevice;
+  const int slot = D == 64 ? 0 : D == 128 ? 1 : 2;
+  std::lock_guard<std::mutex> lock(g_smem_mutex);
+  if (bytes <= g_smem_set[device][slot]) return cudaSuccess;
+  cudaError_t e;
+  if (D == 64) {
+    e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  } else if (D == 128) {
+    e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  } else {
+    e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+  }
+  if (e == cudaSuccess) g_smem_set[device][slot] = bytes;
+  return e;
+}
+
 }  // namespace
 
 struct opw_attn_stage {
@@ -192,19 +222,7 @@ opw_status_t opw_attn_stage_create(const opw_attn_stage_config_t* cfg, opw_attn_
   const Layout lay = carve(cfg, s, sms);
   if (cfg->workspace_bytes < lay.total) return OPW_ERR_CAPACITY;
 
-  cudaError_t e = cudaSuccess;
-  const int smem_i = (int)smem;
-  if (cfg->head_dim == 64) {
-    e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_i);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_i);
-  } else if (cfg->head_dim == 128) {
-    e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_i);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_i);
-  } else {
-    e = cudaFuncSetAttribute(opw::attn_splitkv_kernel<256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_i);
-  }
+  cudaError_t e = raise_smem_limit(cfg->device, cfg->head_dim, (int)smem);
   if (e != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
   {
     // Registers decide how many warps a block may have (eight at head_dim 128, twelve at 64): ask the
@@ -595,10 +613,11 @@ namespace {
 opw_status_t enqueue_plan_overlapped(opw_attn_plan* pl, cudaStream_t stream, cudaStream_t side) {
   opw_attn_stage* st = pl->stage;
   const int n = (int)pl->items.size();
-  int last = -1;
+  int last = -1, live = 0;
+  int last_in_set[2] = {-1, -1};              // the item whose combine last used each workspace set
   for (int i = 0; i < n; ++i) {
     const opw_step_item_t& it = pl->items[i];
-    if (it.batch == 0) continue;
+    if (it.batch == 0) continue;              // nothing is enqueued or recorded for an empty item
     const bool fused = it.k_new && !it.kv_lens;
     if (it.k_new && !fused) {
       opw_status_t rc = opw_kv_append(st, it.layer, it.batch, it.k_new, it.v_new, it.positions, it.page_table, stream);
@@ -606,8 +625,9 @@ opw_status_t enqueue_plan_overlapped(opw_attn_plan* pl, cudaStream_t stream, cud
     }
     const StepArgs a = {it.layer, it.batch, it.q, fused ? nullptr : it.kv_lens, fused ? it.k_new : nullptr,
                         fused ? it.v_new : nullptr, fused ? it.positions : nullptr, it.page_table, it.out, it.lse};
-    const int set = i & 1;
-    if (i >= 2 && cudaStreamWaitEvent(stream, pl->ev_comb[i - 2], 0) != cudaSuccess) return OPW_ERR_CUDA;
+    const int set = live & 1;
+    if (last_in_set[set] >= 0 && cudaStreamWaitEvent(stream, pl->ev_comb[last_in_set[set]], 0) != cudaSuccess)
+      return OPW_ERR_CUDA;
     opw_status_t rc = launch_attention(st, a, set, stream);
     if (rc != OPW_OK) return rc;
     if (cudaEventRecord(pl->ev_attn[i], stream) != cudaSuccess || cudaStreamWaitEvent(side, pl->ev_attn[i], 0) != cudaSuccess)
@@ -615,6 +635,8 @@ opw_status_t enqueue_plan_overlapped(opw_attn_plan* pl, cudaStream_t stream, cud
     rc = launch_combine(st, a, set, side, true, true);
     if (rc != OPW_OK) return rc;
     if (cudaEventRecord(pl->ev_comb[i], side) != cudaSuccess) return OPW_ERR_CUDA;
+    last_in_set[set] = i;
+    ++live;
     last = i;
   }
   if (last >= 0 && cudaStreamWaitEvent(stream, pl->ev_comb[last], 0) != cudaSuccess) return OPW_ERR_CUDA;
@@ -711,9 +733,14 @@ static opw_status_t build_plan(opw_attn_stage_t* st, const opw_step_item_t* item
   }
   if (flags & OPW_PLAN_OVERLAP) {
     // a step's combine runs beside the next step's attention: they must not share outputs
-    for (int i = 0; i + 1 < n_items; ++i)
-      if (items[i].out == items[i + 1].out || (items[i].lse && items[i].lse == items[i + 1].lse))
+    // (consecutive among the items that launch anything: empty items are skipped)
+    int prev = -1;
+    for (int i = 0; i < n_items; ++i) {
+      if (items[i].batch == 0) continue;
+      if (prev >= 0 && (items[prev].out == items[i].out || (items[prev].lse && items[prev].lse == items[i].lse)))
         return OPW_ERR_INVALID_ARG;
+      prev = i;
+    }
   }
   opw_attn_plan* pl = new (std::nothrow) opw_attn_plan();
   if (!pl) return OPW_ERR_INVALID_ARG;

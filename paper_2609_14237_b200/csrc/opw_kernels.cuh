@@ -403,7 +403,14 @@ __global__ void __maxnreg__(D > 128 ? 255 : 200) attn_splitkv_kernel(AttnParams 
   const int64_t U = (int64_t)cum[p.batch] * p.Hkv;
   const int64_t num_workers = (int64_t)gridDim.x * warps;
   const int64_t worker = (int64_t)blockIdx.x * warps + warp;
-  if (U == 0) return;
+  if (U == 0) {
+    // Nothing to stream, but the grid must still pass the dependency wait before it completes: under
+    // programmatic stream serialisation a grid that exits without waiting lets its successor's wait
+    // return while the predecessor of this grid is still running (ordering would not be transitive).
+    pdl_wait();
+    if (blockIdx.x == 0 && threadIdx.x == 0) p.cum[p.batch] = 0;
+    return;
+  }
   uint64_t* tr = p.trace ? p.trace + worker * 4 : nullptr;
   if (tr && lane == 0) tr[1] = global_timer_ns();
 

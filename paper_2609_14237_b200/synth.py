@@ -1,10 +1,11 @@
 """Seeded synthetic inputs for the decode attention stage.
 
 This module is shared by the tests (which feed the same tensors to the CPU oracle and
-to the CUDA path) and by the benchmark.  It contains no attention arithmetic and no
-knowledge of the KV-pool layout: pools are filled with independent N(0,1) bf16 values,
-which is the same distribution under any layout, and page tables are seeded random
-permutations of the physical pages dealt to the sequences.
+to the CUDA path) and by the benchmark.  It contains no attention arithmetic and does not
+know where an element sits inside a pool (only how many elements a page has): pools are
+filled with independent N(0,1) bf16 values, which is the same distribution under any
+layout, and page tables are seeded random permutations of the physical pages dealt to the
+sequences.
 
 The five named workloads stand in for the paper's decode workloads (Section 7.1:
 context-length cohorts derived from a public reasoning dataset and rescaled to 8K /
@@ -57,6 +58,9 @@ WORKLOADS = {
     "c5_hybrid_stack": Workload(
         "c5_hybrid_stack", 128, 32, 8, 128, [4096, 4096, 4096, 0, 4096, 4096, 4096, 0],
         "uniform_8192_65536", 1005),
+    # one sliding-window layer of the hybrid stack on its own (same shape, lengths and seed): 2.15 GB of
+    # mapped pages, small enough to profile where the whole 52 GB stack is not
+    "c5_window_layer": Workload("c5_window_layer", 128, 32, 8, 128, [4096], "uniform_8192_65536", 1005),
     # not one of the five benchmark configurations: a stack shaped like the paper's first evaluated
     # model (sliding-window : full = 5 : 1, 32 query / 16 KV heads of 128; the window, 1024, is an
     # assumption -- the paper prints only the ratio), batch 64, contexts U[8192, 32768]

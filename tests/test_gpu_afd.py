@@ -1,22 +1,36 @@
 """GPU parity of the complete attention module (projections + rotary encoding + core attention)
 against its fp64 oracle, through the C ABI.
 
-The module is checked stage by stage, each stage fed with the GPU's own previous result so that a
-one-ulp rounding flip upstream is not counted again downstream, and once end to end:
-  q, k, v   : both sides round the GEMM result to bf16, rotate, and round again; fp32 against fp64
-              accumulation can flip either rounding by one ulp (<= 2^-7 relative).  A flipped input
-              pair (x0, x1) moves the rotated value by <= 2^-7 (|x0| + |x1|) <= 2^-7 sqrt(2) (|ref| +
-              |partner|), partner being the other element of the rotated pair, and the second flip adds
-              2^-7 |ref|: |err| <= 2.5 * 2^-7 * (|ref| + |partner|).
-              v is not rotated: |err| <= 2^-7 |ref| (one flip).
-              Near zero the fp32 accumulation itself shows: tensor-core accumulators may truncate, so
-              its error can grow linearly, hidden * 2^-24 * rms -- added to all three bounds.
-  append    : the pool afterwards holds the GPU's k, v rows bit for bit
-  attention : the stated core-attention tolerance, oracle run on the GPU's q and that pool
-  y         : a K-term fp32 dot product rounded to bf16: |err| <= 2^-8 |ref| + 2^-10 * rms(y)
-  end to end: independent roundings of relative size 2^-9 (attention output, probabilities, q/k/v)
-              pass through a projection that averages them: max |err| <= 2^-5 rms(y) + 2^-8 |ref|,
-              mean |err| <= 2^-7 rms(y)
+The oracle rounds only at the module's bf16 interfaces (q, k_new, v_new, the attention output); it
+knows nothing of where a kernel rounds inside.  The module is checked stage by stage, each stage fed
+with the GPU's own previous result so that a rounding flip upstream is not counted again downstream,
+and once end to end.  Every bound below is a sum of terms, each with its reason:
+
+  u = 2^-8 : largest relative error of one round-to-nearest bf16 rounding (8 significant bits).
+  E = hidden * 2^-24 * rms(v) : allowance for the fp32 accumulation of a `hidden`-term dot product
+      (products of two bf16 values are exact in fp32; each of the `hidden` additions may lose up to
+      2^-24 of a running sum whose size is of the order of the result's rms; tensor-core adders may
+      truncate, so the losses can add up linearly instead of cancelling).
+  partner : the other element of a rotated pair (i, i + D/2); a rotation mixes the two, so an error
+      of the pair's inputs shows in proportion to |ref| + |partner|, not to |ref| alone.
+
+  v   (both paths) : one rounding on each side of values that differ by <= E:
+                     |err| <= 2u |ref| + E.
+  q,k (tensor-core path: the fp32 accumulators are rotated, then rounded once):
+                     inputs differ by <= E each, |cos|, |sin| <= 1, the fp32 rotation itself loses
+                     <= 2^-22 (|ref| + |partner|), then one rounding on each side:
+                     |err| <= 2u |ref| + 2E + 2^-22 (|ref| + |partner|).
+  q,k (library path: the library GEMM stores bf16, a second kernel rotates and rounds again):
+                     the extra rounding moves each input by <= u |x|, which the rotation turns into
+                     <= u (|x0||cos| + |x1||sin|) <= u (|ref| + |partner|) (a rotation keeps the pair's norm):
+                     |err| <= 2u |ref| + u (|ref| + |partner|) + 2E + 2^-22 (|ref| + |partner|).
+  append    : the pool afterwards holds the GPU's k, v rows bit for bit.
+  attention : the stated core-attention tolerance, oracle run on the GPU's q and that pool.
+  y         : a K-term fp32 dot product of exactly known inputs rounded to bf16 once:
+              |err| <= u |ref| + 2^-10 rms(y)   (K * 2^-24 <= 2^-10 up to K = 16384).
+  end to end: the interface roundings (q, k, v, attention output; relative size <= u each, independent)
+              and the probabilities' bf16 rounding pass through a projection that averages them
+              over Hq*D terms: max |err| <= 2^-5 rms(y) + u |ref|, mean |err| <= 2^-7 rms(y).
 """
 import numpy as np
 import pytest
@@ -83,16 +97,21 @@ def run_module(seed, lens, Hq, Hkv, D, hidden, steps=2, inactive=(), window=0, b
         gq, gk, gv, gattn = mod.intermediates(nb)
         act = pos >= 0
 
-        # q, k, v against the oracle's projections
+        # q, k, v against the oracle's projections (bounds: see the module docstring)
         rq, rk, rv = afd.project_qkv(x, w_qkv, pos, Hq, Hkv, D, THETA)
-        acc = hidden * 2.0 ** -24 * float(np.sqrt(np.mean(rv[act] ** 2))) + 1e-6
+        u = 2.0 ** -8
+        E = hidden * 2.0 ** -24 * float(np.sqrt(np.mean(rv[act] ** 2))) + 1e-30
+        library = bool(flags & B.OPW_AFD_LIBRARY_GEMM) or nb > 96 or D == 256     # what the module switches to the library for
+        pre = u if library else 0.0                          # the library path's extra rounding before the rotation
         for name, got, ref in (("q", f64(gq), rq), ("k", f64(gk), rk)):
             partner = np.concatenate([ref[..., D // 2:], ref[..., :D // 2]], axis=-1)
+            pair = np.abs(ref) + np.abs(partner)
             err = np.abs(got - ref)[act]
-            assert (err <= 2.5 * 2.0 ** -7 * (np.abs(ref) + np.abs(partner))[act] + 2 * acc).all(), (name, err.max())
+            bound = 2 * u * np.abs(ref) + (pre + 2.0 ** -22) * pair + 2 * E
+            assert (err <= bound[act]).all(), (name, float((err - bound[act]).max()))
             worst[name] = max(worst.get(name, 0.0), float(err.max()))
         verr = np.abs(f64(gv) - rv)[act]
-        assert (verr <= 2.0 ** -7 * np.abs(rv)[act] + acc).all(), float((verr - 2.0 ** -7 * np.abs(rv)[act]).max())
+        assert (verr <= 2 * u * np.abs(rv)[act] + E).all(), float((verr - 2 * u * np.abs(rv)[act]).max())
 
         # append: exactly the GPU's k, v rows, nothing else changed
         expect = before.copy()
@@ -165,9 +184,10 @@ def test_batches_of_one_row_and_around_the_switch_to_the_library_path():
 
 
 def test_the_two_projection_paths_agree():
-    """Same inputs through the tensor-core kernel and through the library path: both round the
-    projection to bf16 before rotating, so q, k, v differ only where fp32 summation order flips a
-    rounding (<= 1 % of the elements, each by one bf16 ulp)."""
+    """Same inputs through the tensor-core kernel (rotates the fp32 accumulators, rounds once) and
+    through the library path (rounds the projection, rotates, rounds again): v agrees except where the
+    summation order flips a rounding; q and k differ by the library path's extra rounding, at most
+    u (|ref| + |partner|) before the last rounding (see the module docstring)."""
     outs = []
     for flags in (0, B.OPW_AFD_LIBRARY_GEMM):
         rng = np.random.default_rng(41)
@@ -188,12 +208,12 @@ def test_the_two_projection_paths_agree():
         assert mod.launch_count() == (2 if flags == 0 else 1)
         mod.close()
         stage.close()
+    u = 2.0 ** -8
     for n, (a, b) in enumerate(zip(outs[0][:3], outs[1][:3])):
-        diff = a != b
-        assert diff.mean() <= 0.01, diff.mean()
-        # a flipped input moves a rotated value by an ulp of the pair, not of the value itself
+        if n == 2:
+            assert (a != b).mean() <= 0.01                # v: the same single rounding on both paths
         partner = np.concatenate([b[..., 64:], b[..., :64]], axis=-1) if n < 2 else 0.0
-        assert (np.abs(a - b) <= 2.5 * 2.0 ** -7 * (np.abs(b) + np.abs(partner)) + 1e-30).all()
+        assert (np.abs(a - b) <= 2 * u * np.abs(b) + u * (np.abs(b) + np.abs(partner)) + 1e-6).all()
     rms = float(np.sqrt(np.mean(outs[1][3] ** 2)))
     assert np.abs(outs[0][3] - outs[1][3]).max() <= 2.0 ** -5 * rms
 

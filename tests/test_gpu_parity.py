@@ -9,16 +9,11 @@ import pytest
 import torch
 
 import oracle
-from helpers import P, bits, make_case, rand_bits
+from helpers import MAX_ABS, P, bits, check_close, make_case, out_to_f64, rand_bits
 from paper_2609_14237_b200 import binding as B
 from paper_2609_14237_b200 import synth
 
 pytestmark = pytest.mark.gpu
-
-MAX_ABS, MEAN_ABS = 1e-2, 1e-3          # the stated tolerance
-REL_RMS = 2.0 ** -6                     # max |err| / rms(out): catches dropped chunks on long contexts
-LSE_TOL = 2e-3
-
 
 @pytest.fixture(scope="module", autouse=True)
 def built():
@@ -31,30 +26,6 @@ def dev(a, dtype=None):
     if dtype is torch.bfloat16:
         t = t.view(torch.int16).view(torch.bfloat16)
     return t.cuda()
-
-
-def out_to_f64(t):
-    return oracle.bf16_bits_to_f64(t.cpu().view(torch.int16).numpy().view(np.uint16))
-
-
-def check_close(got, ref, lse_got=None, lse_ref=None, rows=None, max_abs=MAX_ABS):
-    if rows is not None:
-        got, ref = got[rows], ref[rows]
-        if lse_got is not None:
-            lse_got, lse_ref = lse_got[rows], lse_ref[rows]
-    err = np.abs(got - ref)
-    rms = float(np.sqrt(np.mean(ref ** 2)))
-    assert np.isfinite(got).all()
-    assert err.max() <= max_abs, err.max()
-    assert err.mean() <= MEAN_ABS, err.mean()
-    # per (sequence, head) relative check: error against that row's own rms (+ bf16 half-ulp slack)
-    row_rms = np.sqrt(np.mean(ref ** 2, axis=-1, keepdims=True))
-    assert (err <= REL_RMS * row_rms + 2.0 ** -8 * np.abs(ref) + 1e-6).all(), float((err / (row_rms + 1e-30)).max())
-    if lse_got is not None:
-        fin = np.isfinite(lse_ref)
-        assert (np.isneginf(lse_got) == np.isneginf(lse_ref)).all()
-        assert np.abs(lse_got[fin] - lse_ref[fin]).max() <= LSE_TOL
-    return float(err.max()), float(err.mean()), rms
 
 
 def gpu_attention(pool_np, tab, q_bits, lens, Hq, Hkv, D, window=0, scale=0.0, want_lse=True, **tune):
@@ -236,6 +207,82 @@ def test_programmatic_dependent_launch_keeps_back_to_back_steps_ordered(fused):
     for layer in range(2):
         assert (pools[layer].cpu().view(torch.int16).numpy().view(np.uint16) == refs[layer]).all()
     st.close()
+
+
+@pytest.mark.parametrize("fused", [True, False])
+def test_programmatic_dependent_launch_with_an_all_inactive_step_between_two_live_ones(fused):
+    """A grid with nothing to do must still pass its dependency wait before it completes, or the kernels
+    behind it could overtake the step in front of it: live step, all-inactive step, live step, enqueued
+    back to back on one stream with OPW_FLAG_PDL, repeated over two layers; every output and the whole
+    pool against the oracle."""
+    wl = synth.Workload("pdl0", 8, 32, 8, 128, [0, 200], "uniform_1024_4096", 81)
+    inp = synth.make_inputs(wl, device="cpu", growth=3, steps=3)
+    pools = [p.cuda() for p in inp.pools]
+    refs = [oracle.as_u16(p).copy() for p in inp.pools]
+    st = B.Stage(pools=pools, layer_window=wl.layer_window, num_q_heads=32, num_kv_heads=8, head_dim=128,
+                 max_batch=8, max_pages_per_seq=inp.max_pages_per_seq, flags=B.OPW_FLAG_PDL)
+    tabs = [t.cuda() for t in inp.page_tables]
+    dq, dk, dv = inp.q.cuda(), inp.k_new.cuda(), inp.v_new.cuda()
+    # step 1 is the empty one: every slot inactive; the live steps are decode steps 0 and 1 of the sequences
+    pos_np = [inp.positions(0), np.full(8, -1, np.int32), inp.positions(1)]
+    len_np = [np.where(p >= 0, p + 1, 0).astype(np.int32) for p in pos_np]
+    pos, lens = [dev(p) for p in pos_np], [dev(n) for n in len_np]
+    outs = torch.full((3, 2, 8, 32, 128), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lses = torch.full((3, 2, 8, 32), float("nan"), dtype=torch.float32, device="cuda")
+    for rep in range(3):                                   # the same three steps enqueued three times over:
+        for step in range(3):                              # later repetitions rewrite the same slots with the same rows
+            for layer in range(2):
+                if fused:
+                    st.decode_step(layer, dq[step, layer], dk[step, layer], dv[step, layer], pos[step], tabs[layer],
+                                   outs[step, layer], lses[step, layer])
+                else:
+                    st.kv_append(layer, dk[step, layer], dv[step, layer], pos[step], tabs[layer])
+                    st.decode_attention(layer, dq[step, layer], lens[step], tabs[layer], outs[step, layer], lses[step, layer])
+    assert st.poll_error() == B.OPW_OK
+    for step in range(3):
+        for layer in range(2):
+            assert oracle.kv_append(refs[layer], 8, 128, P, inp.k_new[step, layer], inp.v_new[step, layer],
+                                    pos_np[step], inp.page_tables[layer]) == 0
+    for step in range(3):
+        for layer in range(2):
+            # (the live steps of every repetition saw the pool with both new rows already in place or being
+            # rewritten with identical bytes; attention reads only rows below its own length)
+            ref, ref_lse, _ = oracle.decode_attention(refs[layer], 32, 8, 128, P, inp.q[step, layer], len_np[step],
+                                                      inp.page_tables[layer], window=wl.layer_window[layer])
+            check_close(out_to_f64(outs[step, layer]), ref, lses[step, layer].cpu().numpy().astype(np.float64), ref_lse)
+    assert (out_to_f64(outs[1]) == 0).all() and np.isneginf(lses[1].cpu().numpy()).all()
+    for layer in range(2):
+        assert (pools[layer].cpu().view(torch.int16).numpy().view(np.uint16) == refs[layer]).all()
+    st.close()
+
+
+def test_a_smaller_stage_created_later_leaves_an_earlier_larger_stage_working():
+    """The kernels' shared-memory limit belongs to the device, not to a stage: creating a stage with a
+    small static batch after one with a large static batch must not lower it under the first one."""
+    rng = np.random.default_rng(67)
+    Hq, Hkv, D = 8, 2, 64
+    lens = rng.integers(1, 60, size=4096).astype(np.int32)
+    lens[::7] = 0
+    pool_np, tab, q, _, _ = make_case(rng, [max(int(n), 1) for n in lens], Hq, Hkv, D)
+    pool = dev(pool_np, torch.bfloat16)
+    big = B.Stage(pools=[pool], layer_window=[0], num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, max_batch=4096,
+                  max_pages_per_seq=tab.shape[1], tune_warps=12, tune_stages=4)
+    small = B.Stage(pools=[pool], layer_window=[0], num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, max_batch=2,
+                    max_pages_per_seq=tab.shape[1], tune_warps=2, tune_stages=2)
+    out = torch.full((4096, Hq, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((4096, Hq), float("nan"), dtype=torch.float32, device="cuda")
+    big.decode_attention(0, dev(q, torch.bfloat16), dev(lens), dev(tab), out, lse)     # raises OpwError if the launch is refused
+    assert big.poll_error() == B.OPW_OK
+    ref, ref_lse, rc = oracle.decode_attention(pool_np, Hq, Hkv, D, P, q, lens, tab)
+    assert rc == 0
+    check_close(out_to_f64(out), ref, lse.cpu().numpy().astype(np.float64), ref_lse,
+                max_abs=2.0 ** -8 * float(np.abs(ref).max()) + 1e-3)
+    out2 = torch.empty(2, Hq, D, dtype=torch.bfloat16, device="cuda")
+    small.decode_attention(0, dev(q[:2], torch.bfloat16), dev(lens[:2]), dev(tab[:2]), out2)
+    assert small.poll_error() == B.OPW_OK
+    check_close(out_to_f64(out2), ref[:2], max_abs=2.0 ** -8 * float(np.abs(ref).max()) + 1e-3)
+    small.close()
+    big.close()
 
 
 def test_single_key_returns_v_bit_exactly():
@@ -481,6 +528,39 @@ def test_plan_submits_a_multi_layer_multi_microbatch_step_in_one_call(flags, fus
     st.close()
 
 
+@pytest.mark.parametrize("flags", [B.OPW_PLAN_OVERLAP, B.OPW_PLAN_OVERLAP | B.OPW_PLAN_GRAPH])
+def test_overlapped_plan_with_an_empty_item_between_live_ones(flags):
+    """An item with batch 0 enqueues nothing and records no event; the items around it must still be
+    ordered through the workspace set they share (as a captured graph too)."""
+    wl = synth.Workload("pe", 4, 32, 8, 128, [0, 48, 0, 48], "uniform_1024_4096", 83)
+    inp = synth.make_inputs(wl, device="cpu", growth=1, steps=1, lengths=np.array([700, 33, 2500, 16], np.int32))
+    pools = [p.cuda() for p in inp.pools]
+    refs = [oracle.as_u16(p).copy() for p in inp.pools]
+    st = B.Stage(pools=pools, layer_window=wl.layer_window, num_q_heads=32, num_kv_heads=8, head_dim=128,
+                 max_batch=4, max_pages_per_seq=inp.max_pages_per_seq)
+    dq, dk, dv = inp.q.cuda(), inp.k_new.cuda(), inp.v_new.cuda()
+    pos = dev(inp.positions(0))
+    tabs = [t.cuda() for t in inp.page_tables]
+    outs = [torch.full((4, 32, 128), float("nan"), dtype=torch.bfloat16, device="cuda") for _ in range(4)]
+    items = []
+    for l in range(4):
+        items.append(dict(layer=l, batch=0 if l == 1 else 4, q=dq[0, l].data_ptr(), k_new=dk[0, l].data_ptr(),
+                          v_new=dv[0, l].data_ptr(), positions=pos.data_ptr(), page_table=tabs[l].data_ptr(),
+                          out=outs[l].data_ptr()))
+    plan = B.opw_attn_plan_create(st.handle, items, flags)
+    B.opw_attn_plan_submit(plan, torch.cuda.current_stream().cuda_stream)
+    assert st.poll_error() == B.OPW_OK
+    for l in (0, 2, 3):
+        assert oracle.kv_append(refs[l], 8, 128, P, inp.k_new[0, l], inp.v_new[0, l], inp.positions(0), inp.page_tables[l]) == 0
+        ref, _, _ = oracle.decode_attention(refs[l], 32, 8, 128, P, inp.q[0, l], inp.kv_lens(0), inp.page_tables[l],
+                                            window=wl.layer_window[l])
+        check_close(out_to_f64(outs[l]), ref)
+    for l in range(4):                                      # layer 1's pool is untouched
+        assert (pools[l].cpu().view(torch.int16).numpy().view(np.uint16) == refs[l]).all()
+    B.opw_attn_plan_destroy(plan)
+    st.close()
+
+
 def test_overlapped_plan_needs_distinct_outputs_for_consecutive_items():
     pool = torch.zeros(4 * 2 * 2 * 16 * 64, dtype=torch.bfloat16, device="cuda")
     st = B.Stage(pools=[pool], layer_window=[0], num_q_heads=8, num_kv_heads=2, head_dim=64, max_batch=2, max_pages_per_seq=2)
@@ -648,59 +728,81 @@ def compact_rows(pool, table, rows, Hkv, D):
     return oracle.as_u16(small.cpu()), new_tab.cpu().numpy()
 
 
-def run_full_config(name, sample, layers=None, tune=None, fused=True):
+def run_full_config(name, sample=None, sample_full=None, layers=None, tune=None, fused=True):
+    """One decode step of a benchmark configuration at full size, in the launch configuration bench.py
+    times, against the oracle.  sample=None compares every row of the batch; a number compares that many
+    seeded rows plus the shortest and the longest (sample_full: the same, for full-attention layers of a
+    stack whose window layers are compared whole)."""
     wl = synth.WORKLOADS[name]
     inp = synth.make_inputs(wl, device="cuda", growth=1, steps=1)
     st = B.Stage(pools=inp.pools, layer_window=wl.layer_window, num_q_heads=wl.num_q_heads, num_kv_heads=wl.num_kv_heads,
                  head_dim=wl.head_dim, max_batch=wl.batch, max_pages_per_seq=inp.max_pages_per_seq, **(tune or {}))
     pos, n = inp.positions(0), inp.kv_lens(0)
     order = np.argsort(n)
-    rows = sorted(set([int(order[0]), int(order[-1])] + [int(r) for r in np.random.default_rng(wl.seed).choice(wl.batch, size=min(sample, wl.batch), replace=False)]))
+
+    def pick(k):
+        if k is None or k >= wl.batch:
+            return list(range(wl.batch))
+        drawn = np.random.default_rng(wl.seed).choice(order[1:-1], size=k, replace=False)      # k rows besides the two extremes
+        return sorted([int(order[0]), int(order[-1])] + [int(r) for r in drawn])
+
     stats = []
     for layer in (layers if layers is not None else range(wl.num_layers)):
+        rows = pick(sample_full if (sample_full is not None and wl.layer_window[layer] == 0) else sample)
         tab = inp.page_tables[layer]
         q, k, v = inp.q[0, layer], inp.k_new[0, layer], inp.v_new[0, layer]
         small_before, small_tab = compact_rows(inp.pools[layer], tab, rows, wl.num_kv_heads, wl.head_dim)
-        out = torch.empty(wl.batch, wl.num_q_heads, wl.head_dim, dtype=torch.bfloat16, device="cuda")
-        lse = torch.empty(wl.batch, wl.num_q_heads, dtype=torch.float32, device="cuda")
+        out = torch.full((wl.batch, wl.num_q_heads, wl.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda")
+        lse = torch.full((wl.batch, wl.num_q_heads), float("nan"), dtype=torch.float32, device="cuda")
         if fused:                                   # the launch configuration bench.py times
             st.decode_step(layer, q, k, v, dev(pos), tab, out, lse)
         else:
             st.kv_append(layer, k, v, dev(pos), tab)
             st.decode_attention(layer, q, dev(n), tab, out, lse)
         assert st.poll_error() == B.OPW_OK
-        # append parity on the sampled rows' pages (bit-exact), then attention on the oracle's own pool
-        ref_pool = small_before.copy()
+        assert torch.isfinite(out.float()).all()    # every row was written, compared or not
+        # append parity on the compared rows' pages (bit-exact), then attention on the oracle's own pool
+        ref_pool = small_before
         assert oracle.kv_append(ref_pool, wl.num_kv_heads, wl.head_dim, P, k[rows].cpu(), v[rows].cpu(), pos[rows], small_tab) == 0
         small_after, _ = compact_rows(inp.pools[layer], tab, rows, wl.num_kv_heads, wl.head_dim)
-        assert (small_after == ref_pool).all()
+        assert np.array_equal(small_after, ref_pool)
+        del small_after
         ref, ref_lse, rc = oracle.decode_attention(ref_pool, wl.num_q_heads, wl.num_kv_heads, wl.head_dim, P, q[rows].cpu(),
                                                    n[rows], small_tab, window=wl.layer_window[layer])
         assert rc == 0
-        stats.append(check_close(out_to_f64(out[rows]), ref, lse[rows].cpu().numpy().astype(np.float64), ref_lse))
+        stats.append((layer, len(rows)) + check_close(out_to_f64(out[rows]), ref, lse[rows].cpu().numpy().astype(np.float64), ref_lse))
+        del ref_pool, small_before
     st.close()
     return stats
 
 
 @pytest.mark.parametrize("fused", [True, False])
-def test_config2_llama8b_shape_all_rows(fused):
-    run_full_config("c2_llama8b", sample=64, fused=fused)
-
-
-def test_config3_long_context_sampled_rows():
-    run_full_config("c3_long_context", sample=3)
+def test_config2_llama8b_shape_all_64_rows(fused):
+    stats = run_full_config("c2_llama8b", fused=fused)
+    assert [s[1] for s in stats] == [64]
 
 
 @pytest.mark.parametrize("fused", [True, False])
-def test_config4_large_batch_sampled_rows(fused):
-    run_full_config("c4_large_batch", sample=12, fused=fused)
+def test_config3_long_context_all_16_rows(fused):
+    stats = run_full_config("c3_long_context", fused=fused)
+    assert [s[1] for s in stats] == [16]
 
 
-def test_config5_hybrid_stack_sampled_rows_one_window_and_one_full_layer():
+@pytest.mark.parametrize("fused", [True, False])
+def test_config4_large_batch_all_256_rows(fused):
+    stats = run_full_config("c4_large_batch", fused=fused)
+    assert [s[1] for s in stats] == [256]
+
+
+def test_config5_hybrid_stack_all_eight_layers_window_layers_whole_full_layers_on_10_rows():
+    """All eight layers of the stack: the six sliding-window layers on all 128 rows, the two
+    full-attention layers (19 GB of KV each) on the shortest, the longest and eight seeded rows."""
     free, _ = torch.cuda.mem_get_info()
     if free < 70 * (1 << 30):
         pytest.skip("needs ~55 GB of device memory")
-    run_full_config("c5_hybrid_stack", sample=1, layers=[2, 3])
+    stats = run_full_config("c5_hybrid_stack", sample=None, sample_full=8)
+    assert [s[0] for s in stats] == list(range(8))
+    assert [s[1] for s in stats] == [128, 128, 128, 10, 128, 128, 128, 10]
 
 
 def test_read_probe_touches_every_word_and_validates_arguments():
