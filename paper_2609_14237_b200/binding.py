@@ -20,7 +20,7 @@ SOURCES = [os.path.join(_HERE, "csrc", "opw_attn.cu"), os.path.join(_HERE, "csrc
 HEADERS = [os.path.join(_HERE, "csrc", "opw_kernels.cuh"), os.path.join(_HERE, "csrc", "opw_afd_gemm.cuh"), os.path.join(_ROOT, "include", "opw_attn.h"),
            os.path.join(_ROOT, "include", "opw_linear_attn.h"), os.path.join(_ROOT, "include", "opw_afd.h")]
 
-OPW_FLAG_PDL = 1
+OPW_FLAG_NO_PDL = 1
 OPW_OK, OPW_ERR_INVALID_ARG, OPW_ERR_UNSUPPORTED, OPW_ERR_CAPACITY, OPW_ERR_CUDA, OPW_ERR_BAD_PAGE, OPW_ERR_TIMEOUT = range(7)
 
 EXPORTS = [

@@ -192,6 +192,7 @@ size_t opw_attn_stage_workspace_bytes(const opw_attn_stage_config_t* cfg) {
 opw_status_t opw_attn_stage_create(const opw_attn_stage_config_t* cfg, opw_attn_stage_t** out) {
   if (!cfg || !out) return OPW_ERR_INVALID_ARG;
   if (cfg->struct_size != sizeof(opw_attn_stage_config_t) || cfg->reserved != 0) return OPW_ERR_INVALID_ARG;
+  if (cfg->flags & ~(uint32_t)OPW_FLAG_NO_PDL) return OPW_ERR_INVALID_ARG;
   if (!shape_ok(cfg) || cfg->device < 0) return OPW_ERR_INVALID_ARG;
   if (!cfg->layer_window || !cfg->layer_num_pages || !cfg->layer_kv_pool || !cfg->workspace) return OPW_ERR_INVALID_ARG;
   if (cfg->head_dim != 64 && cfg->head_dim != 128 && cfg->head_dim != 256) return OPW_ERR_UNSUPPORTED;
@@ -319,7 +320,7 @@ opw_status_t opw_kv_append(opw_attn_stage_t* st, int32_t layer, int32_t batch, c
   p.max_pages = st->cfg.max_pages_per_seq;
   const int groups = p.Hkv * 2 * (p.D / 8);
   const int threads = groups < 256 ? ((groups + 31) / 32 * 32) : 256;
-  const bool pdl = (st->cfg.flags & OPW_FLAG_PDL) != 0;
+  const bool pdl = (st->cfg.flags & OPW_FLAG_NO_PDL) == 0;
   if (launch(opw::kv_append_kernel, dim3(batch), dim3(threads), 0, static_cast<cudaStream_t>(cuda_stream), pdl, p) !=
       cudaSuccess) {
     (void)cudaGetLastError();
@@ -384,7 +385,7 @@ static opw_status_t launch_attention(opw_attn_stage_t* st, const StepArgs& a, in
 
   const dim3 grid(st->grid), block(st->shape.warps * 32);
   const size_t smem = attn_smem_bytes(D, st->shape, a.batch);
-  const bool pdl = (st->cfg.flags & OPW_FLAG_PDL) != 0;
+  const bool pdl = (st->cfg.flags & OPW_FLAG_NO_PDL) == 0;
   cudaError_t e;
   if (D == 64) {
     if (G > 8) e = launch(opw::attn_splitkv_kernel<64, true>, grid, block, smem, stream, pdl, p);
@@ -431,7 +432,7 @@ static opw_status_t launch_combine(opw_attn_stage_t* st, const StepArgs& a, int 
   if (splits > opw::kCombineBatch) splits = opw::kCombineBatch;
   if (splits > kCombineScratchSlots / rows) splits = kCombineScratchSlots / rows;
   if (splits < 1) splits = 1;
-  const bool pdl = (st->cfg.flags & OPW_FLAG_PDL) != 0 && !side_stream;
+  const bool pdl = (st->cfg.flags & OPW_FLAG_NO_PDL) == 0 && !side_stream;
   const dim3 grid(rows, splits);
   cudaError_t e;
 #define OPW_LAUNCH_COMBINE(DIM)                                                                                            \

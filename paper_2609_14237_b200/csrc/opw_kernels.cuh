@@ -236,6 +236,31 @@ __host__ __device__ __forceinline__ void segment_bounds(int64_t U, int64_t num_w
   b = s0 + stat + ((dyn * dyn_cut(J, k)) >> 4);
 }
 
+// The same boundaries with one 64-bit division per thread instead of two per segment (the combine
+// kernel is bound by this integer arithmetic, not by memory):
+// begin(w) = floor(U*w/nw) = per*w + floor(rem*w/nw) with per = U / nw, rem = U % nw, and
+// rem*w < nw^2 fits 32 bits (nw <= 16 warps x 4 blocks x a few hundred SMs).
+struct ShareMath {
+  int64_t per;
+  uint32_t rem, nw;
+  int J;
+  __device__ __forceinline__ void init(int64_t U, int64_t num_workers) {
+    nw = (uint32_t)num_workers;
+    per = U / num_workers;
+    rem = (uint32_t)(U - per * num_workers);
+    J = dyn_chunks(U, num_workers);
+  }
+  __device__ __forceinline__ int64_t begin(uint32_t w) const { return per * (int64_t)w + (int64_t)((rem * w) / nw); }
+  __device__ __forceinline__ void bounds(uint32_t w, int k, int64_t& a, int64_t& b) const {   // == segment_bounds
+    const int64_t s0 = begin(w), s1 = begin(w + 1);
+    const int64_t len = s1 - s0, dyn = J > 0 ? (len * OPW_DYN_32NDS) >> 5 : 0, stat = len - dyn;
+    if (k == 0) { a = s0; b = s0 + stat; return; }
+    if (k > J) { a = b = s1; return; }
+    a = s0 + stat + ((dyn * dyn_cut(J, k - 1)) >> 4);
+    b = s0 + stat + ((dyn * dyn_cut(J, k)) >> 4);
+  }
+};
+
 // ---------------------------------------------------------------------------------
 // KV append: one thread block per sequence, one thread per 16-byte group
 // ---------------------------------------------------------------------------------
@@ -913,14 +938,16 @@ __global__ void __launch_bounds__(kCT, kCT == 128 ? 6 : 2) combine_kernel(Combin
   const int64_t stride = (int64_t)G * (D + 2);
   // segments a share really has in this launch (1 + the number of ticketed chunks, which depends on the
   // share length only): small launches have fewer than kSegPerShare, and fewer candidates to test
-  const int segs = dyn_chunks(U, p.num_workers) + 1;
+  ShareMath sm;
+  sm.init(U, p.num_workers);
+  const int segs = sm.J + 1;
   // If the segment that holds the row's first unit also holds its last, that segment's worker
   // has already stored the final result: nothing to merge (every block of the row sees this).
   {
     bool whole = false;
     if (threadIdx.x < segs) {
       int64_t a, bnd;
-      segment_bounds(U, p.num_workers, wf, (int)threadIdx.x, a, bnd);
+      sm.bounds((uint32_t)wf, (int)threadIdx.x, a, bnd);
       whole = a <= ustart && ustart < bnd && bnd >= uend;
     }
     if (__syncthreads_or(whole)) return;
@@ -995,7 +1022,9 @@ __global__ void __launch_bounds__(kCT, kCT == 128 ? 6 : 2) combine_kernel(Combin
     bool hit = false;
     int32_t slot = 0;
     if (threadIdx.x < kCombineBatch && i < ncand) {
-      const int64_t j = i / segs;
+      int64_t j;                                   // candidate i = (share or unit j, segment k); 32-bit division where it fits
+      if (ncand < (int64_t)1 << 31) j = (int64_t)((uint32_t)i / (uint32_t)segs);
+      else j = i / segs;
       const int k = (int)(i - j * segs);
       int64_t w;
       bool counted = true;
@@ -1006,7 +1035,7 @@ __global__ void __launch_bounds__(kCT, kCT == 128 ? 6 : 2) combine_kernel(Combin
         w = wf + j;
       }
       int64_t a, bnd;
-      segment_bounds(U, p.num_workers, w, k, a, bnd);
+      sm.bounds((uint32_t)w, k, a, bnd);
       hit = counted && a < bnd && a < uend && bnd > ustart;
       slot = (int32_t)(2 * (w * kSegPerShare + k) + (a >= ustart ? 0 : 1));
     }

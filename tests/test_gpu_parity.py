@@ -176,14 +176,14 @@ def test_fused_step_with_a_position_beyond_the_table_appends_nothing_for_that_ro
 
 @pytest.mark.parametrize("fused", [True, False])
 def test_programmatic_dependent_launch_keeps_back_to_back_steps_ordered(fused):
-    """With OPW_FLAG_PDL every kernel may start while its predecessor finishes; eight steps enqueued
+    """By default every kernel may start while its predecessor finishes; eight steps enqueued
     without a host synchronisation in between must still leave the exact pool and the right outputs."""
     wl = synth.Workload("pdl", 8, 32, 8, 128, [0, 200], "uniform_1024_4096", 80)
     inp = synth.make_inputs(wl, device="cpu", growth=4, steps=4)
     pools = [p.cuda() for p in inp.pools]
     refs = [oracle.as_u16(p).copy() for p in inp.pools]
     st = B.Stage(pools=pools, layer_window=wl.layer_window, num_q_heads=32, num_kv_heads=8, head_dim=128,
-                 max_batch=8, max_pages_per_seq=inp.max_pages_per_seq, flags=B.OPW_FLAG_PDL)
+                 max_batch=8, max_pages_per_seq=inp.max_pages_per_seq)
     tabs = [t.cuda() for t in inp.page_tables]
     dq, dk, dv = inp.q.cuda(), inp.k_new.cuda(), inp.v_new.cuda()
     pos = [dev(inp.positions(s)) for s in range(4)]
@@ -213,14 +213,14 @@ def test_programmatic_dependent_launch_keeps_back_to_back_steps_ordered(fused):
 def test_programmatic_dependent_launch_with_an_all_inactive_step_between_two_live_ones(fused):
     """A grid with nothing to do must still pass its dependency wait before it completes, or the kernels
     behind it could overtake the step in front of it: live step, all-inactive step, live step, enqueued
-    back to back on one stream with OPW_FLAG_PDL, repeated over two layers; every output and the whole
+    back to back on one stream (programmatic dependent launch is the default), repeated over two layers; every output and the whole
     pool against the oracle."""
     wl = synth.Workload("pdl0", 8, 32, 8, 128, [0, 200], "uniform_1024_4096", 81)
     inp = synth.make_inputs(wl, device="cpu", growth=3, steps=3)
     pools = [p.cuda() for p in inp.pools]
     refs = [oracle.as_u16(p).copy() for p in inp.pools]
     st = B.Stage(pools=pools, layer_window=wl.layer_window, num_q_heads=32, num_kv_heads=8, head_dim=128,
-                 max_batch=8, max_pages_per_seq=inp.max_pages_per_seq, flags=B.OPW_FLAG_PDL)
+                 max_batch=8, max_pages_per_seq=inp.max_pages_per_seq)
     tabs = [t.cuda() for t in inp.page_tables]
     dq, dk, dv = inp.q.cuda(), inp.k_new.cuda(), inp.v_new.cuda()
     # step 1 is the empty one: every slot inactive; the live steps are decode steps 0 and 1 of the sequences
@@ -410,7 +410,8 @@ def test_bad_page_ids_are_masked_and_reported_not_dereferenced():
 
 @pytest.mark.parametrize("tune", [dict(tune_warps=1, tune_stages=2), dict(tune_warps=4, tune_stages=6),
                                   dict(tune_warps=4, tune_stages=3, tune_ctas_per_sm=2), dict(tune_warps=8, tune_stages=3),
-                                  dict(tune_warps=3, tune_stages=8)])
+                                  dict(tune_warps=3, tune_stages=8), dict(flags=B.OPW_FLAG_NO_PDL),
+                                  dict(tune_warps=5, tune_stages=3, flags=B.OPW_FLAG_NO_PDL)])
 def test_result_does_not_depend_on_the_split(tune):
     """The log-sum-exp merge is exact in real arithmetic: any split agrees within rounding."""
     rng = np.random.default_rng(56)

@@ -44,11 +44,11 @@ def draw_case(rng):
     if rng.integers(0, 3) == 0:
         tune = dict(tune_warps=int(rng.choice([1, 2, 4, 6] if D == 256 else [1, 3, 4, 8])), tune_stages=int(rng.choice([2, 3, 4])))
     if rng.integers(0, 4) == 0:
-        tune["flags"] = B.OPW_FLAG_PDL
+        tune["flags"] = B.OPW_FLAG_NO_PDL
     return D, Hkv * G, Hkv, [int(x) for x in lens], window, bool(rng.integers(0, 2)), tune
 
 
-@pytest.mark.parametrize("block", range(6))
+@pytest.mark.parametrize("block", range(8))
 def test_random_cases_match_the_oracle(block):
     B.build()
     for it in range(12):
@@ -91,5 +91,5 @@ def test_random_cases_match_the_oracle(block):
         assert (err <= 2.0 ** -6 * row_rms + 2.0 ** -8 * np.abs(ref) + 1e-6).all(), (what, float(err.max()))
         fin = np.isfinite(ref_lse)
         assert (np.isneginf(gl) == np.isneginf(ref_lse)).all(), what
-        assert (np.abs(gl[fin] - ref_lse[fin]) <= 2e-3).all(), what
+        assert (np.abs(gl[fin] - ref_lse[fin]) <= 1e-3).all(), what
         st.close()
