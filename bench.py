@@ -604,7 +604,7 @@ def run_linear_layer(steps, batch=256, Hk=16, Hv=32, dk=128, dv=128, rotate=4):
             "steps": steps}
 
 
-def run_afd_module(steps, name="c2_llama8b", hidden=4096, layers=4):
+def run_afd_module(steps, name="c2_llama8b", hidden=4096, layers=4, batch=None):
     """The complete attention module (QKV projection + rotary encoding + core attention + output
     projection) on the workload's shape: time per module step with the projections on the
     tensor-core kernel and on the library path, back to back over `layers` layers with their own
@@ -615,6 +615,8 @@ def run_afd_module(steps, name="c2_llama8b", hidden=4096, layers=4):
     from paper_2609_14237_b200 import binding, synth
 
     wl = dataclasses.replace(synth.WORKLOADS[name], layer_window=[0] * layers)
+    if batch:
+        wl = dataclasses.replace(wl, batch=int(batch))
     total = steps + 8
     inp = synth.make_inputs(wl, device="cuda", growth=4 * (total // layers + 4), steps=1)
     Hq, Hkv, D, Bn = wl.num_q_heads, wl.num_kv_heads, wl.head_dim, wl.batch
@@ -649,15 +651,15 @@ def run_afd_module(steps, name="c2_llama8b", hidden=4096, layers=4):
         torch.cuda.synchronize()
         return e0.elapsed_time(e1) / steps
 
-    stage_pdl = binding.Stage(pools=inp.pools, layer_window=wl.layer_window, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D,
-                              max_batch=Bn, max_pages_per_seq=inp.max_pages_per_seq)
+    stage_plain = binding.Stage(pools=inp.pools, layer_window=wl.layer_window, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D,
+                                max_batch=Bn, max_pages_per_seq=inp.max_pages_per_seq, flags=binding.OPW_FLAG_NO_PDL)
     res = {}
     for label, st, flags in (("tcgen05", stage, 0), ("library", stage, binding.OPW_AFD_LIBRARY_GEMM),
-                             ("tcgen05_pdl", stage_pdl, binding.OPW_AFD_PDL)):
+                             ("tcgen05_no_pdl", stage_plain, binding.OPW_AFD_NO_PDL)):
         mods = [binding.AfdModule(st, l, w_qkv[l], w_o[l], 10000.0, flags) for l in range(layers)]
         res[label] = timed(lambda l, pos: mods[l].step(x, pos, inp.page_tables[l], y))
         assert all(m.poll_error() == 0 for m in mods) and st.poll_error() == 0
-        if label == "tcgen05_pdl":
+        if label == "tcgen05":
             # the same steps as one plan: all layers' module steps in one CUDA graph, positions advanced on the device
             pos = pos0.clone()
             ops = [dict(kind="afd_module", module=mods[l].handle, batch=Bn, x=x.data_ptr(), positions=pos.data_ptr(),
@@ -678,14 +680,14 @@ def run_afd_module(steps, name="c2_llama8b", hidden=4096, layers=4):
             binding.opw_attn_plan_destroy(plan)
         for m in mods:
             m.close()
-    stage_pdl.close()
+    stage_plain.close()
     q, k, v = inp.q[0, 0], inp.k_new[0, 0], inp.v_new[0, 0]
     res["attention"] = timed(lambda l, pos: stage.decode_step(l, q, k, v, pos, inp.page_tables[l], out))
     stage.close()
     weight_bytes = 2 * ((Hq + 2 * Hkv) * D * hidden + hidden * Hq * D)
     return {"value": round(Bn / (res["tcgen05"] * 1e-3), 1), "unit": "sequence-steps/s per layer (whole attention module)",
             "ms_per_step": round(res["tcgen05"], 5), "ms_per_step_library_gemm": round(res["library"], 5),
-            "ms_per_step_programmatic_dependent_launch": round(res["tcgen05_pdl"], 5),
+            "ms_per_step_without_programmatic_dependent_launch": round(res["tcgen05_no_pdl"], 5),
             "ms_per_step_plan": round(res["plan"], 5),
             "ms_per_step_core_attention_alone": round(res["attention"], 5),
             "projection_weight_bytes_per_step": weight_bytes, "kv_bytes_per_step": int(inp.kv_bytes(0, 0)),
@@ -796,6 +798,7 @@ def main():
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--ctas", type=int, default=0)
     ap.add_argument("--unfused", action="store_true", help="separate opw_kv_append + opw_decode_attention calls")
+    ap.add_argument("--module-batch", type=int, default=0, help="batch rows of --workload attention_module (default: the shape's own)")
     ap.add_argument("--no-pdl", action="store_true", help="launch the kernels without programmatic stream serialisation")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -831,7 +834,7 @@ def main():
     steps = args.steps if args.steps is not None else 2000
     warmup = args.warmup if args.warmup is not None else 20
     if args.workload == "attention_module":         # the AFD partition's stage alone (1 GPU)
-        r = run_afd_module(max(8, min(steps, 2000)))
+        r = run_afd_module(max(8, min(steps, 2000)), batch=args.module_batch)
         r.update({"metric": "attention module decode: sequence-steps/s per layer", "n_gpus": 1, "warmup": 8,
                   "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                   "gpu_launches": r["steps"] * 4})

@@ -11,9 +11,9 @@
  *     y = out W_o^T
  * The two projections run on a hand-written tcgen05 kernel made for decode shapes: the weight
  * rows fill the tensor core's M dimension and TMEM lanes, the few batch rows its N dimension,
- * TMA streams the weights once, K is split over CTAs so that every SM pulls weights.  With
- * OPW_AFD_LIBRARY_GEMM (and for the QKV projection at head_dim 256, whose rotated pairs do not
- * fit one tile) they are cuBLASLt calls followed by a separate rotary kernel instead.
+ * TMA streams the weights once, K is split over CTAs so that every SM pulls weights; batches of
+ * more than 256 rows are walked in tiles of 256.  Only with OPW_AFD_LIBRARY_GEMM, kept as a
+ * comparison arm, are they cuBLASLt calls followed by a separate rotary kernel instead.
  * It exists to measure the contrast the paper's analysis rests on (Section 3.1: memory-bound
  * attention against GEMM-dominated projections) on the same device, and to let a caller move
  * the stage boundary from CAD to AFD without touching the KV cache.
@@ -21,7 +21,7 @@
  * The paper fixes no rotary convention; the reading taken here is the rotate-half form: for
  * i < D/2 the pair (x_i, x_{i+D/2}) turns by the angle position * theta^(-2i/D).
  *
- * Conventions as in opw_attn.h.  On the library path the module holds a cuBLASLt handle (the
+ * Conventions as in opw_attn.h.  With OPW_AFD_LIBRARY_GEMM the module holds a cuBLASLt handle (the
  * library allocates its own host-side state for it); all device memory, including the GEMM
  * workspace, is the caller's.  The tensor-core kernels wait with a bound (0.2 s) on their
  * shared-memory barriers; a wait that runs out is recorded in a status word that
@@ -39,12 +39,13 @@ extern "C" {
 typedef struct opw_afd_module opw_afd_module_t;
 
 #define OPW_AFD_LIBRARY_GEMM 1u /* projections by cuBLASLt + separate rotary kernel */
-#define OPW_AFD_PDL 2u          /* launch the tensor-core projections with programmatic dependent launch: their
-                                   set-up and the first weight tiles overlap the tail of the previous kernel in
-                                   the stream (pairs with OPW_FLAG_PDL of the stage) */
+#define OPW_AFD_NO_PDL 2u       /* launch the tensor-core projections without programmatic dependent launch (by
+                                   default their set-up and first weight tiles overlap the tail of the previous
+                                   kernel in the stream, as the stage's own kernels do) */
 
 /* Scratch bytes of one module: qkv, q, k_new, v_new and attention-output buffers for
- * max_batch rows, split-K partial tiles, 32 MiB of library GEMM workspace.  0 on invalid
+ * max_batch rows, split-K partial tiles, the table of rotation angles, 32 MiB of workspace for
+ * the library arm.  0 on invalid
  * arguments. */
 size_t opw_afd_module_workspace_bytes(int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim, int32_t max_batch,
                                       int32_t hidden);
@@ -66,8 +67,8 @@ opw_status_t opw_afd_module_create(opw_attn_stage_t *stage, int32_t layer, int32
  * One decode step of the module: x [batch, hidden] bf16 in, y [batch, hidden] bf16 out, the
  * layer's KV cache appended at positions[b] (< 0: inactive row, y row = 0).  x and y 16-byte
  * aligned.  Enqueues four kernels on the stream (QKV projection with the rotary epilogue,
- * attention, combine, output projection); batches above 96 rows take the library path for the
- * two projections (cuBLASLt, plus the separate rotary kernel).
+ * attention, combine, output projection), five for batches above 96 rows, whose table of rotation
+ * angles is written by a small kernel first instead of inside the QKV projection.
  */
 opw_status_t opw_afd_module_step(opw_afd_module_t *module, int32_t batch, const void *x, const int32_t *positions,
                                  const int32_t *page_table, void *y, void *cuda_stream);

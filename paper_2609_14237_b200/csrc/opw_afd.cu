@@ -1,8 +1,8 @@
 // The complete attention module as one stage (AFD partition): QKV projection with the rotary
 // encoding and the split into q / k_new / v_new in its epilogue, core attention
 // (opw_decode_step), output projection.  The projections run on the tcgen05 kernel of
-// opw_afd_gemm.cuh; cuBLASLt plus a separate rotary kernel is the alternative path
-// (OPW_AFD_LIBRARY_GEMM, and head_dim 256).  See include/opw_afd.h.
+// opw_afd_gemm.cuh at every batch size and head dimension; cuBLASLt plus a separate rotary
+// kernel is a comparison arm that only OPW_AFD_LIBRARY_GEMM selects.  See include/opw_afd.h.
 #include "opw_afd.h"
 #include "opw_afd_gemm.cuh"
 
@@ -114,7 +114,7 @@ struct opw_afd_module {
   const void* w_o;
   double log_theta;
   unsigned char* ws;
-  size_t off_qkv, off_q, off_k, off_v, off_out, off_gemm, off_partials, off_tickets, off_status;
+  size_t off_qkv, off_q, off_k, off_v, off_out, off_gemm, off_partials, off_tickets, off_angles, off_status;
   // tensor-core path
   bool tc_qkv, tc_o, pdl;
   int sms;
@@ -132,44 +132,47 @@ struct opw_afd_module {
 namespace {
 
 constexpr int kSmsBound = 160;             // split-K sizing assumes no more SMs than this
-// Above this batch the skinny kernel stops paying: every CTA streams the whole activation matrix
-// beside its 128 weight rows, so at 256 rows two thirds of its traffic is activations re-read from
-// L2 by every CTA, and a square-tiled library GEMM wins (measured: ahead up to 32 rows, level at
-// 64 and 96, behind at 128).
-constexpr int kTcMaxBatch = 96;
+// Up to this batch the step's (cos, sin) table is computed inside the QKV kernel, in shared memory behind
+// the ring; above it the table (batch * D/2 * 8 bytes) would crowd the ring out, so a small kernel
+// writes it to global memory first.
+constexpr int kSmemAngleBatch = 96;
 constexpr size_t kGemmSmemBudget = 226 * 1024;
 
 inline int round16(int x) { return (x + 15) / 16 * 16; }
 inline int tiles_of(int n_out) { return (n_out + opw_afd::kTileM - 1) / opw_afd::kTileM; }
-inline int ksplit_of(int n_out, int k, int sms) {
-  int ks = sms / tiles_of(n_out);
+inline int batch_tiles_of(int batch) { return (batch + opw_afd::kMaxNb - 1) / opw_afd::kMaxNb; }
+inline int nb_of(int batch) { return round16(batch < opw_afd::kMaxNb ? batch : opw_afd::kMaxNb); }
+inline int ksplit_of(int n_out, int k, int batch, int sms) {
+  int ks = sms / (tiles_of(n_out) * batch_tiles_of(batch));
   if (ks > opw_afd::kMaxSplit) ks = opw_afd::kMaxSplit;
   const int kblocks = (k + opw_afd::kBlockK - 1) / opw_afd::kBlockK;
   if (ks > kblocks) ks = kblocks;
   return ks < 1 ? 1 : ks;
 }
-inline size_t partial_bytes(int n_out, int k, int nb) {
-  return (size_t)tiles_of(n_out) * ksplit_of(n_out, k, kSmsBound) * nb * opw_afd::kTileM * sizeof(float);
+inline size_t partial_bytes(int n_out, int k, int batch) {
+  // the widest split any device can pick (an upper bound over SM counts), every batch tile
+  return (size_t)tiles_of(n_out) * batch_tiles_of(batch) * opw_afd::kMaxSplit * nb_of(batch) * opw_afd::kTileM * sizeof(float);
 }
 
-struct Carve { size_t qkv, q, k, v, out, gemm, partials, tickets, status, total; };
+struct Carve { size_t qkv, q, k, v, out, gemm, partials, tickets, angles, status, total; };
 
 Carve carve(int Hq, int Hkv, int D, int max_batch, int hidden) {
   Carve c;
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
   const int n_qkv = (Hq + 2 * Hkv) * D, n_attn = Hq * D;
-  const int nb = round16(max_batch < kTcMaxBatch ? max_batch : kTcMaxBatch);
   c.qkv = take((size_t)max_batch * n_qkv * 2);
   c.q = take((size_t)max_batch * n_attn * 2);
   c.k = take((size_t)max_batch * Hkv * D * 2);
   c.v = take((size_t)max_batch * Hkv * D * 2);
   c.out = take((size_t)max_batch * n_attn * 2);
   c.gemm = take(kGemmWorkspace);
-  const size_t p1 = partial_bytes(n_qkv, hidden, nb), p2 = partial_bytes(hidden, n_attn, nb);
+  // partial tiles: the largest over every batch <= max_batch (nb * batch tiles is monotone in the batch)
+  const size_t p1 = partial_bytes(n_qkv, hidden, max_batch), p2 = partial_bytes(hidden, n_attn, max_batch);
   c.partials = take(p1 > p2 ? p1 : p2);
+  c.angles = take((size_t)max_batch * (D / 2) * sizeof(float2));
   const int t1 = tiles_of(n_qkv), t2 = tiles_of(hidden);
-  c.tickets = take((size_t)(t1 > t2 ? t1 : t2) * sizeof(uint32_t));
+  c.tickets = take((size_t)(t1 > t2 ? t1 : t2) * batch_tiles_of(max_batch) * sizeof(uint32_t));
   c.status = take(sizeof(uint32_t));
   c.total = off;
   return c;
@@ -192,20 +195,48 @@ bool encode_map(TensorMapEncodeFn fn, CUtensorMap* map, const void* base, uint64
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// One projection on the tensor-core kernel (batch <= kTcMaxBatch).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, bool pdl, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+// One projection on the tensor-core kernel.
 opw_status_t run_tc_gemm(opw_afd_module* m, const CUtensorMap& map_w, const void* x, int batch, int n_out, int k, int mode,
                          const int32_t* positions, __nv_bfloat16* out, __nv_bfloat16* q, __nv_bfloat16* kn,
                          __nv_bfloat16* vn, cudaStream_t stream) {
   opw_afd::GemmParams p;
-  p.n_out = n_out; p.k = k; p.batch = batch; p.nb = round16(batch);
+  p.n_out = n_out; p.k = k; p.batch = batch; p.nb = nb_of(batch);
+  p.group = (mode == 1 && m->D > opw_afd::kTileM) ? 2 : 1;   // a head of 256 spans two weight tiles
   const size_t stage_bytes = opw_afd::kTileABytes + (size_t)p.nb * 128;
-  // mode 1 keeps the step's angle table behind the ring: (cos, sin) per row and pair, then D/2 doubles
-  const size_t angle_bytes = mode == 1 ? (size_t)batch * (m->D / 2) * sizeof(float2) + (size_t)(m->D / 2) * sizeof(double) : 0;
-  int stages = (int)((kGemmSmemBudget - 1024 - angle_bytes) / stage_bytes);
-  if (stages > opw_afd::kMaxStages) stages = opw_afd::kMaxStages;
-  if ((size_t)stages * stage_bytes < (size_t)p.nb * opw_afd::kTileM * sizeof(float)) return OPW_ERR_UNSUPPORTED;   // the epilogue reuses the ring
+  // The step's (cos, sin) table: behind the ring for small batches, from global memory (written by a small
+  // kernel launched just before) for large ones and wherever the table would leave the ring too small.
+  // The epilogue reuses the ring: one tile of sums for all columns, or two tiles for a chunk of columns.
+  const int chunk_cols = batch < opw_afd::kChunkCols ? batch : opw_afd::kChunkCols;
+  const size_t epi_bytes = p.group == 1 ? (size_t)p.nb * opw_afd::kTileM * sizeof(float)
+                                        : ((size_t)opw_afd::kChunkCols + chunk_cols) * opw_afd::kTileM * sizeof(float);
+  bool angles_global = mode == 1 && batch > kSmemAngleBatch;
+  size_t angle_bytes = 0;
+  int stages = 0;
+  for (;;) {
+    angle_bytes = (mode == 1 && !angles_global) ? (size_t)batch * (m->D / 2) * sizeof(float2) + (size_t)(m->D / 2) * sizeof(double) : 0;
+    stages = (int)((kGemmSmemBudget - 1024 - angle_bytes) / stage_bytes);
+    if (stages > opw_afd::kMaxStages) stages = opw_afd::kMaxStages;
+    if ((stages >= 4 && (size_t)stages * stage_bytes >= epi_bytes) || angles_global || mode != 1) break;
+    angles_global = true;
+  }
+  if (stages < 2 || (size_t)stages * stage_bytes < epi_bytes) return OPW_ERR_UNSUPPORTED;
   p.stages = stages;
-  p.ksplit = ksplit_of(n_out, k, m->sms < kSmsBound ? m->sms : kSmsBound);
+  p.ksplit = ksplit_of(n_out, k, batch, m->sms < kSmsBound ? m->sms : kSmsBound);
   p.mode = mode;
   p.out = out; p.q = q; p.kn = kn; p.vn = vn;
   p.positions = positions;
@@ -214,21 +245,22 @@ opw_status_t run_tc_gemm(opw_afd_module* m, const CUtensorMap& map_w, const void
   p.partials = reinterpret_cast<float*>(m->ws + m->off_partials);
   p.tickets = reinterpret_cast<uint32_t*>(m->ws + m->off_tickets);
   p.status = reinterpret_cast<uint32_t*>(m->ws + m->off_status);
+  p.angles_g = angles_global ? reinterpret_cast<const float2*>(m->ws + m->off_angles) : nullptr;
   // trace region 0: output projection, region 1: QKV projection
   p.trace = m->trace ? m->trace + (size_t)mode * opw_afd::kTraceMaxCtas * opw_afd::kTraceWords : nullptr;
+  if (angles_global) {
+    if (launch_pdl(opw_afd::rope_table_kernel, dim3(batch), dim3(128), 0, stream, m->pdl, positions,
+                   reinterpret_cast<float2*>(m->ws + m->off_angles), (int)m->D, m->log_theta) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return OPW_ERR_CUDA;
+    }
+    ++m->launches;
+  }
   CUtensorMap map_x;       // the activation pointer and the batch change from call to call: encoded per launch, on the host
   if (!encode_map(m->encode, &map_x, x, (uint64_t)batch, (uint64_t)k, (uint32_t)p.nb)) return OPW_ERR_CUDA;
-  cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(tiles_of(n_out), p.ksplit);
-  cfg.blockDim = dim3(opw_afd::kGemmThreads);
-  cfg.dynamicSmemBytes = 1024 + (size_t)stages * stage_bytes + angle_bytes;
-  cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = m->pdl ? 1 : 0;
-  if (cudaLaunchKernelEx(&cfg, opw_afd::skinny_gemm_kernel, map_w, map_x, p) != cudaSuccess) {
+  const dim3 grid(tiles_of(n_out), p.ksplit, batch_tiles_of(batch));
+  if (launch_pdl(opw_afd::skinny_gemm_kernel, grid, dim3(opw_afd::kGemmThreads), 1024 + (size_t)stages * stage_bytes + angle_bytes,
+                 stream, m->pdl, map_w, map_x, p) != cudaSuccess) {
     (void)cudaGetLastError();
     return OPW_ERR_CUDA;
   }
@@ -249,7 +281,7 @@ opw_status_t opw_afd_module_create(opw_attn_stage_t* stage, int32_t layer, int32
                                    const void* w_o, float rope_theta, uint32_t flags, void* workspace,
                                    size_t workspace_bytes, opw_afd_module_t** out) {
   if (!stage || !w_qkv || !w_o || !workspace || !out) return OPW_ERR_INVALID_ARG;
-  if (hidden < 8 || hidden % 8 != 0 || !(rope_theta > 0.f) || (flags & ~(OPW_AFD_LIBRARY_GEMM | OPW_AFD_PDL))) return OPW_ERR_INVALID_ARG;
+  if (hidden < 8 || hidden % 8 != 0 || !(rope_theta > 0.f) || (flags & ~(OPW_AFD_LIBRARY_GEMM | OPW_AFD_NO_PDL))) return OPW_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255) || (reinterpret_cast<uintptr_t>(w_qkv) & 15) ||
       (reinterpret_cast<uintptr_t>(w_o) & 15))
     return OPW_ERR_INVALID_ARG;
@@ -268,16 +300,16 @@ opw_status_t opw_afd_module_create(opw_attn_stage_t* stage, int32_t layer, int32
   m->log_theta = std::log((double)rope_theta);
   m->ws = static_cast<unsigned char*>(workspace);
   m->off_qkv = c.qkv; m->off_q = c.q; m->off_k = c.k; m->off_v = c.v; m->off_out = c.out; m->off_gemm = c.gemm;
-  m->off_partials = c.partials; m->off_tickets = c.tickets; m->off_status = c.status;
+  m->off_partials = c.partials; m->off_tickets = c.tickets; m->off_angles = c.angles; m->off_status = c.status;
   m->plan_batch = 0;
   m->launches = 0;
   m->trace = nullptr;
   m->lt = nullptr;
   m->encode = nullptr;
   const bool library = (flags & OPW_AFD_LIBRARY_GEMM) != 0;
-  m->tc_qkv = !library && D <= 128;         // the rotary epilogue needs a rotated pair inside one 128-row tile
+  m->tc_qkv = !library;
   m->tc_o = !library;
-  m->pdl = (flags & OPW_AFD_PDL) != 0;
+  m->pdl = (flags & OPW_AFD_NO_PDL) == 0;
   bool ok = true;
   if (m->tc_qkv || m->tc_o) {
     void* fn = nullptr;
@@ -295,8 +327,8 @@ opw_status_t opw_afd_module_create(opw_attn_stage_t* stage, int32_t layer, int32
     ok = ok && encode_map(m->encode, &m->map_wo, w_o, (uint64_t)hidden, (uint64_t)n_attn, opw_afd::kTileM);
   }
   // tickets and the status word start at zero (synchronously, on the default stream, as the stage does)
-  ok = ok && cudaMemset(m->ws + c.tickets, 0, c.total - c.tickets) == cudaSuccess;
-  if (ok) ok = cublasLtCreate(&m->lt) == CUBLAS_STATUS_SUCCESS;   // also serves batches beyond kTcMaxBatch
+  ok = ok && cudaMemset(m->ws + c.tickets, 0, c.total - c.tickets) == cudaSuccess;   // tickets, then the status word
+  if (ok && library) ok = cublasLtCreate(&m->lt) == CUBLAS_STATUS_SUCCESS;   // only the comparison arm touches the library
   if (!ok) {
     (void)cudaGetLastError();
     if (m->lt) cublasLtDestroy(m->lt);
@@ -314,7 +346,7 @@ opw_status_t opw_afd_module_step(opw_afd_module_t* m, int32_t batch, const void*
   if (batch > m->max_batch) return OPW_ERR_CAPACITY;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const int n_qkv = (m->Hq + 2 * m->Hkv) * m->D, n_attn = m->Hq * m->D;
-  const bool tc_qkv = m->tc_qkv && batch <= kTcMaxBatch, tc_o = m->tc_o && batch <= kTcMaxBatch;
+  const bool tc_qkv = m->tc_qkv, tc_o = m->tc_o;
   if ((!tc_qkv || !tc_o) && m->plan_batch != batch) {
     m->plan_batch = 0;
     if (!tc_qkv && !make_plan(m->lt, m->plan_qkv, batch, n_qkv, m->hidden)) return OPW_ERR_CUDA;

@@ -1,7 +1,7 @@
 // Skinny projection GEMM of the decode step on the 5th-generation tensor cores (sm_100a).
 //
-//   C[b, n] = sum_k x[b, k] * W[n, k]          x: [batch, K] bf16 (batch <= 256; the module stops at 96), W: [N, K] bf16,
-//                                               fp32 accumulate
+//   C[b, n] = sum_k x[b, k] * W[n, k]          x: [batch, K] bf16, W: [N, K] bf16, fp32 accumulate
+//                                               (any batch: blockIdx.z walks over tiles of 256 rows)
 //
 // A decode step has few rows (the batch) and a large weight matrix that is read once, so the
 // kernel is built around streaming W: the WEIGHT rows take the tensor core's M dimension (one
@@ -45,9 +45,14 @@ constexpr uint32_t kTileABytes = kTileM * kBlockK * 2;
 constexpr uint64_t kGemmWaitNs = 200ull * 1000 * 1000;
 constexpr uint32_t kGemmErrTimeout = 2u;  // same bit as the attention kernels' timeout
 
+constexpr int kMaxNb = 256;               // batch rows per CTA (the MMA's N); more rows: blockIdx.z
+constexpr int kChunkCols = 128;           // batch columns the epilogue of a two-tile group handles at a time
+
 struct GemmParams {
   int n_out, k, batch;
-  int nb;                 // MMA N: batch rounded up to a multiple of 16 (16..256)
+  int nb;                 // MMA N of a full batch tile: min(batch, 256) rounded up to a multiple of 16
+  int group;              // weight tiles that share a ticket and an epilogue: 1, or 2 (rotary at D = 256)
+  const float2* angles_g; // mode 1: [batch, D/2] (cos, sin) in global memory, or null: computed here in shared memory
   int stages;
   int ksplit;
   int mode;               // 0: plain, 1: rotary + split into q / k / v
@@ -157,9 +162,67 @@ __device__ __forceinline__ uint32_t g_instr_desc(int n) {
   return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(kTileM >> 4) << 24);
 }
 
-// grid = (ceil(n_out / 128), ksplit), 512 threads, 1 CTA per SM.
-// Dynamic shared memory: 1024 (alignment slack) + stages * (16384 + nb * 128) bytes, then in mode 1
-// the angle table, batch * D/2 (cos, sin) pairs of 8 bytes.
+// dst[i] = sum over the ksplit partial tiles of part[s * split_stride + i], in split order (so the result does
+// not depend on which CTA came last); if own >= 0 the partial of that split is read from dst itself (it is
+// still in shared memory there).  Every other split's values are requested at once: the reduction would
+// otherwise be a chain of L2 round trips.  A function of its own so that it is compiled once.
+__device__ __noinline__ void gemm_reduce_partials(const float4* part, float4* dst, int n4, int ksplit, int own, size_t split_stride) {
+  constexpr int R = 2;
+  const int step = R * kGemmThreads;
+  auto fetch = [&](float4 (&v)[R][kMaxSplit], int ib) {
+#pragma unroll
+    for (int r = 0; r < R; ++r)
+#pragma unroll
+      for (int sp = 0; sp < kMaxSplit; ++sp) {
+        const int i = ib + r * kGemmThreads;
+        if (i < n4 && sp < ksplit && sp != own) v[r][sp] = __ldcg(part + sp * split_stride + i);
+      }
+  };
+  auto sum = [&](const float4 (&v)[R][kMaxSplit], int ib) {
+#pragma unroll
+    for (int r = 0; r < R; ++r) {
+      const int i = ib + r * kGemmThreads;
+      if (i >= n4) break;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int sp = 0; sp < kMaxSplit; ++sp)
+        if (sp < ksplit) {
+          const float4 t = sp == own ? dst[i] : v[r][sp];
+          acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+        }
+      dst[i] = acc;
+    }
+  };
+  // two buffers: the loads of the next pair of rows are in flight while this pair is summed
+  float4 va[R][kMaxSplit], vb[R][kMaxSplit];
+  int ib = threadIdx.x;
+  if (ib < n4) fetch(va, ib);
+  for (; ib < n4; ib += 2 * step) {
+    if (ib + step < n4) fetch(vb, ib + step);
+    sum(va, ib);
+    if (ib + 2 * step < n4) fetch(va, ib + 2 * step);
+    if (ib + step < n4) sum(vb, ib + step);
+  }
+}
+
+// (cos, sin) of position * theta^(-2i/D) for every sequence b and pair i < D/2, in double (a float angle is
+// off by 1e-7 * position radians), stored as float2 [batch, D/2].  One block per sequence.
+__global__ void rope_table_kernel(const int32_t* __restrict__ positions, float2* __restrict__ table, int D, double log_theta) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  const int b = blockIdx.x, half = D >> 1;
+  int32_t pos = positions[b];
+  if (pos < 0) pos = 0;                              // inactive row: any finite value, the row is never appended
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // the table may still be read by an earlier kernel of the stream
+  for (int i = threadIdx.x; i < half; i += blockDim.x) {
+    double sn, cn;
+    sincos((double)pos * exp(-2.0 * i / D * log_theta), &sn, &cn);
+    table[(size_t)b * half + i] = make_float2((float)cn, (float)sn);
+  }
+}
+
+// grid = (ceil(n_out / 128), ksplit, ceil(batch / 256)), 512 threads, 1 CTA per SM.
+// Dynamic shared memory: 1024 (alignment slack) + stages * (16384 + nb * 128) bytes, then in mode 1 without a
+// global angle table the table itself, batch * D/2 (cos, sin) pairs of 8 bytes and D/2 doubles.
 __global__ void __launch_bounds__(kGemmThreads, 1)
 skinny_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const GemmParams p) {
   extern __shared__ unsigned char g_smem_raw[];
@@ -172,18 +235,23 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tile = blockIdx.x, split = blockIdx.y;
+  const int b_off = blockIdx.z * kMaxNb;                     // first batch row of this CTA's batch tile
+  const int batch_here = p.batch - b_off < kMaxNb ? p.batch - b_off : kMaxNb;
+  const int nb = p.nb;                                       // MMA N (rows beyond the batch arrive as zeros)
   const uint32_t raw = g_smem_u32(g_smem_raw);
   const uint32_t ring = (raw + 1023u) & ~1023u;             // swizzled tiles need 1024-byte alignment
-  float* stage_f = reinterpret_cast<float*>(g_smem_raw + (ring - raw));   // the ring again, after the last MMA: [nb][128] fp32
-  const uint32_t stage_bytes = kTileABytes + (uint32_t)p.nb * 128u;
-  float2* angles = reinterpret_cast<float2*>(g_smem_raw + (ring - raw) + (size_t)p.stages * stage_bytes);   // [batch][D/2]
+  float* stage_f = reinterpret_cast<float*>(g_smem_raw + (ring - raw));   // the ring again, after the last MMA: [col][128] fp32
+  const uint32_t stage_bytes = kTileABytes + (uint32_t)nb * 128u;
+  const int half = p.D >> 1;
+  float2* angles_s = reinterpret_cast<float2*>(g_smem_raw + (ring - raw) + (size_t)p.stages * stage_bytes);   // [batch_here][D/2]
+  const float2* angles = p.angles_g ? p.angles_g + (size_t)b_off * half : angles_s;   // indexed by the local row
   const int kblocks = (p.k + kBlockK - 1) / kBlockK;
   const int kb0 = (int)((int64_t)kblocks * split / p.ksplit);
   const int kb1 = (int)((int64_t)kblocks * (split + 1) / p.ksplit);
   const int nkb = kb1 - kb0;
   uint32_t ncols = 32;
-  while (ncols < (uint32_t)p.nb) ncols <<= 1;
-  const int cta = blockIdx.y * gridDim.x + blockIdx.x;
+  while (ncols < (uint32_t)nb) ncols <<= 1;
+  const int cta = (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x;
   g_stamp(p, cta, 0);
   if (p.trace && cta < kTraceMaxCtas && tid == 0) {
     uint32_t sm;
@@ -200,7 +268,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
   };
   auto issue_x = [&](int i) {
     const int s = i % p.stages;
-    g_tma_load_2d(ring + (uint32_t)s * stage_bytes + kTileABytes, &map_x, (kb0 + i) * kBlockK, 0, g_smem_u32(&full_bar[s]));
+    g_tma_load_2d(ring + (uint32_t)s * stage_bytes + kTileABytes, &map_x, (kb0 + i) * kBlockK, b_off, g_smem_u32(&full_bar[s]));
   };
 
   if (tid == 0) {
@@ -226,8 +294,9 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
   g_tc_fence_after();
   const uint32_t tmem_d = tmem_slot;
   // Programmatic dependent launch (no-ops without the launch attribute): the next kernel may queue
-  // up now; from here on this one touches what earlier kernels wrote (activations, positions,
-  // partial tiles, tickets), so it waits for them to be complete.
+  // up now; from here on this one touches what earlier kernels wrote (activations, positions, the
+  // angle table, partial tiles, tickets), so it waits for them to be complete.  Every thread of
+  // every CTA passes this wait.
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   asm volatile("griddepcontrol.wait;" ::: "memory");
   g_stamp(p, cta, 1);
@@ -246,7 +315,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     }
   } else if (tid == 32) {
     // ---- MMA issuer ----
-    const uint32_t idesc = g_instr_desc(p.nb);
+    const uint32_t idesc = g_instr_desc(nb);
     bool ok = true;
     for (int i = 0; i < nkb; ++i) {
       const int s = i % p.stages;
@@ -265,20 +334,19 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
       g_umma_commit(g_smem_u32(&empty_bar[s]));         // the slot is free once these MMAs have read it
     }
     if (ok) g_umma_commit(g_smem_u32(&acc_bar));        // the accumulator is complete
-  } else if (tid >= 64 && p.mode == 1 && (tile * kTileM) / p.D < p.Hq + p.Hkv) {
-    // ---- warps 2..15, idle in the main loop: (cos, sin) of position * theta^(-2i/D) for every
-    // sequence and pair i, in double (a float angle is off by 1e-7 * position radians) ----
-    const int half = p.D >> 1, t = tid - 64;
-    double* inv_freq = reinterpret_cast<double*>(angles + (size_t)p.batch * half);
+  } else if (tid >= 64 && p.mode == 1 && p.angles_g == nullptr && (tile * kTileM) / p.D < p.Hq + p.Hkv) {
+    // ---- warps 2..15, idle in the main loop: the (cos, sin) table of this batch tile, in double ----
+    const int t = tid - 64;
+    double* inv_freq = reinterpret_cast<double*>(angles_s + (size_t)batch_here * half);
     for (int i = t; i < half; i += kGemmThreads - 64) inv_freq[i] = exp(-2.0 * i / p.D * p.log_theta);
     asm volatile("bar.sync 1, %0;" ::"n"(kGemmThreads - 64) : "memory");
-    for (int idx = t; idx < p.batch * half; idx += kGemmThreads - 64) {
+    for (int idx = t; idx < batch_here * half; idx += kGemmThreads - 64) {
       const int b = idx / half, i = idx - b * half;
-      int32_t pos = __ldg(p.positions + b);
+      int32_t pos = __ldg(p.positions + b_off + b);
       if (pos < 0) pos = 0;                             // inactive row: any finite value, the row is never appended
       double sn, cn;
       sincos((double)pos * inv_freq[i], &sn, &cn);
-      angles[idx] = make_float2((float)cn, (float)sn);
+      angles_s[idx] = make_float2((float)cn, (float)sn);
     }
   }
   __syncwarp();
@@ -292,7 +360,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
   if (good) {
     g_tc_fence_after();
     const int quad = warp & 3, row = quad * 32 + lane;
-    for (int c0 = 16 * (warp >> 2); c0 < p.nb; c0 += 64) {
+    for (int c0 = 16 * (warp >> 2); c0 < nb; c0 += 64) {
       uint32_t r[16];
       g_tmem_ld16(tmem_d + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0, r);
 #pragma unroll
@@ -304,23 +372,27 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
   if (warp == 1) g_tmem_dealloc(tmem_d, ncols);
   g_stamp(p, cta, 3);
 
-  // ---- split-K: the last CTA of the tile to arrive adds the partial tiles in split order ----
+  // ---- hand-off: the last CTA of a ticket group to arrive reduces the partial tiles in split order ----
+  // A ticket group is the ksplit CTAs of one weight tile, or of the two tiles of a head (group = 2).
   // Ordering: every thread's partial stores happen before the CTA barrier, thread 0's ticket is an
   // acq_rel atomic at gpu scope after it (release is cumulative over the barrier), and the last
   // CTA's threads read only after a second barrier behind that atomic.
+  const bool shared_epilogue = p.ksplit > 1 || p.group > 1;
+  const int ptile = blockIdx.z * gridDim.x + tile;                       // tile index over all batch tiles
+  const size_t split_floats = (size_t)nb * kTileM;                        // one CTA's partial tile
   bool finish = good;
-  if (p.ksplit > 1) {
-    const int n4 = p.batch * kTileM / 4;
-    const size_t split_stride = (size_t)p.nb * kTileM / 4;
-    float4* part = reinterpret_cast<float4*>(p.partials + ((size_t)tile * p.ksplit * p.nb) * kTileM);
+  if (shared_epilogue) {
+    const int n4 = batch_here * kTileM / 4;
+    float4* part = reinterpret_cast<float4*>(p.partials + ((size_t)ptile * p.ksplit + split) * split_floats);
     if (good)
-      for (int i = tid; i < n4; i += kGemmThreads) part[split * split_stride + i] = reinterpret_cast<const float4*>(stage_f)[i];
+      for (int i = tid; i < n4; i += kGemmThreads) part[i] = reinterpret_cast<const float4*>(stage_f)[i];
     __syncthreads();
     if (tid == 0) {
       uint32_t prev;                                           // taken on failure too, so the count always completes
-      asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(p.tickets + tile) : "memory");
-      s_last = prev == (uint32_t)p.ksplit - 1u;
-      if (s_last) p.tickets[tile] = 0;                         // ready for the next launch
+      uint32_t* tk = p.tickets + ptile / p.group;
+      asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(tk) : "memory");
+      s_last = prev == (uint32_t)(p.ksplit * p.group) - 1u;
+      if (s_last) *tk = 0;                                     // ready for the next launch
     }
     __syncthreads();
     g_stamp(p, cta, 4);
@@ -331,79 +403,88 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     return;
   }
 
-  // ---- epilogue set-up (before the reduction, so that its loads overlap the reduction's) ----
-  const int r0 = 2 * (tid & 63), n0 = tile * kTileM + r0;
-  const bool live = n0 < p.n_out;
-  const int half = p.D >> 1;
-  int head = 0, d = 0, hh = 0, H = 1;
-  __nv_bfloat16* base = nullptr;
-  bool rotate = false;
-  if (p.mode == 1 && live) {
-    head = n0 / p.D;
-    d = n0 - head * p.D;
+  // Epilogue of weight tile T over the local batch columns [cb, ce): `val` holds the tile's sums as
+  // [column - cb][128 rows], `par` the sums of the tile that holds the rotation partners (val itself
+  // when a head fits one tile).  Thread = two adjacent weight rows, every kColPhases-th column.
+  auto epilogue = [&](int T, const float* val, const float* par, int cb, int ce) {
+    const int r0 = 2 * (tid & 63), n0 = T * kTileM + r0;
+    if (n0 >= p.n_out) return;
+    if (p.mode == 0) {
+      for (int b = cb + (tid >> 6); b < ce; b += kColPhases) {
+        const float2 v = *reinterpret_cast<const float2*>(&val[(b - cb) * kTileM + r0]);
+        *reinterpret_cast<__nv_bfloat162*>(&p.out[(size_t)(b_off + b) * p.n_out + n0]) = __floats2bfloat162_rn(v.x, v.y);
+      }
+      return;
+    }
+    const int head = n0 / p.D, d = n0 - head * p.D;
+    int hh, H;
+    __nv_bfloat16* base;
     if (head < p.Hq) { base = p.q; hh = head; H = p.Hq; }
     else if (head < p.Hq + p.Hkv) { base = p.kn; hh = head - p.Hq; H = p.Hkv; }
     else { base = p.vn; hh = head - p.Hq - p.Hkv; H = p.Hkv; }
-    rotate = head < p.Hq + p.Hkv;
-  }
-  const int pr = r0 ^ half, i0 = d & (half - 1);
-  const float sgn = d < half ? -1.f : 1.f;      // out_i = x_i c - x_{i+half} s ; out_{i+half} = x_{i+half} c + x_i s
-  const float4* angles4 = reinterpret_cast<const float4*>(angles);   // (cos, sin) of pairs i0 and i0 + 1: 16 bytes
-
-  if (p.ksplit > 1) {
-    // Every other split's values are fetched at once (the reduction would otherwise be a chain of
-    // L2 round trips); this CTA's own are already in shared memory.  Summed in split order, so the
-    // result does not depend on which CTA came last.
-    const int n4 = p.batch * kTileM / 4;
-    const size_t split_stride = (size_t)p.nb * kTileM / 4;
-    const float4* part = reinterpret_cast<const float4*>(p.partials + ((size_t)tile * p.ksplit * p.nb) * kTileM);
-    constexpr int R = 4;
-    for (int ib = tid; ib < n4; ib += R * kGemmThreads) {
-      float4 v[R][kMaxSplit];
+    const bool rotate = head < p.Hq + p.Hkv;
+    const int pr = half < kTileM ? (r0 ^ half) : r0;          // the partner's row in `par`
+    const int i0 = d & (half - 1);
+    const float sgn = d < half ? -1.f : 1.f;      // out_i = x_i c - x_{i+half} s ; out_{i+half} = x_{i+half} c + x_i s
+    const float4* angles4 = reinterpret_cast<const float4*>(angles);   // (cos, sin) of pairs i0 and i0 + 1: 16 bytes
+    // four columns at a time: the angle table may sit in global memory, and four independent loads in
+    // flight per thread keep the loop from being a chain of L2 round trips
+    constexpr int UN = 4;
+    for (int b = cb + (tid >> 6); b < ce; b += UN * kColPhases) {
+      float4 cs[UN];
 #pragma unroll
-      for (int r = 0; r < R; ++r)
-#pragma unroll
-        for (int s = 0; s < kMaxSplit; ++s) {
-          const int i = ib + r * kGemmThreads;
-          if (i < n4 && s < p.ksplit && s != split) v[r][s] = __ldcg(part + s * split_stride + i);
-        }
-#pragma unroll
-      for (int r = 0; r < R; ++r) {
-        const int i = ib + r * kGemmThreads;
-        if (i >= n4) break;
-        const float4 own = reinterpret_cast<const float4*>(stage_f)[i];
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-        for (int s = 0; s < kMaxSplit; ++s)
-          if (s < p.ksplit) {
-            const float4 t = s == split ? own : v[r][s];
-            acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
-          }
-        reinterpret_cast<float4*>(stage_f)[i] = acc;
+      for (int u = 0; u < UN; ++u) {
+        const int bu = b + u * kColPhases;
+        cs[u] = (rotate && bu < ce) ? angles4[(bu * half + i0) >> 1] : make_float4(1.f, 0.f, 1.f, 0.f);
       }
-    }
-    __syncthreads();
-    g_stamp(p, cta, 5);
-  }
-
-  // ---- epilogue: thread = two adjacent weight rows, every kColPhases-th batch column ----
-  if (live) {
-    if (p.mode == 0) {
-      for (int b = tid >> 6; b < p.batch; b += kColPhases) {
-        const float2 v = *reinterpret_cast<const float2*>(&stage_f[b * kTileM + r0]);
-        *reinterpret_cast<__nv_bfloat162*>(&p.out[(size_t)b * p.n_out + n0]) = __floats2bfloat162_rn(v.x, v.y);
-      }
-    } else {
-      for (int b = tid >> 6; b < p.batch; b += kColPhases) {
-        float2 v = *reinterpret_cast<const float2*>(&stage_f[b * kTileM + r0]);
+#pragma unroll
+      for (int u = 0; u < UN; ++u) {
+        const int bu = b + u * kColPhases;
+        if (bu >= ce) break;
+        float2 v = *reinterpret_cast<const float2*>(&val[(bu - cb) * kTileM + r0]);
         if (rotate) {                            // on the fp32 accumulators: one rounding, at the bf16 output
-          const float2 w = *reinterpret_cast<const float2*>(&stage_f[b * kTileM + pr]);
-          const float4 cs = angles4[(b * half + i0) >> 1];
-          v = make_float2(v.x * cs.x + sgn * (w.x * cs.y), v.y * cs.z + sgn * (w.y * cs.w));
+          const float2 w = *reinterpret_cast<const float2*>(&par[(bu - cb) * kTileM + pr]);
+          v = make_float2(v.x * cs[u].x + sgn * (w.x * cs[u].y), v.y * cs[u].z + sgn * (w.y * cs[u].w));
         }
-        *reinterpret_cast<__nv_bfloat162*>(&base[((size_t)b * H + hh) * p.D + d]) = __floats2bfloat162_rn(v.x, v.y);
+        *reinterpret_cast<__nv_bfloat162*>(&base[((size_t)(b_off + bu) * H + hh) * p.D + d]) = __floats2bfloat162_rn(v.x, v.y);
       }
     }
+  };
+
+  // Sum of the ksplit partial tiles of weight tile index `pt` (over all batch tiles) for the local columns
+  // [cb, ce), in split order, into dst[column - cb][128].  `own`: this CTA's own partial of that tile is still
+  // in shared memory at `dst` (cb = 0) and is taken from there.
+  auto reduce_tile = [&](int pt, float* dst, int cb, int ce, bool own) {
+    const float4* part = reinterpret_cast<const float4*>(p.partials + (size_t)pt * p.ksplit * split_floats) + (size_t)cb * kTileM / 4;
+    gemm_reduce_partials(part, reinterpret_cast<float4*>(dst), (ce - cb) * kTileM / 4, p.ksplit, own ? split : -1, split_floats / 4);
+  };
+
+  if (p.group == 1) {
+    if (p.ksplit > 1) {
+      // Every other split's values are fetched at once (the reduction would otherwise be a chain of
+      // L2 round trips); this CTA's own are already in shared memory.  Summed in split order, so the
+      // result does not depend on which CTA came last.
+      reduce_tile(ptile, stage_f, 0, batch_here, true);
+      __syncthreads();
+      g_stamp(p, cta, 5);
+    }
+    epilogue(tile, stage_f, stage_f, 0, batch_here);
+  } else {
+    // Two tiles of one head: both are reduced from the partial tiles in global memory (this CTA's own
+    // included), kChunkCols batch columns at a time so that both fit the ring's shared memory.
+    const int t0 = tile & ~1;                                  // first tile of the head
+    float* buf0 = stage_f;
+    float* buf1 = stage_f + (size_t)kChunkCols * kTileM;
+    for (int cb = 0; cb < batch_here; cb += kChunkCols) {
+      const int ce = cb + kChunkCols < batch_here ? cb + kChunkCols : batch_here;
+      __syncthreads();                                         // the previous chunk's epilogue is done with the buffers
+      reduce_tile(blockIdx.z * gridDim.x + t0, buf0, cb, ce, false);
+      reduce_tile(blockIdx.z * gridDim.x + t0 + 1, buf1, cb, ce, false);
+      __syncthreads();
+      epilogue(t0, buf0, buf1, cb, ce);
+      epilogue(t0 + 1, buf1, buf0, cb, ce);
+    }
+    g_stamp(p, cta, 5);
   }
   g_stamp(p, cta, 6);
 }

@@ -101,7 +101,7 @@ def run_module(seed, lens, Hq, Hkv, D, hidden, steps=2, inactive=(), window=0, b
         rq, rk, rv = afd.project_qkv(x, w_qkv, pos, Hq, Hkv, D, THETA)
         u = 2.0 ** -8
         E = hidden * 2.0 ** -24 * float(np.sqrt(np.mean(rv[act] ** 2))) + 1e-30
-        library = bool(flags & B.OPW_AFD_LIBRARY_GEMM) or nb > 96 or D == 256     # what the module switches to the library for
+        library = bool(flags & B.OPW_AFD_LIBRARY_GEMM)           # the comparison arm; everything else is the tensor-core kernel
         pre = u if library else 0.0                          # the library path's extra rounding before the rotation
         for name, got, ref in (("q", f64(gq), rq), ("k", f64(gk), rk)):
             partner = np.concatenate([ref[..., D // 2:], ref[..., :D // 2]], axis=-1)
@@ -145,6 +145,7 @@ def run_module(seed, lens, Hq, Hkv, D, hidden, steps=2, inactive=(), window=0, b
         assert (err <= 2.0 ** -5 * rms + 2.0 ** -8 * np.abs(e2e_y)).all(), (err.max(), rms)
         assert err[act].mean() <= 2.0 ** -7 * rms, (err[act].mean(), rms)
         worst["y_rel"] = max(worst.get("y_rel", 0.0), float(err.max() / rms))
+    worst["launches"] = mod.launch_count() // steps
     mod.close()
     stage.close()
     return worst
@@ -163,10 +164,10 @@ def test_module_on_a_sliding_window_layer():
     run_module(5, [30, 100, 2000], 8, 2, 64, 256, steps=2, window=64)
 
 
-def test_module_with_programmatic_dependent_launch_over_back_to_back_steps():
-    """Projections launched with the attribute: the appended rows, q and y of every step are checked
-    after steps were enqueued without a host synchronisation in between."""
-    run_module(17, [40, 900, 33, 2047], 16, 4, 128, 1024, steps=3, flags=B.OPW_AFD_PDL)
+def test_module_without_programmatic_dependent_launch():
+    """The projections are launched with programmatic dependent launch by default (every other test);
+    this is the opt-out: same checks with plain stream order."""
+    run_module(17, [40, 900, 33, 2047], 16, 4, 128, 1024, steps=3, flags=B.OPW_AFD_NO_PDL)
 
 
 @BOTH
@@ -174,13 +175,22 @@ def test_llama8b_layer_shape_and_a_batch_that_changes_between_steps(flags):
     run_module(21, [17, 900, 33, 2047, 512, 64, 5, 1200], 32, 8, 128, 4096, steps=3, batches=[8, 3, 8], flags=flags)
 
 
-def test_batches_of_one_row_and_around_the_switch_to_the_library_path():
-    """One row uses the narrowest accumulator (16 columns), 96 rows the widest the tensor-core path
-    takes (six column chunks), 97 and 300 rows go to the library path inside the same module."""
-    run_module(31, [77], 8, 2, 128, 512, steps=2)
-    rng = np.random.default_rng(32)
-    for n in (96, 97, 300):
-        run_module(33 + n, list(rng.integers(1, 60, n)), 8, 2, 64, 256, steps=1, inactive=(0, n - 1))
+@pytest.mark.parametrize("D", [64, 128, 256])
+def test_batch_sizes_from_one_row_to_several_batch_tiles(D):
+    """One row uses the narrowest accumulator (16 columns); 96 rows is the largest batch whose angle table
+    is computed inside the kernel, 97 the first that reads it from global memory; 128 and 256 fill one
+    batch tile (at head_dim 256 the two-tile epilogue then runs in one and two column chunks); 300 rows
+    need two batch tiles.  All on the tensor-core kernel."""
+    run_module(31, [77], 8, 2, D, 512, steps=2)
+    rng = np.random.default_rng(32 + D)
+    for n in (64, 96, 97, 128, 256, 300):
+        w = run_module(33 + n, list(rng.integers(1, 60, n)), 4, 2, D, 256, steps=1, inactive=(0, n - 1))
+        assert w["launches"] == (2 if n <= 96 else 3)          # two projections, and the angle-table kernel above 96 rows
+
+
+def test_library_arm_at_large_batch_and_head_dim_256():
+    rng = np.random.default_rng(35)
+    run_module(36, list(rng.integers(1, 60, 130)), 4, 2, 256, 256, steps=1, flags=B.OPW_AFD_LIBRARY_GEMM)
 
 
 def test_the_two_projection_paths_agree():
