@@ -149,9 +149,17 @@ inline int ksplit_of(int n_out, int k, int batch, int sms) {
   if (ks > kblocks) ks = kblocks;
   return ks < 1 ? 1 : ks;
 }
-inline size_t partial_bytes(int n_out, int k, int batch) {
-  // the widest split any device can pick (an upper bound over SM counts), every batch tile
-  return (size_t)tiles_of(n_out) * batch_tiles_of(batch) * opw_afd::kMaxSplit * nb_of(batch) * opw_afd::kTileM * sizeof(float);
+inline size_t partial_bytes_at(int n_out, int k, int batch) {
+  return (size_t)tiles_of(n_out) * batch_tiles_of(batch) * ksplit_of(n_out, k, batch, kSmsBound) * nb_of(batch) *
+         opw_afd::kTileM * sizeof(float);
+}
+// Partial tiles of any batch up to max_batch on any device of at most kSmsBound SMs (more SMs split K further, never
+// beyond kMaxSplit).  Up to 256 rows the need grows with the batch; beyond, the batch tiles multiply while the
+// K-split falls to one, so the largest need is at 256 rows or at max_batch.
+inline size_t partial_bytes(int n_out, int k, int max_batch) {
+  const size_t a = partial_bytes_at(n_out, k, max_batch < opw_afd::kMaxNb ? max_batch : opw_afd::kMaxNb);
+  const size_t b = partial_bytes_at(n_out, k, max_batch);
+  return a > b ? a : b;
 }
 
 struct Carve { size_t qkv, q, k, v, out, gemm, partials, tickets, angles, status, total; };
