@@ -283,12 +283,12 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
     stack = wl.num_layers > 1                       # the hybrid stack: a step runs all its layers
     R = wl.num_layers if stack else rotate
     e2e_steps = max(3, min(steps, 200)) if want_e2e else 0
-    n_timed = warmup + steps + (e2e_steps + 3 if want_e2e else 0)
+    n_timed = warmup + steps + (e2e_steps + max(3, rotate) if want_e2e else 0)
     n_used = n_timed                                 # steps the call-by-call and host-buffer loops take
     # a plan submission advances every layer by one token; two plans run, each 3 warm-up submissions + n_sub timed
     n_sub = (steps if stack else max(steps // R, 10)) if want_submit else 0
-    if want_e2e and world == 1 and not stack and R % 2 == 0:
-        n_used += e2e_steps + 8                      # the two-microbatch host-buffer loop
+    if want_e2e and world == 1 and not stack and R >= 2:
+        n_used += e2e_steps + 2 * R + 8              # the two-microbatch host-buffer loop
     rounds = (n_used if stack else (n_used + R - 1) // R) + (2 * (3 + n_sub) + 2 if want_submit else 0)
     wl_r, inp, st, pos_all, len_all = build_stage(wl, R, rounds, dev, tune)
     B, Hq, Hkv, D = wl.batch, wl.num_q_heads, wl.num_kv_heads, wl.head_dim
@@ -410,7 +410,10 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
 
     if want_e2e:
         # q, k_new, v_new and positions of one call sit in one pinned buffer at the stage's packed
-        # offsets (they travel as one copy); the page table and the output have buffers of their own
+        # offsets (they travel as one copy); the output has a pinned buffer of its own.  The page table is
+        # handled as a server would: sent in full when a sequence set is admitted to a layer (with nothing
+        # mapped beyond the page the next token goes to; that happens in the untimed warm-up), and after that
+        # only the (row, logical page, physical page) triple of every sequence whose new token opens a page.
         packs = [[st.packed_host_buffers(B) for _ in range(R)] for _ in range(2)]
         for i in range(2):
             for l in range(R):
@@ -419,25 +422,77 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
                 pk.copy_(inp.k_new[i, l].cpu())
                 pv.copy_(inp.v_new[i, l].cpu())
         hpos = pos_all.cpu()
-        htab = [t.cpu().pin_memory() for t in inp.page_tables]
+        hpos_np = hpos.numpy()
+        pos_views = {}                                 # numpy views of the packed buffers' position fields (a 64-byte host write per step)
+
+        def write_positions(ppos, t):
+            v = pos_views.get(ppos.data_ptr())
+            if v is None:
+                v = pos_views[ppos.data_ptr()] = ppos.numpy()
+            v[:] = hpos_np[t]
+
+        full_tab = [t.cpu().numpy() for t in inp.page_tables]
         hout = torch.empty(B, Hq, D, dtype=torch.bfloat16).pin_memory()
         base = warmup + steps
+        keep_alive = []                                # pinned tables and triples of copies that may still be in flight
+
+        def admission_table(l, t):
+            tab = full_tab[l].copy()
+            beyond = np.arange(tab.shape[1])[None, :] > (hpos_np[t].astype(np.int64) // 16)[:, None]
+            tab[beyond] = -1
+            ten = torch.from_numpy(tab).pin_memory()
+            keep_alive.append(ten)
+            return ten
+
+        deltas = {}                                    # (layer, round) -> pinned int32 [n, 3], for rounds whose token opens a page
+
+        def delta_of(l, t):
+            key = (l, t)
+            if key not in deltas:
+                rows = np.nonzero(hpos_np[t] % 16 == 0)[0]
+                if len(rows) == 0:
+                    deltas[key] = None
+                else:
+                    lp = hpos_np[t][rows].astype(np.int64) // 16
+                    tri = np.stack([rows, lp, full_tab[l][rows, lp]], axis=1).astype(np.int32)
+                    deltas[key] = torch.from_numpy(tri).pin_memory()
+            return deltas[key]
+
+        for l in range(R):                             # built before any timed region
+            for t in range(pos_all.shape[0]):
+                delta_of(l, t)
+        admitted = {}                                  # stage handle -> layers whose table it holds
+        delta_bytes = [0]
+
+        def send_table(stage, l, t):
+            """The page_table_host argument of this visit, after any delta call it needs."""
+            seen = admitted.setdefault(id(stage), set())
+            if l not in seen:
+                seen.add(l)
+                return admission_table(l, t)
+            tri = delta_of(l, t)
+            if tri is not None:
+                stage.page_table_delta_host(l, tri)
+                delta_bytes[0] += tri.numel() * 4
+            return None
 
         def host_step(s):
             layers, t = layer_round(s)
             for l in layers:
                 _, pq, pk, pv, ppos = packs[s & 1][l]
-                ppos.copy_(hpos[t])                  # this step's positions, written by the host
-                st.decode_step_host(l, pq, pk, pv, ppos, htab[l], hout)
+                write_positions(ppos, t)             # this step's positions, written by the host
+                st.decode_step_host(l, pq, pk, pv, ppos, send_table(st, l, t), hout)
             stream.synchronize()                     # the caller reads the result every step
 
-        for s in range(base, base + 3):
+        warm = max(3, 1 if stack else R)             # every layer is admitted (its table sent in full) before timing
+        for s in range(base, base + warm):
             host_step(s)
         barrier()
         torch.cuda.synchronize()
+        delta_bytes[0] = 0
         w0 = time.perf_counter()
         t0.record(stream)
-        for s in range(base + 3, base + 3 + e2e_steps):
+        for s in range(base + warm, base + warm + e2e_steps):
             host_step(s)
         t1.record(stream)
         torch.cuda.synchronize()
@@ -449,19 +504,24 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
             tmax = torch.tensor([e_ms], dtype=torch.float64, device=dev if dist.get_backend() == "nccl" else "cpu")
             dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
             e_ms = float(tmax.item())
-        e_bytes = sum(kv_bytes_of_step(s) for s in range(base + 3, base + 3 + e2e_steps))
-        h2d = layers_per_step * (B * Hq * D * 2 + 2 * B * Hkv * D * 2 + B * 4 + htab[0].numel() * 4)
+        e_bytes = sum(kv_bytes_of_step(s) for s in range(base + warm, base + warm + e2e_steps))
+        packed = layers_per_step * (B * Hq * D * 2 + 2 * B * Hkv * D * 2 + B * 4)
+        h2d = packed + delta_bytes[0] / e2e_steps
         d2h = layers_per_step * hout.numel() * 2
         assert st.poll_error() == binding.OPW_OK
+        table_note = ("sent in full at admission (untimed warm-up); inside the timed region 12 bytes per page a sequence opens, "
+                      f"{delta_bytes[0] / e2e_steps:.1f} bytes per step on average")
         res["e2e"] = {"value": round(world * e_bytes / (e_ms * 1e-3) / 1e9, 1), "unit": "GB/s", "steps": e2e_steps,
-                      "ms_per_step": round(e_ms / e2e_steps, 5), "h2d_bytes_per_step": int(h2d),
-                      "d2h_bytes_per_step": int(d2h)}
-    if want_e2e and world == 1 and not stack and R % 2 == 0:
+                      "ms_per_step": round(e_ms / e2e_steps, 5), "h2d_bytes_per_step": int(round(h2d)),
+                      "d2h_bytes_per_step": int(d2h), "page_table": table_note,
+                      "frac_of_value": round(world * e_bytes / (e_ms * 1e-3) / 1e9 / value, 4)}
+    if want_e2e and world == 1 and not stack and R >= 2:
         # The same host-buffer steps with two microbatches in flight (the paper keeps mu microbatches resident
-        # on a stage so that transfers hide behind compute): even steps belong to microbatch A (even layer
-        # pools, stage handle `st`, stream A), odd steps to B (odd pools, a second handle with its own
-        # workspace, stream B).  Every step still copies its inputs in and its output out; the host waits
+        # on a stage so that transfers hide behind compute): even steps belong to microbatch A (stage handle
+        # `st`, stream A), odd steps to B (a second handle with its own workspace and staged tables, stream
+        # B), over disjoint layer pools.  Every step still copies its inputs in and its output out; the host waits
         # for a microbatch's previous step (and reads its result) before it reuses that microbatch's buffers.
+        Re = R - R % 2                                        # an even number of pools: half for each microbatch
         st2 = binding.Stage(pools=inp.pools, layer_window=wl_r.layer_window, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D,
                             max_batch=B, max_pages_per_seq=inp.max_pages_per_seq, **tune)
         packs2 = [[(st, st2)[l & 1].packed_host_buffers(B) for l in range(R)] for _ in range(2)]
@@ -473,34 +533,41 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
                 pv.copy_(inp.v_new[i, l].cpu())
         houts = [torch.empty(B, Hq, D, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
         streams = [torch.cuda.Stream(), torch.cuda.Stream()]
-        base2 = base + 3 + e2e_steps
-        base2 += base2 % 2                                    # start on an even step
+        # This loop has its own step numbering: step s2 visits pool s2 % Re at round r0 + s2 // Re, r0 the first round
+        # no pool has been appended at yet; an even pool belongs to microbatch A, an odd one to B.
+        r0 = (base + warm + e2e_steps + R - 1) // R
+        admitted.clear()                                      # rounds were skipped: both handles take their tables afresh
 
         def host_step_mb(s2):
-            layers, t = layer_round(s2)
-            mb = s2 & 1
+            l, t = s2 % Re, r0 + s2 // Re
+            mb = l & 1
             streams[mb].synchronize()                         # this microbatch's previous result is on the host now
             with torch.cuda.stream(streams[mb]):
-                for l in layers:
-                    _, pq, pk, pv, ppos = packs2[(s2 >> 1) & 1][l]
-                    ppos.copy_(hpos[t])
-                    (st, st2)[mb].decode_step_host(l, pq, pk, pv, ppos, htab[l], houts[mb])
+                _, pq, pk, pv, ppos = packs2[(s2 >> 1) & 1][l]
+                write_positions(ppos, t)
+                stage = (st, st2)[mb]
+                stage.decode_step_host(l, pq, pk, pv, ppos, send_table(stage, l, t), houts[mb])
+            return inp.kv_bytes(l, t)
 
-        n2 = min(e2e_steps, (rounds * R - base2 - 4) // 2 * 2)
+        warm2 = max(4, Re)
+        n2 = min(e2e_steps, ((pos_all.shape[0] - 1 - r0) * Re - warm2) // 2 * 2)
         if n2 >= 4:
-            for s2 in range(base2, base2 + 4):
+            for s2 in range(warm2):
                 host_step_mb(s2)
             torch.cuda.synchronize()
+            delta_bytes[0] = 0
+            mb_bytes = 0
             w0 = time.perf_counter()
-            for s2 in range(base2 + 4, base2 + 4 + n2):
-                host_step_mb(s2)
+            for s2 in range(warm2, warm2 + n2):
+                mb_bytes += host_step_mb(s2)
             torch.cuda.synchronize()
             mb_ms = (time.perf_counter() - w0) * 1e3
-            mb_bytes = sum(kv_bytes_of_step(s2) for s2 in range(base2 + 4, base2 + 4 + n2))
             assert st.poll_error() == binding.OPW_OK and st2.poll_error() == binding.OPW_OK
-            res["e2e_two_microbatches"] = {"value": round(mb_bytes / (mb_ms * 1e-3) / 1e9, 1), "unit": "GB/s", "steps": n2,
+            v2 = mb_bytes / (mb_ms * 1e-3) / 1e9
+            res["e2e_two_microbatches"] = {"value": round(v2, 1), "unit": "GB/s", "steps": n2,
                                            "ms_per_step": round(mb_ms / n2, 5), "timing": "wall clock, device synchronised at both ends",
-                                           "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h)}
+                                           "h2d_bytes_per_step": int(round(packed + delta_bytes[0] / n2)), "d2h_bytes_per_step": int(d2h),
+                                           "frac_of_value": round(v2 / value, 4)}
         st2.close()
     if want_submit:
         # The same steps through a plan: one native call (one CUDA graph launch) per pass over
@@ -798,6 +865,7 @@ def main():
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--ctas", type=int, default=0)
     ap.add_argument("--unfused", action="store_true", help="separate opw_kv_append + opw_decode_attention calls")
+    ap.add_argument("--module-layers", type=int, default=4, help="layers (weights and KV pools) --workload attention_module cycles through")
     ap.add_argument("--module-batch", type=int, default=0, help="batch rows of --workload attention_module (default: the shape's own)")
     ap.add_argument("--no-pdl", action="store_true", help="launch the kernels without programmatic stream serialisation")
     args = ap.parse_args()
@@ -834,7 +902,7 @@ def main():
     steps = args.steps if args.steps is not None else 2000
     warmup = args.warmup if args.warmup is not None else 20
     if args.workload == "attention_module":         # the AFD partition's stage alone (1 GPU)
-        r = run_afd_module(max(8, min(steps, 2000)), batch=args.module_batch)
+        r = run_afd_module(max(8, min(steps, 2000)), batch=args.module_batch, layers=args.module_layers)
         r.update({"metric": "attention module decode: sequence-steps/s per layer", "n_gpus": 1, "warmup": 8,
                   "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
                   "gpu_launches": r["steps"] * 4})

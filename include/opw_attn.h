@@ -213,6 +213,23 @@ opw_status_t opw_decode_step_host(opw_attn_stage_t *stage, int32_t layer, int32_
                                   void *cuda_stream);
 
 /*
+ * Page-table delta from HOST memory (Section 6, first paragraph: only token, position and KV-cache
+ * metadata change between iterations; Section 6.2, low-overhead communication: many short transfers
+ * cost more than the bytes they carry).  A sequence gets a new page once every page_size steps, so
+ * re-sending its whole table row each step moves thousands of entries to change one.  This call
+ * updates the table that opw_decode_step_host keeps staged for `layer` (the one its
+ * page_table_host == NULL reuses): triples_host is int32 [n][3] = (batch row, logical page, physical
+ * page), copied with one transfer and scattered by one small kernel, both enqueued on the stream;
+ * the host array must stay valid until the stream has passed the copy (pinned for an asynchronous
+ * copy).  The staged table must have been sent in full once (opw_decode_step_host with a non-NULL
+ * page_table_host).  n == 0 enqueues nothing.  n > 4 * max_batch: OPW_ERR_CAPACITY.  A row or a
+ * logical page outside the table is skipped and recorded as OPW_ERR_BAD_PAGE in the status word; the
+ * physical page id is checked when a step reads it, as for any table.
+ */
+opw_status_t opw_attn_stage_page_table_delta_host(opw_attn_stage_t *stage, int32_t layer, const int32_t *triples_host,
+                                                  int32_t n, void *cuda_stream);
+
+/*
  * Plans: the per-token action sequence of a stage, enqueued by ONE native call (Section 6.2,
  * "Single native submission": the complete per-rank sequence is compiled once and each token
  * enqueues all graph launches with no host dispatch between stages and microbatches; Section 6,

@@ -30,6 +30,7 @@ EXPORTS = [
     "opw_decode_attention_noalloc", "opw_attn_plan_create", "opw_attn_plan_submit", "opw_attn_plan_destroy",
     "opw_decode_step", "opw_attn_stage_host_layout", "opw_attn_stage_probe_timeout",
     "opw_linear_attn_decode_step", "opw_linear_attn_state_bytes", "opw_attn_plan_create_mixed",
+    "opw_attn_stage_page_table_delta_host",
     "opw_attn_stage_shape", "opw_afd_module_workspace_bytes", "opw_afd_module_create", "opw_afd_module_step",
     "opw_afd_module_intermediates", "opw_afd_module_destroy", "opw_afd_module_poll_error",
     "opw_afd_module_launch_count", "opw_afd_module_set_trace", "opw_hbm_read_probe",
@@ -155,6 +156,8 @@ def lib() -> ctypes.CDLL:
     L.opw_attn_stage_host_layout.argtypes = [vp] + [ctypes.POINTER(ctypes.c_size_t)] * 5
     L.opw_decode_step_host.restype = ctypes.c_int
     L.opw_decode_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.opw_attn_stage_page_table_delta_host.restype = ctypes.c_int
+    L.opw_attn_stage_page_table_delta_host.argtypes = [vp, i32, vp, i32, vp]
     L.opw_linear_attn_decode_step.restype = ctypes.c_int
     L.opw_linear_attn_decode_step.argtypes = [i32, i32, i32, i32, i32, vp, i64, vp, vp, vp, vp, vp, vp, ctypes.c_float, vp, vp]
     L.opw_linear_attn_state_bytes.restype = ctypes.c_size_t
@@ -300,6 +303,13 @@ def opw_decode_step_host(stage: int, layer: int, batch: int, q_host: int, k_new_
                          lse_host: Optional[int] = None, stream: Optional[int] = None) -> None:
     _check(lib().opw_decode_step_host(stage, layer, batch, q_host, k_new_host, v_new_host, positions_host,
                                       page_table_host, out_host, lse_host, stream), "opw_decode_step_host")
+
+
+def opw_attn_stage_page_table_delta_host(stage: int, layer: int, triples_host: int, n: int,
+                                         stream: Optional[int] = None) -> None:
+    """triples_host: host address of int32 [n][3] = (batch row, logical page, physical page)."""
+    _check(lib().opw_attn_stage_page_table_delta_host(stage, layer, triples_host, n, stream),
+           "opw_attn_stage_page_table_delta_host")
 
 
 def opw_decode_attention_noalloc(*, num_q_heads: int, num_kv_heads: int, head_dim: int, kv_pool: int, num_pages: int,
@@ -512,6 +522,10 @@ class Stage:
         opw_decode_step_host(self.handle, layer, positions.shape[0], q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(),
                              positions.data_ptr(), None if page_table is None else page_table.data_ptr(),
                              out.data_ptr(), None if lse is None else lse.data_ptr(), self._stream())
+
+    def page_table_delta_host(self, layer, triples):
+        """triples: int32 host tensor [n, 3] of (batch row, logical page, physical page), pinned for an asynchronous copy."""
+        opw_attn_stage_page_table_delta_host(self.handle, layer, triples.data_ptr(), int(triples.shape[0]), self._stream())
 
     def enable_trace(self):
         """Allocate a trace buffer (torch) and switch per-worker tracing on; returns the int64 tensor [workers, 4]."""

@@ -21,6 +21,7 @@ constexpr int kDefaultWarps = 8;
 constexpr int kDefaultStages = 2;
 constexpr int kDefaultCtasPerSm = 1;
 constexpr size_t kSmemLimit = 227 * 1024;
+constexpr size_t kDeltaPerRow = 4;               // page-table delta entries one call may carry, per static batch slot
 constexpr int kCombineScratchSlots = 1024;       // rows * splits of the split combine never exceed this
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -30,7 +31,7 @@ struct Shape {
 };
 
 struct Layout {          // byte offsets into the caller's workspace
-  size_t status, cum[2], partials[2], comb_scratch, row_count, st_q, st_k, st_v, st_pos, st_out, st_lse, st_table, total;
+  size_t status, cum[2], partials[2], comb_scratch, row_count, st_q, st_k, st_v, st_pos, st_out, st_lse, st_delta, st_table, total;
 };
 
 bool shape_ok(const opw_attn_stage_config_t* c) {
@@ -76,6 +77,7 @@ Layout carve(const opw_attn_stage_config_t* c, const Shape& s, int sms) {
   L.st_pos = off;  off += align_up(B * 4, 256);
   L.st_out = off;  off += align_up(B * Hq * D * 2, 256);
   L.st_lse = off;  off += align_up(B * Hq * 4, 256);
+  L.st_delta = off; off += align_up(kDeltaPerRow * B * 12, 256);
   L.st_table = off; off += align_up((size_t)c->num_layers * B * c->max_pages_per_seq * 4, 256);
   L.total = off;
   return L;
@@ -545,6 +547,26 @@ opw_status_t opw_decode_step_host(opw_attn_stage_t* st, int32_t layer, int32_t b
   ok &= cudaMemcpyAsync(out_host, d_out, B * Hq * D * 2, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
   if (lse_host) ok &= cudaMemcpyAsync(lse_host, d_lse, B * Hq * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
   if (!ok) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
+  return OPW_OK;
+}
+
+opw_status_t opw_attn_stage_page_table_delta_host(opw_attn_stage_t* st, int32_t layer, const int32_t* triples_host,
+                                                  int32_t n, void* cuda_stream) {
+  if (!st || layer < 0 || layer >= st->cfg.num_layers || n < 0 || (n > 0 && !triples_host)) return OPW_ERR_INVALID_ARG;
+  if ((size_t)n > kDeltaPerRow * (size_t)st->cfg.max_batch) return OPW_ERR_CAPACITY;
+  if (n == 0) return OPW_OK;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  int32_t* d_tri = reinterpret_cast<int32_t*>(st->ws + st->lay.st_delta);
+  const size_t table_elems = (size_t)st->cfg.max_batch * st->cfg.max_pages_per_seq;
+  int32_t* d_table = reinterpret_cast<int32_t*>(st->ws + st->lay.st_table) + (size_t)layer * table_elems;
+  if (cudaMemcpyAsync(d_tri, triples_host, (size_t)n * 12, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+    (void)cudaGetLastError();
+    return OPW_ERR_CUDA;
+  }
+  opw::table_delta_kernel<<<(n + 255) / 256, 256, 0, stream>>>(d_table, d_tri, n, st->cfg.max_batch, st->cfg.max_pages_per_seq,
+                                                               reinterpret_cast<uint32_t*>(st->ws + st->lay.status));
+  if (cudaGetLastError() != cudaSuccess) return OPW_ERR_CUDA;
+  st->launches += 1;
   return OPW_OK;
 }
 

@@ -301,6 +301,20 @@ __global__ void advance_kernel(int32_t* positions, int32_t* kv_lens, int32_t n) 
   }
 }
 
+// Page-table delta: entry i of `triples` is (batch row, logical page, physical page); the staged table of a
+// layer takes the new mapping.  Entries outside the table are skipped and recorded.
+__global__ void table_delta_kernel(int32_t* table, const int32_t* triples, int32_t n, int32_t max_batch, int32_t max_pages,
+                                   uint32_t* status) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const int32_t row = triples[3 * i], lp = triples[3 * i + 1], pid = triples[3 * i + 2];
+  if (row < 0 || row >= max_batch || lp < 0 || lp >= max_pages) {
+    atomicOr(status, kErrBadPage);
+    return;
+  }
+  table[(int64_t)row * max_pages + lp] = pid;
+}
+
 // Self-test of the bounded wait: one warp arms a shared-memory barrier for bytes that no copy
 // will ever deliver, waits for it the way the attention kernel waits for a tile, and must come
 // back after kWaitLimitNs with the time-out recorded in the status word.  Nothing is in

@@ -469,6 +469,72 @@ def test_host_buffer_step_matches_the_device_step():
     st.close()
 
 
+def test_host_steps_with_page_table_deltas_equal_steps_with_the_table_resent_in_full():
+    """Forty decode steps from host buffers, twice: once re-sending the whole page table every step, once sending it
+    in full at the first step only (with the pages of later steps still unmapped) and from then on just the
+    (row, logical page, physical page) triple of every sequence that crosses into a new page.  Pools and outputs
+    must agree bit for bit, and with the oracle at the end."""
+    steps = 40
+    wl = synth.Workload("pd", 5, 32, 8, 128, [0, 64], "uniform_1024_4096", 84)
+    lens = np.array([5, 200, 1023, 64, 15], np.int32)
+    inp = synth.make_inputs(wl, device="cpu", growth=steps, steps=steps, lengths=lens)
+    results = []
+    for use_delta in (False, True):
+        pools = [p.clone().cuda() for p in inp.pools]
+        st = B.Stage(pools=pools, layer_window=wl.layer_window, num_q_heads=32, num_kv_heads=8, head_dim=128,
+                     max_batch=5, max_pages_per_seq=inp.max_pages_per_seq)
+        outs = torch.empty(steps, 2, 5, 32, 128, dtype=torch.bfloat16).pin_memory()
+        tri = torch.empty(steps, 2, 5, 3, dtype=torch.int32).pin_memory()
+        sent = 0
+        for step in range(steps):
+            pos_np = inp.positions(step)
+            for layer in range(2):
+                _, q, k, v, pos = st.packed_host_buffers(5)
+                q.copy_(inp.q[step, layer]); k.copy_(inp.k_new[step, layer]); v.copy_(inp.v_new[step, layer])
+                pos.copy_(torch.from_numpy(pos_np))
+                full = inp.page_tables[layer]
+                if not use_delta:
+                    tab = full.clone().pin_memory()
+                elif step == 0:                                  # the table as a server holds it at admission: nothing
+                    tab = full.clone()                            # mapped beyond the page the first token goes to
+                    for b in range(5):
+                        tab[b, int(pos_np[b]) // P + 1:] = -1
+                    tab = tab.pin_memory()
+                else:
+                    tab = None
+                    rows = [b for b in range(5) if int(pos_np[b]) % P == 0]       # this step's token opens a new page
+                    for i, b in enumerate(rows):
+                        lp = int(pos_np[b]) // P
+                        tri[step, layer, i] = torch.tensor([b, lp, int(full[b, lp])], dtype=torch.int32)
+                    st.page_table_delta_host(layer, tri[step, layer, :len(rows)])
+                    sent += len(rows)
+                st.decode_step_host(layer, q, k, v, pos, tab, outs[step, layer])
+                assert st.poll_error() == B.OPW_OK
+        results.append((outs.clone(), [p.cpu() for p in pools]))
+        if use_delta:
+            assert sent == 2 * sum((int(n) + steps - 1) // P - int(n) // P for n in lens)      # one triple per page opened
+            with pytest.raises(B.OpwError) as e:
+                B.opw_attn_stage_page_table_delta_host(st.handle, 0, tri.data_ptr(), 4 * 5 + 1)
+            assert e.value.status == B.OPW_ERR_CAPACITY
+            bad = torch.tensor([[7, 0, 0], [0, 10 ** 6, 0]], dtype=torch.int32).pin_memory()     # row / logical page outside the table
+            st.page_table_delta_host(0, bad)
+            assert st.poll_error() == B.OPW_ERR_BAD_PAGE
+        st.close()
+    assert torch.equal(results[0][0].view(torch.int16), results[1][0].view(torch.int16))
+    for a, b in zip(results[0][1], results[1][1]):
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    refs = [oracle.as_u16(p).copy() for p in inp.pools]
+    for step in range(steps):
+        for layer in range(2):
+            assert oracle.kv_append(refs[layer], 8, 128, P, inp.k_new[step, layer], inp.v_new[step, layer],
+                                    inp.positions(step), inp.page_tables[layer]) == 0
+    for layer in range(2):
+        assert (oracle.as_u16(results[1][1][layer]) == refs[layer]).all()
+        ref, _, _ = oracle.decode_attention(refs[layer], 32, 8, 128, P, inp.q[steps - 1, layer], inp.kv_lens(steps - 1),
+                                            inp.page_tables[layer], window=wl.layer_window[layer])
+        check_close(out_to_f64(results[1][0][steps - 1, layer]), ref)
+
+
 @pytest.mark.parametrize("fused", [False, True])
 @pytest.mark.parametrize("flags", [0, B.OPW_PLAN_GRAPH, B.OPW_PLAN_GRAPH | B.OPW_PLAN_ADVANCE, B.OPW_PLAN_ADVANCE,
                                    B.OPW_PLAN_OVERLAP, B.OPW_PLAN_GRAPH | B.OPW_PLAN_ADVANCE | B.OPW_PLAN_OVERLAP])
