@@ -116,7 +116,7 @@ struct opw_afd_module {
   unsigned char* ws;
   size_t off_qkv, off_q, off_k, off_v, off_out, off_gemm, off_partials, off_tickets, off_angles, off_status;
   // tensor-core path
-  bool tc_qkv, tc_o, pdl;
+  bool tc_qkv, tc_o, pdl, coop_ok;
   int sms;
   TensorMapEncodeFn encode;
   CUtensorMap map_wqkv, map_wo;
@@ -136,6 +136,7 @@ constexpr int kSmsBound = 160;             // split-K sizing assumes no more SMs
 // the ring; above it the table (batch * D/2 * 8 bytes) would crowd the ring out, so a small kernel
 // writes it to global memory first.
 constexpr int kSmemAngleBatch = 96;
+constexpr int kCoopMinBatch = 128;         // above this batch the CTAs of a tile share the back end (cooperative launch)
 constexpr size_t kGemmSmemBudget = 226 * 1024;
 
 inline int round16(int x) { return (x + 15) / 16 * 16; }
@@ -180,7 +181,7 @@ Carve carve(int Hq, int Hkv, int D, int max_batch, int hidden) {
   c.partials = take(p1 > p2 ? p1 : p2);
   c.angles = take((size_t)max_batch * (D / 2) * sizeof(float2));
   const int t1 = tiles_of(n_qkv), t2 = tiles_of(hidden);
-  c.tickets = take((size_t)(t1 > t2 ? t1 : t2) * batch_tiles_of(max_batch) * sizeof(uint32_t));
+  c.tickets = take((size_t)(t1 > t2 ? t1 : t2) * batch_tiles_of(max_batch) * 2 * sizeof(uint32_t));
   c.status = take(sizeof(uint32_t));
   c.total = off;
   return c;
@@ -203,18 +204,29 @@ bool encode_map(TensorMapEncodeFn fn, CUtensorMap* map, const void* base, uint64
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// `coop`: a cooperative launch -- the whole grid is resident at once or the launch is refused.
 template <typename... KArgs, typename... Args>
-cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, bool pdl, Args&&... args) {
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, bool pdl, bool coop,
+                       Args&&... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchAttribute attr[2];
+  int n = 0;
+  if (pdl) {
+    attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  if (coop) {
+    attr[n].id = cudaLaunchAttributeCooperative;
+    attr[n].val.cooperative = 1;
+    ++n;
+  }
   cfg.attrs = attr;
-  cfg.numAttrs = pdl ? 1 : 0;
+  cfg.numAttrs = n;
   return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
 }
 
@@ -229,9 +241,21 @@ opw_status_t run_tc_gemm(opw_afd_module* m, const CUtensorMap& map_w, const void
   // The step's (cos, sin) table: behind the ring for small batches, from global memory (written by a small
   // kernel launched just before) for large ones and wherever the table would leave the ring too small.
   // The epilogue reuses the ring: one tile of sums for all columns, or two tiles for a chunk of columns.
+  p.ksplit = ksplit_of(n_out, k, batch, m->sms < kSmsBound ? m->sms : kSmsBound);
+  const int ctas = tiles_of(n_out) * p.ksplit * batch_tiles_of(batch);
+  // The shared back end pays at large batches, where publishing and reducing the partial tiles is bandwidth work
+  // that a third of the CTAs would otherwise do alone (batch 256: 31 -> 27 us for the QKV projection); at small
+  // batches the back end is a latency chain either way, and a cooperative launch cannot start under the previous
+  // kernel's tail, which costs more than the sharing gives (batch 64: 149 -> 157 us per module step).
+  p.coop = (m->coop_ok && ctas <= m->sms && (p.ksplit > 1 || p.group > 1) && batch > kCoopMinBatch) ? 1 : 0;
   const int chunk_cols = batch < opw_afd::kChunkCols ? batch : opw_afd::kChunkCols;
-  const size_t epi_bytes = p.group == 1 ? (size_t)p.nb * opw_afd::kTileM * sizeof(float)
-                                        : ((size_t)opw_afd::kChunkCols + chunk_cols) * opw_afd::kTileM * sizeof(float);
+  const int members = p.ksplit * p.group;
+  // cooperative back end: the CTA's own tile, plus (two-tile heads) its slice of the other tile's sums
+  const size_t epi_coop = ((size_t)p.nb + (p.group == 2 ? (size_t)((batch < opw_afd::kMaxNb ? batch : opw_afd::kMaxNb) + members - 1) / members + 1 : 0)) *
+                          opw_afd::kTileM * sizeof(float);
+  const size_t epi_last = p.group == 1 ? (size_t)p.nb * opw_afd::kTileM * sizeof(float)
+                                       : ((size_t)opw_afd::kChunkCols + chunk_cols) * opw_afd::kTileM * sizeof(float);
+  const size_t epi_bytes = p.coop ? epi_coop : epi_last;
   bool angles_global = mode == 1 && batch > kSmemAngleBatch;
   size_t angle_bytes = 0;
   int stages = 0;
@@ -244,7 +268,6 @@ opw_status_t run_tc_gemm(opw_afd_module* m, const CUtensorMap& map_w, const void
   }
   if (stages < 2 || (size_t)stages * stage_bytes < epi_bytes) return OPW_ERR_UNSUPPORTED;
   p.stages = stages;
-  p.ksplit = ksplit_of(n_out, k, batch, m->sms < kSmsBound ? m->sms : kSmsBound);
   p.mode = mode;
   p.out = out; p.q = q; p.kn = kn; p.vn = vn;
   p.positions = positions;
@@ -257,7 +280,7 @@ opw_status_t run_tc_gemm(opw_afd_module* m, const CUtensorMap& map_w, const void
   // trace region 0: output projection, region 1: QKV projection
   p.trace = m->trace ? m->trace + (size_t)mode * opw_afd::kTraceMaxCtas * opw_afd::kTraceWords : nullptr;
   if (angles_global) {
-    if (launch_pdl(opw_afd::rope_table_kernel, dim3(batch), dim3(128), 0, stream, m->pdl, positions,
+    if (launch_pdl(opw_afd::rope_table_kernel, dim3(batch), dim3(128), 0, stream, m->pdl, false, positions,
                    reinterpret_cast<float2*>(m->ws + m->off_angles), (int)m->D, m->log_theta) != cudaSuccess) {
       (void)cudaGetLastError();
       return OPW_ERR_CUDA;
@@ -268,7 +291,7 @@ opw_status_t run_tc_gemm(opw_afd_module* m, const CUtensorMap& map_w, const void
   if (!encode_map(m->encode, &map_x, x, (uint64_t)batch, (uint64_t)k, (uint32_t)p.nb)) return OPW_ERR_CUDA;
   const dim3 grid(tiles_of(n_out), p.ksplit, batch_tiles_of(batch));
   if (launch_pdl(opw_afd::skinny_gemm_kernel, grid, dim3(opw_afd::kGemmThreads), 1024 + (size_t)stages * stage_bytes + angle_bytes,
-                 stream, m->pdl, map_w, map_x, p) != cudaSuccess) {
+                 stream, m->pdl, p.coop != 0, map_w, map_x, p) != cudaSuccess) {
     (void)cudaGetLastError();
     return OPW_ERR_CUDA;
   }
@@ -328,6 +351,9 @@ opw_status_t opw_afd_module_create(opw_attn_stage_t* stage, int32_t layer, int32
     int sms = 0;
     ok = ok && cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) == cudaSuccess && sms > 0;
     m->sms = sms;
+    int coop = 0;
+    if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, device) != cudaSuccess) { (void)cudaGetLastError(); coop = 0; }
+    m->coop_ok = coop != 0;
     ok = ok && cudaFuncSetAttribute(opw_afd::skinny_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)kGemmSmemBudget) == cudaSuccess;
     const int n_qkv = (Hq + 2 * Hkv) * D, n_attn = Hq * D;
@@ -410,7 +436,16 @@ opw_status_t opw_afd_module_poll_error(opw_afd_module_t* m, void* cuda_stream) {
     (void)cudaGetLastError();
     return OPW_ERR_CUDA;
   }
-  return (word & opw_afd::kGemmErrTimeout) ? OPW_ERR_TIMEOUT : OPW_OK;
+  if (word & opw_afd::kGemmErrTimeout) {
+    // a kernel that gave up may have left its group counters mid-count
+    if (cudaMemsetAsync(m->ws + m->off_tickets, 0, m->off_status - m->off_tickets, stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess) {
+      (void)cudaGetLastError();
+      return OPW_ERR_CUDA;
+    }
+    return OPW_ERR_TIMEOUT;
+  }
+  return OPW_OK;
 }
 
 opw_status_t opw_afd_module_set_trace(opw_afd_module_t* m, void* trace, size_t trace_bytes) {

@@ -14,8 +14,12 @@
 //
 // With N/128 tiles alone a 6144 x 4096 projection would occupy 48 of 148 SMs, too few to pull
 // the weights at HBM speed, so K is also split over `ksplit` CTAs per tile; each writes its fp32
-// partial tile to a workspace and the last to arrive (an atomic ticket per tile) adds them in
-// split order -- deterministic -- and runs the epilogue.
+// partial tile to a workspace.  When the whole grid fits the device (a cooperative launch guarantees
+// that every CTA is resident) the CTAs of a tile meet at a counter and each of them reduces and
+// finishes its own slice of the batch columns -- the back end would otherwise sit on a third of the
+// SMs while the others idle; with more CTAs than SMs nobody may wait, and the last CTA of a tile to
+// arrive (an atomic ticket) reduces and finishes all of it.  Either way the partial tiles are added
+// in split order: deterministic.
 //
 // Epilogues: plain (bf16 C[b, n]) and rotary (the QKV projection of the attention module: pairs
 // (d, d + D/2) of the q and k heads are rotated, still as fp32 accumulators, by angles that the
@@ -52,6 +56,7 @@ struct GemmParams {
   int n_out, k, batch;
   int nb;                 // MMA N of a full batch tile: min(batch, 256) rounded up to a multiple of 16
   int group;              // weight tiles that share a ticket and an epilogue: 1, or 2 (rotary at D = 256)
+  int coop;               // the launch is cooperative (every CTA resident): the CTAs of a ticket group share the back end
   const float2* angles_g; // mode 1: [batch, D/2] (cos, sin) in global memory, or null: computed here in shared memory
   int stages;
   int ksplit;
@@ -64,7 +69,7 @@ struct GemmParams {
   double log_theta;
   int Hq, Hkv, D;
   float* partials;        // [tiles, ksplit, nb, 128] fp32, used when ksplit > 1
-  uint32_t* tickets;      // [tiles], zero between launches
+  uint32_t* tickets;      // [ticket groups][2] {arrived, departed}, zero between launches
   uint32_t* status;
   unsigned long long* trace;   // optional: [grid][8] global-timer stamps of each CTA's phases (see kTrace*)
 };
@@ -372,36 +377,9 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
   if (warp == 1) g_tmem_dealloc(tmem_d, ncols);
   g_stamp(p, cta, 3);
 
-  // ---- hand-off: the last CTA of a ticket group to arrive reduces the partial tiles in split order ----
-  // A ticket group is the ksplit CTAs of one weight tile, or of the two tiles of a head (group = 2).
-  // Ordering: every thread's partial stores happen before the CTA barrier, thread 0's ticket is an
-  // acq_rel atomic at gpu scope after it (release is cumulative over the barrier), and the last
-  // CTA's threads read only after a second barrier behind that atomic.
   const bool shared_epilogue = p.ksplit > 1 || p.group > 1;
   const int ptile = blockIdx.z * gridDim.x + tile;                       // tile index over all batch tiles
   const size_t split_floats = (size_t)nb * kTileM;                        // one CTA's partial tile
-  bool finish = good;
-  if (shared_epilogue) {
-    const int n4 = batch_here * kTileM / 4;
-    float4* part = reinterpret_cast<float4*>(p.partials + ((size_t)ptile * p.ksplit + split) * split_floats);
-    if (good)
-      for (int i = tid; i < n4; i += kGemmThreads) part[i] = reinterpret_cast<const float4*>(stage_f)[i];
-    __syncthreads();
-    if (tid == 0) {
-      uint32_t prev;                                           // taken on failure too, so the count always completes
-      uint32_t* tk = p.tickets + ptile / p.group;
-      asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(tk) : "memory");
-      s_last = prev == (uint32_t)(p.ksplit * p.group) - 1u;
-      if (s_last) *tk = 0;                                     // ready for the next launch
-    }
-    __syncthreads();
-    g_stamp(p, cta, 4);
-    finish = good && s_last != 0;
-  }
-  if (!finish) {
-    g_stamp(p, cta, 6);
-    return;
-  }
 
   // Epilogue of weight tile T over the local batch columns [cb, ce): `val` holds the tile's sums as
   // [column - cb][128 rows], `par` the sums of the tile that holds the rotation partners (val itself
@@ -453,26 +431,109 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
 
   // Sum of the ksplit partial tiles of weight tile index `pt` (over all batch tiles) for the local columns
   // [cb, ce), in split order, into dst[column - cb][128].  `own`: this CTA's own partial of that tile is still
-  // in shared memory at `dst` (cb = 0) and is taken from there.
+  // in shared memory at `dst` and is taken from there.
   auto reduce_tile = [&](int pt, float* dst, int cb, int ce, bool own) {
     const float4* part = reinterpret_cast<const float4*>(p.partials + (size_t)pt * p.ksplit * split_floats) + (size_t)cb * kTileM / 4;
     gemm_reduce_partials(part, reinterpret_cast<float4*>(dst), (ce - cb) * kTileM / 4, p.ksplit, own ? split : -1, split_floats / 4);
   };
 
-  if (p.group == 1) {
-    if (p.ksplit > 1) {
-      // Every other split's values are fetched at once (the reduction would otherwise be a chain of
-      // L2 round trips); this CTA's own are already in shared memory.  Summed in split order, so the
-      // result does not depend on which CTA came last.
-      reduce_tile(ptile, stage_f, 0, batch_here, true);
+  if (!shared_epilogue) {                     // one CTA holds the whole sum of its tile
+    if (good) epilogue(tile, stage_f, stage_f, 0, batch_here);
+    g_stamp(p, cta, 6);
+    return;
+  }
+
+  // ---- hand-off through global memory: every CTA publishes its partial tile ----
+  // A ticket group is the ksplit CTAs of one weight tile, or of the two tiles of a head (group = 2).
+  // Ordering: every thread's partial stores happen before the CTA barrier, thread 0's arrival is an
+  // acq_rel atomic at gpu scope after it (release is cumulative over the barrier), and readers read
+  // only after a barrier behind their own acquire of the full count.
+  {
+    const int n4 = batch_here * kTileM / 4;
+    float4* part = reinterpret_cast<float4*>(p.partials + ((size_t)ptile * p.ksplit + split) * split_floats);
+    if (good)
+      for (int i = tid; i < n4; i += kGemmThreads) part[i] = reinterpret_cast<const float4*>(stage_f)[i];
+  }
+  __syncthreads();
+  const int members = p.ksplit * p.group;                                 // CTAs of this ticket group
+  uint32_t* tk = p.tickets + 2 * (ptile / p.group);                       // {arrived, departed}, zero between launches
+  const int t0 = tile - tile % p.group;                                   // first tile of the group
+
+  if (p.coop) {
+    // ---- every CTA of the group takes a slice of the batch columns (the launch is cooperative: all CTAs are
+    // resident, so the wait below ends when the slowest member has published; it is bounded all the same) ----
+    if (tid == 0) {
+      uint32_t seen;
+      asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(seen) : "l"(tk) : "memory");
+      ++seen;
+      uint64_t t_start, t_now;
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_start));
+      while (seen < (uint32_t)members) {
+        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(tk) : "memory");
+        asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t_now));
+        if (t_now - t_start > kGemmWaitNs) break;
+      }
+      if (seen < (uint32_t)members) {
+        s_fail = 1;
+        atomicOr(p.status, kGemmErrTimeout);
+      }
+    }
+    __syncthreads();
+    g_stamp(p, cta, 4);
+    if (s_fail != 0 || !good) {                 // recorded; the host clears the counters when it polls the error
+      g_stamp(p, cta, 6);
+      return;
+    }
+    const int rank = (tile - t0) * p.ksplit + split;
+    const int cb = (int)((int64_t)batch_here * rank / members), ce = (int)((int64_t)batch_here * (rank + 1) / members);
+    if (ce > cb) {
+      float* mine = stage_f + (size_t)cb * kTileM;                        // this tile's sums, in place over the own partial
+      reduce_tile(ptile, mine, cb, ce, true);
+      float* other = stage_f + split_floats;                              // the head's other tile (group = 2)
+      if (p.group == 2) reduce_tile(blockIdx.z * gridDim.x + (tile ^ 1), other, cb, ce, false);
       __syncthreads();
       g_stamp(p, cta, 5);
+      if (p.group == 1) {
+        epilogue(tile, mine, mine, cb, ce);
+      } else {
+        epilogue(tile, mine, other, cb, ce);
+        epilogue(tile ^ 1, other, mine, cb, ce);
+      }
     }
+    __syncthreads();
+    if (tid == 0) {                             // the last member to leave puts both counters back to zero
+      uint32_t left;
+      asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(left) : "l"(tk + 1) : "memory");
+      if (left == (uint32_t)members - 1u) { tk[0] = 0; tk[1] = 0; }
+    }
+    g_stamp(p, cta, 6);
+    return;
+  }
+
+  // ---- no residency guarantee (more CTAs than SMs): the last CTA of the group to arrive does it all, nobody waits ----
+  if (tid == 0) {
+    uint32_t prev;                                             // taken on failure too, so the count always completes
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(tk) : "memory");
+    s_last = prev == (uint32_t)members - 1u;
+    if (s_last) *tk = 0;                                       // ready for the next launch
+  }
+  __syncthreads();
+  g_stamp(p, cta, 4);
+  if (!(good && s_last != 0)) {
+    g_stamp(p, cta, 6);
+    return;
+  }
+  if (p.group == 1) {
+    // Every other split's values are fetched at once (the reduction would otherwise be a chain of
+    // L2 round trips); this CTA's own are already in shared memory.  Summed in split order, so the
+    // result does not depend on which CTA came last.
+    reduce_tile(ptile, stage_f, 0, batch_here, true);
+    __syncthreads();
+    g_stamp(p, cta, 5);
     epilogue(tile, stage_f, stage_f, 0, batch_here);
   } else {
     // Two tiles of one head: both are reduced from the partial tiles in global memory (this CTA's own
     // included), kChunkCols batch columns at a time so that both fit the ring's shared memory.
-    const int t0 = tile & ~1;                                  // first tile of the head
     float* buf0 = stage_f;
     float* buf1 = stage_f + (size_t)kChunkCols * kTileM;
     for (int cb = 0; cb < batch_here; cb += kChunkCols) {

@@ -156,9 +156,9 @@ def test_attention_module_workspace_and_null_arguments_need_no_device():
     assert base >= acts + (32 << 20) and base % 256 == 0
     assert B.opw_afd_module_workspace_bytes(32, 8, 128, 128, 4096) > base          # grows with the batch
     # from 2048 to 4096 rows: the activation buffers, eight more batch tiles of unsplit partial sums for the wider
-    # projection (48 weight tiles x 256 columns x 128 rows of fp32), the angle table, a ticket per (weight, batch) tile
+    # projection (48 weight tiles x 256 columns x 128 rows of fp32), the angle table, two counters per (weight, batch) tile
     grow = B.opw_afd_module_workspace_bytes(32, 8, 128, 4096, 4096) - B.opw_afd_module_workspace_bytes(32, 8, 128, 2048, 4096)
-    assert grow == 2048 * (48 + 32 + 8 + 8 + 32) * 128 * 2 + 8 * 48 * 256 * 128 * 4 + 2048 * 64 * 8 + 8 * 48 * 4
+    assert grow == 2048 * (48 + 32 + 8 + 8 + 32) * 128 * 2 + 8 * 48 * 256 * 128 * 4 + 2048 * 64 * 8 + 8 * 48 * 2 * 4
     for bad in ((32, 7, 128, 64, 4096), (32, 8, 96, 64, 4096), (32, 8, 128, 0, 4096), (32, 8, 128, 64, 4100), (0, 8, 128, 64, 4096)):
         assert B.opw_afd_module_workspace_bytes(*bad) == 0
     L = B.lib()
