@@ -876,6 +876,7 @@ constexpr int kCombineThreads = 256;
 constexpr int kCombineThreadsSmall = 128;
 constexpr int kCombineMaxG = 16;
 constexpr int kCombineBatch = 64;               // segments merged per pass
+constexpr int kCombineScanBatch = 1024;         // up to this batch a combine block recomputes the page prefix sums itself
 // acc[j] = acc[j] * scale[h] + sum over the listed partials of weight * o, for the thread's
 // elements e = tid + j * kCT.  The loads of one pass are all independent.
 template <int NEL, int kCT>
@@ -922,18 +923,142 @@ __device__ __forceinline__ void combine_accumulate(float* acc, const float* part
 // kD: the head dimension as a compile-time constant (0: read it from the parameters); the kernel is
 // bound by integer arithmetic more than by memory, and divisions by D are a good part of it.
 template <int kCT, int kD = 0>
-__global__ void __launch_bounds__(kCT, kCT == 128 ? 6 : 2) combine_kernel(CombineParams p) {
+__global__ void __launch_bounds__(kCT, kCT == 128 ? 5 : 2) combine_kernel(CombineParams p) {
   pdl_launch_dependents();
   const int row = blockIdx.x;
   const int splits = gridDim.y, split = blockIdx.y;
   const int b = row / p.Hkv, g = row - b * p.Hkv;
   const int D = kD ? kD : p.D, G = p.G;
   const int GD = G * D;
-  int32_t n = visible_keys(p.kv_lens, p.positions, b);   // an input: may be read before the attention kernel is done
-  pdl_wait();                                  // partials, prefix sums and complete rows are final now
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  __shared__ int32_t seg_slot[kCombineBatch];
+  __shared__ int32_t warp_cnt[kCT / 32];
+  __shared__ int32_t scan_s[2][kCT / 32];
+  __shared__ float w_s[kCombineBatch * kCombineMaxG];   // per (segment, head): m, then the weight
+  __shared__ float l_s[kCombineBatch * kCombineMaxG];
+  __shared__ float run_M[kCombineMaxG], run_L[kCombineMaxG], run_scale[kCombineMaxG];
+  __shared__ int32_t is_last;
+  constexpr int kMaxElems = kCombineMaxG * 128 / kCT;   // 8 (256 threads) or 16 (128 threads)
+  const int nel = (GD + kCT - 1) / kCT;
+  const int64_t stride = (int64_t)G * (D + 2);
+  float acc[kMaxElems];
+#pragma unroll
+  for (int j = 0; j < kMaxElems; ++j) acc[j] = 0.f;
+  if (threadIdx.x < kCombineMaxG) { run_M[threadIdx.x] = -INFINITY; run_L[threadIdx.x] = 0.f; }
+
+  // keys visible to sequence bb, as the attention kernel counts them (clamped to the table)
+  auto keys_of = [&](int bb) -> int32_t {
+    int32_t nn = visible_keys(p.kv_lens, p.positions, bb);
+    if (nn > p.max_pages * kPage) nn = p.max_pages * kPage;
+    return nn;
+  };
+  const int32_t n = keys_of(b);               // an input: may be read before the attention kernel is done
+
+  // Which segments overlap this row follows from the step's metadata alone (kv_lens / positions, the
+  // window, the grid).  For batches up to kCombineScanBatch the block therefore works it out BEFORE the
+  // dependency wait -- the page prefix sums, the candidate test and the list of partial slots of the
+  // first batch of candidates -- so that under programmatic dependent launch all of it runs beneath the
+  // attention kernel's tail and only the loads of the partials are left for afterwards.  Larger batches
+  // read the prefix sums the attention kernel stored, after the wait.
+  const bool early = p.batch <= kCombineScanBatch;
+  int32_t cum_b = 0, cum_all = 0, cnt = 0;
+  int64_t U = 0, ustart = 0, uend = 0, wf = 0, wl = 0, ncand = 0;
+  ShareMath sm;
+  int segs = 1;
+  bool by_unit = false, whole = false;
+  int nseg_first = 0;
+
+  // candidates [base, base + kCombineBatch): test, ordered compaction into seg_slot; returns how many were listed
+  auto list_candidates = [&](int64_t base) -> int {
+    const int64_t i = base + threadIdx.x;
+    bool hit = false;
+    int32_t slot = 0;
+    if (threadIdx.x < kCombineBatch && i < ncand) {
+      int64_t j;                                   // candidate i = (share or unit j, segment k); 32-bit division where it fits
+      if (ncand < (int64_t)1 << 31) j = (int64_t)((uint32_t)i / (uint32_t)segs);
+      else j = i / segs;
+      const int k = (int)(i - j * segs);
+      int64_t w;
+      bool counted = true;
+      if (by_unit) {
+        w = worker_of(U, ustart + j, p.num_workers);
+        counted = j == 0 || worker_of(U, ustart + j - 1, p.num_workers) != w;
+      } else {
+        w = wf + j;
+      }
+      int64_t a, bnd;
+      sm.bounds((uint32_t)w, k, a, bnd);
+      hit = counted && a < bnd && a < uend && bnd > ustart;
+      slot = (int32_t)(2 * (w * kSegPerShare + k) + (a >= ustart ? 0 : 1));
+    }
+    const uint32_t bal = __ballot_sync(0xffffffffu, hit);
+    if (lane == 0) warp_cnt[warp] = __popc(bal);
+    __syncthreads();
+    int pos = __popc(bal & ((1u << lane) - 1u));
+    int nseg = 0;
+    for (int j = 0; j < kCombineBatch / 32; ++j) {
+      if (j < warp) pos += warp_cnt[j];
+      nseg += warp_cnt[j];
+    }
+    if (hit) seg_slot[pos] = slot;
+    __syncthreads();
+    return nseg;
+  };
+
+  // everything between the prefix sums and the first list of partial slots
+  auto prepare = [&]() {
+    if (n <= 0) return;                         // (uniform over the block)
+    int32_t first, lo;
+    visible_pages(n, p.window, p.max_pages, first, cnt, lo);
+    U = (int64_t)cum_all * p.Hkv;
+    ustart = (int64_t)cum_b * p.Hkv + (int64_t)g * cnt;
+    uend = ustart + cnt;
+    wf = worker_of(U, ustart, p.num_workers);
+    wl = worker_of(U, uend - 1, p.num_workers);
+    // segments a share really has in this launch (1 + the number of ticketed chunks, which depends on the
+    // share length only): small launches have fewer than kSegPerShare, and fewer candidates to test
+    sm.init(U, p.num_workers);
+    segs = sm.J + 1;
+    // If the segment that holds the row's first unit also holds its last, that segment's worker
+    // stores the final result itself: nothing to merge (every block of the row sees this).
+    bool w0 = false;
+    if (threadIdx.x < segs) {
+      int64_t a, bnd;
+      sm.bounds((uint32_t)wf, (int)threadIdx.x, a, bnd);
+      w0 = a <= ustart && ustart < bnd && bnd >= uend;
+    }
+    whole = __syncthreads_or(w0);
+    if (whole) return;
+    // Candidate shares are listed by share index (wf..wl), or, when the row has fewer units than
+    // that (tiny launches: most shares are empty), by unit: the share holding unit ustart + j,
+    // counted once, at its first unit inside the row.
+    by_unit = (wl - wf + 1) > (int64_t)cnt;
+    ncand = (by_unit ? (int64_t)cnt : (wl - wf + 1)) * segs;
+    if ((int64_t)split * kCombineBatch < ncand) nseg_first = list_candidates((int64_t)split * kCombineBatch);
+  };
+
+  if (early) {
+    // pages before sequence b and of the whole batch, from the metadata
+    int32_t before = 0, total = 0;
+    for (int bb = threadIdx.x; bb < p.batch; bb += kCT) {
+      int32_t f, c, l;
+      visible_pages(keys_of(bb), p.window, p.max_pages, f, c, l);
+      total += c;
+      if (bb < b) before += c;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      before += __shfl_xor_sync(0xffffffffu, before, o);
+      total += __shfl_xor_sync(0xffffffffu, total, o);
+    }
+    if (lane == 0) { scan_s[0][warp] = before; scan_s[1][warp] = total; }
+    __syncthreads();
+    for (int wq = 0; wq < kCT / 32; ++wq) { cum_b += scan_s[0][wq]; cum_all += scan_s[1][wq]; }
+    prepare();
+  }
+
+  pdl_wait();                                  // partials and complete rows are final now
   if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *p.ticket = 0;
-  const int32_t cum_b = p.cum[b], cum_all = p.cum[p.batch];     // independent of the load above
-  if (n > p.max_pages * kPage) n = p.max_pages * kPage;
   __nv_bfloat16* ob = p.out + ((int64_t)b * p.Hq + (int64_t)g * G) * D;
   float* lse_row = p.lse ? p.lse + (int64_t)b * p.Hq + g * G : nullptr;
   if (n <= 0) {   // inactive slot: zeros, lse = -inf
@@ -943,53 +1068,18 @@ __global__ void __launch_bounds__(kCT, kCT == 128 ? 6 : 2) combine_kernel(Combin
     }
     return;
   }
-  int32_t first, cnt, lo;
-  visible_pages(n, p.window, p.max_pages, first, cnt, lo);
-  const int64_t U = (int64_t)cum_all * p.Hkv;
-  const int64_t ustart = (int64_t)cum_b * p.Hkv + (int64_t)g * cnt;
-  const int64_t uend = ustart + cnt;
-  const int64_t wf = worker_of(U, ustart, p.num_workers), wl = worker_of(U, uend - 1, p.num_workers);
-  const int64_t stride = (int64_t)G * (D + 2);
-  // segments a share really has in this launch (1 + the number of ticketed chunks, which depends on the
-  // share length only): small launches have fewer than kSegPerShare, and fewer candidates to test
-  ShareMath sm;
-  sm.init(U, p.num_workers);
-  const int segs = sm.J + 1;
-  // If the segment that holds the row's first unit also holds its last, that segment's worker
-  // has already stored the final result: nothing to merge (every block of the row sees this).
-  {
-    bool whole = false;
-    if (threadIdx.x < segs) {
-      int64_t a, bnd;
-      sm.bounds((uint32_t)wf, (int)threadIdx.x, a, bnd);
-      whole = a <= ustart && ustart < bnd && bnd >= uend;
-    }
-    if (__syncthreads_or(whole)) return;
+  if (!early) {
+    cum_b = p.cum[b];
+    cum_all = p.cum[p.batch];
+    prepare();
   }
+  if (whole) return;
   // The row's partials come from the segments (share w in wf..wl, k in 0..kSegPerShare) that
   // overlap it.  A batch of candidate segments at a time: each thread tests one, an ordered
   // compaction lists the partial slots in shared memory, one warp per head turns the partials'
   // running maxima into weights 2^(m - M), and every thread sums its elements over the list.
   // A segment's partial for this row is in the segment's slot 0 if the segment starts inside
   // the row, else in slot 1.
-  __shared__ int32_t seg_slot[kCombineBatch];
-  __shared__ int32_t warp_cnt[kCT / 32];
-  __shared__ float w_s[kCombineBatch * kCombineMaxG];   // per (segment, head): m, then the weight
-  __shared__ float l_s[kCombineBatch * kCombineMaxG];
-  __shared__ float run_M[kCombineMaxG], run_L[kCombineMaxG], run_scale[kCombineMaxG];
-  __shared__ int32_t is_last;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  constexpr int kMaxElems = kCombineMaxG * 128 / kCT;   // 8 (256 threads) or 16 (128 threads)
-  const int nel = (GD + kCT - 1) / kCT;
-  float acc[kMaxElems];
-#pragma unroll
-  for (int j = 0; j < kMaxElems; ++j) acc[j] = 0.f;
-  if (threadIdx.x < kCombineMaxG) { run_M[threadIdx.x] = -INFINITY; run_L[threadIdx.x] = 0.f; }
-  // Candidate shares are listed by share index (wf..wl), or, when the row has fewer units than
-  // that (tiny launches: most shares are empty), by unit: the share holding unit ustart + j,
-  // counted once, at its first unit inside the row.
-  const bool by_unit = (wl - wf + 1) > (int64_t)cnt;
-  const int64_t ncand = (by_unit ? (int64_t)cnt : (wl - wf + 1)) * segs;
 
   // One merge pass over `nseg` listed partials at `base_ptr` (slot stride `stride`): stage
   // (m, l), weights per head, then the weighted sums.
@@ -1032,38 +1122,8 @@ __global__ void __launch_bounds__(kCT, kCT == 128 ? 6 : 2) combine_kernel(Combin
   };
 
   for (int64_t base = (int64_t)split * kCombineBatch; base < ncand; base += (int64_t)splits * kCombineBatch) {
-    const int64_t i = base + threadIdx.x;
-    bool hit = false;
-    int32_t slot = 0;
-    if (threadIdx.x < kCombineBatch && i < ncand) {
-      int64_t j;                                   // candidate i = (share or unit j, segment k); 32-bit division where it fits
-      if (ncand < (int64_t)1 << 31) j = (int64_t)((uint32_t)i / (uint32_t)segs);
-      else j = i / segs;
-      const int k = (int)(i - j * segs);
-      int64_t w;
-      bool counted = true;
-      if (by_unit) {
-        w = worker_of(U, ustart + j, p.num_workers);
-        counted = j == 0 || worker_of(U, ustart + j - 1, p.num_workers) != w;
-      } else {
-        w = wf + j;
-      }
-      int64_t a, bnd;
-      sm.bounds((uint32_t)w, k, a, bnd);
-      hit = counted && a < bnd && a < uend && bnd > ustart;
-      slot = (int32_t)(2 * (w * kSegPerShare + k) + (a >= ustart ? 0 : 1));
-    }
-    const uint32_t bal = __ballot_sync(0xffffffffu, hit);
-    if (lane == 0) warp_cnt[warp] = __popc(bal);
-    __syncthreads();
-    int pos = __popc(bal & ((1u << lane) - 1u));
-    int nseg = 0;
-    for (int j = 0; j < kCombineBatch / 32; ++j) {
-      if (j < warp) pos += warp_cnt[j];
-      nseg += warp_cnt[j];
-    }
-    if (hit) seg_slot[pos] = slot;
-    __syncthreads();
+    // the first batch was listed by prepare()
+    const int nseg = base == (int64_t)split * kCombineBatch ? nseg_first : list_candidates(base);
     merge_listed(p.partials, nseg);
   }
 
