@@ -100,6 +100,7 @@ def test_workspace_bytes_needs_a_valid_shape():
     (dict(softmax_scale=-1.0), B.OPW_ERR_INVALID_ARG),
     (dict(head_dim=128, tune_warps=8, tune_stages=4), B.OPW_ERR_CAPACITY),
     (dict(max_batch=0), B.OPW_ERR_INVALID_ARG),
+    (dict(flags=2), B.OPW_ERR_INVALID_ARG),                      # only OPW_FLAG_NO_PDL is defined
 ])
 def test_create_rejects_bad_configs_before_touching_cuda(over, want):
     cfg, keep = good_cfg(**over)
@@ -122,6 +123,7 @@ def test_step_calls_reject_a_null_handle_and_destroy_accepts_it():
     assert L.opw_decode_attention(None, 0, 1, 16, 16, 16, 16, None, None) == B.OPW_ERR_INVALID_ARG
     assert L.opw_decode_step_host(None, 0, 1, 16, 16, 16, 16, None, 16, None, None) == B.OPW_ERR_INVALID_ARG
     assert L.opw_attn_stage_poll_error(None, None) == B.OPW_ERR_INVALID_ARG
+    assert L.opw_attn_stage_page_table_delta_host(None, 0, 16, 1, None) == B.OPW_ERR_INVALID_ARG
     assert L.opw_attn_stage_launch_count(None) == 0
     assert L.opw_attn_stage_destroy(None) == B.OPW_OK
 
