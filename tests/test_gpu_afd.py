@@ -358,3 +358,48 @@ def test_a_plan_of_module_steps_equals_the_same_steps_called_one_by_one(flags, p
     for a, b in zip(results[0][1], results[1][1]):
         assert (a == b).all()
     assert np.isfinite(oracle.bf16_bits_to_f64(results[1][0][-1])).all() and results[1][0][-1].any()
+
+
+def test_large_batch_module_steps_in_a_captured_plan_equal_the_same_steps_called_one_by_one():
+    """160 rows: the projections' CTAs share their back end under a cooperative launch (with programmatic
+    dependent launch on top) and the angle table comes from its own kernel; all of it captured into one CUDA graph
+    must give the outputs and the KV pool of plain calls, bit for bit."""
+    rng = np.random.default_rng(93)
+    Hq, Hkv, D, hidden, Bn, steps = 8, 2, 128, 512, 160, 3
+    lens = [int(n) for n in rng.integers(1, 200, Bn)]
+    case = make_case(rng, [n + steps for n in lens], Hq, Hkv, D)
+    w1 = to_dev_bf16(oracle.f32_to_bf16_bits((rng.standard_normal(((Hq + 2 * Hkv) * D, hidden)) / 22).astype(np.float32)))
+    w2 = to_dev_bf16(oracle.f32_to_bf16_bits((rng.standard_normal((hidden, Hq * D)) / 32).astype(np.float32)))
+    x = to_dev_bf16(oracle.f32_to_bf16_bits(rng.standard_normal((Bn, hidden)).astype(np.float32)))
+    tab = torch.from_numpy(case[1]).cuda()
+    results = []
+    for use_plan in (False, True):
+        pool = to_dev_bf16(case[0])
+        stage = B.Stage(pools=[pool], layer_window=[0], num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, max_batch=Bn,
+                        max_pages_per_seq=tab.shape[1])
+        mod = B.AfdModule(stage, 0, w1, w2, THETA)
+        pos = torch.tensor(lens, dtype=torch.int32, device="cuda")
+        y = torch.zeros(Bn, hidden, dtype=torch.bfloat16, device="cuda")
+        outs = []
+        if use_plan:
+            plan = B.opw_attn_plan_create_mixed(stage.handle, [dict(kind="afd_module", module=mod.handle, batch=Bn, x=x.data_ptr(),
+                                                                    positions=pos.data_ptr(), page_table=tab.data_ptr(), y=y.data_ptr())],
+                                                B.OPW_PLAN_GRAPH | B.OPW_PLAN_ADVANCE)
+        for _ in range(steps):
+            if use_plan:
+                B.opw_attn_plan_submit(plan, torch.cuda.current_stream().cuda_stream)
+            else:
+                mod.step(x, pos, tab, y)
+                pos.add_(1)
+            torch.cuda.synchronize()
+            outs.append(tobits(y).copy())
+        assert stage.poll_error() == B.OPW_OK and mod.poll_error() == B.OPW_OK
+        results.append((outs, tobits(pool).copy()))
+        if use_plan:
+            B.opw_attn_plan_destroy(plan)
+        mod.close()
+        stage.close()
+    for a, b in zip(results[0][0], results[1][0]):
+        assert (a == b).all()
+    assert (results[0][1] == results[1][1]).all()
+    assert np.isfinite(oracle.bf16_bits_to_f64(results[1][0][-1])).all() and results[1][0][-1].any()
