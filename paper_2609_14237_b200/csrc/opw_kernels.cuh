@@ -199,7 +199,10 @@ __host__ __device__ __forceinline__ int64_t worker_of(int64_t U, int64_t u, int6
 // Segments of a share: k = 0 is the static first 13/16; k = 1..J cut the last 3/16 into ever
 // smaller chunks (cut points in sixteenths of that part).  J depends on the share length
 // only (the same for every share of a launch): a segment costs a couple of microseconds of
-// fixed work (ticket, descriptors, Q reload, partial flush), so short shares get fewer chunks.
+// fixed work (ticket, descriptors, Q reload, partial flush) and two more partials for the combine,
+// so short shares get fewer chunks (measured per step, back to back: shares of 28 units 53.1 -> 50.3 us
+// with none instead of two, shares of 69 units 107.9 -> 105.8 us with two instead of four; shares of
+// 221 units run the same with four as with six).
 #ifndef OPW_DYN_PER_SHARE
 #define OPW_DYN_PER_SHARE 6      /* upper bound of J; 0 builds static shares only */
 #endif
@@ -215,7 +218,7 @@ constexpr int kSegPerShare = kDynPerShare + 1;   // partial slots are indexed wi
 __host__ __device__ __forceinline__ int dyn_chunks(int64_t U, int64_t num_workers) {
   if (kDynPerShare == 0) return 0;
   const int64_t per = U / num_workers;
-  return per < 8 ? 0 : per < 48 ? 2 : per < 128 ? 4 : 6;
+  return per < 32 ? 0 : per < 96 ? 2 : per < 256 ? 4 : 6;
 }
 __host__ __device__ __forceinline__ int64_t dyn_cut(int J, int k) {   // five bits per cut point
   const uint64_t cuts6 = 0ull | (5ull << 5) | (9ull << 10) | (12ull << 15) | (14ull << 20) | (15ull << 25) |
