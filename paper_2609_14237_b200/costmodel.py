@@ -167,3 +167,39 @@ def cad_feasible(gpu_attn: Gpu, microbatches: int, gpu_rest: Gpu, m_weights_per_
 def with_measured_bandwidth(gpu: Gpu, beta_eff: float) -> Gpu:
     """The same GPU type with the bandwidth the attention stage actually sustains."""
     return dataclasses.replace(gpu, beta=beta_eff)
+
+
+# ------------------------------------------------ measured profile -> latency model ---
+
+def fit_affine_latency(points: Sequence[Tuple[float, float]], relative: bool = True) -> Tuple[float, float]:
+    """Least-squares fit of T = t0 + D / beta to measured (bytes D, latency T) pairs of an attention stage.
+
+    The paper's roofline for the operator is T = D / beta (Appendix A.1, A.4); a measured stage also has a
+    latency floor t0 (first-tile latency, tail, combine) that matters for the small steps a stage runs when
+    it holds few microbatches under a tight time-per-output-token target (Section 4: stage latencies come
+    from profiled execution latency).  `relative` weights every point by 1 / T^2, i.e. minimises the relative
+    error, so that microsecond-sized steps count as much as millisecond-sized ones.  Returns (t0, beta) in the
+    units of the inputs."""
+    pts = [(float(d), float(t)) for d, t in points]
+    if len(pts) < 2:
+        raise ValueError("need at least two measured points")
+    if any(t <= 0.0 for _, t in pts):
+        raise ValueError("latencies must be positive")
+    w = [1.0 / (t * t) if relative else 1.0 for _, t in pts]
+    sw = sum(w)
+    sx = sum(wi * d for wi, (d, _) in zip(w, pts))
+    sy = sum(wi * t for wi, (_, t) in zip(w, pts))
+    sxx = sum(wi * d * d for wi, (d, _) in zip(w, pts))
+    sxy = sum(wi * d * t for wi, (d, t) in zip(w, pts))
+    den = sw * sxx - sx * sx
+    if den <= 1e-12 * sw * sxx:
+        raise ValueError("the points need at least two distinct sizes")
+    slope = (sw * sxy - sx * sy) / den
+    if slope <= 0.0:
+        raise ValueError("latency does not grow with the bytes loaded")
+    return (sy - slope * sx) / sw, 1.0 / slope
+
+
+def attention_latency_affine(batch: float, m_kv: float, t0: float, beta: float) -> float:
+    """The profiled form of `attention_latency`: a latency floor plus memory traffic over bandwidth."""
+    return t0 + batch * m_kv / beta

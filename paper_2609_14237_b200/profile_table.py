@@ -99,9 +99,17 @@ def main():
                 print(json.dumps(r), flush=True)
     if os.path.dirname(args.out):
         os.makedirs(os.path.dirname(args.out), exist_ok=True)
+    # the two-parameter latency model of the stage: a floor plus bytes over bandwidth, fitted to the table
+    from paper_2609_14237_b200 import costmodel
+
+    t0_s, beta = costmodel.fit_affine_latency([(r["kv_bytes"], r["t_us"] * 1e-6) for r in rows])
+    worst = max(abs(costmodel.attention_latency_affine(1, r["kv_bytes"], t0_s, beta) / (r["t_us"] * 1e-6) - 1) for r in rows)
+    fit = {"t0_us": round(t0_s * 1e6, 2), "beta_gbs": round(beta / 1e9, 1), "max_rel_error": round(worst, 4),
+           "model": "t = t0 + kv_bytes / beta, relative least squares"}
+    print(json.dumps({"fit": fit}), flush=True)
     with open(args.out, "w") as fh:
-        json.dump({"shape": {"num_q_heads": 32, "num_kv_heads": 8, "head_dim": 128, "page_size": 16}, "points": rows}, fh,
-                  indent=1)
+        json.dump({"shape": {"num_q_heads": 32, "num_kv_heads": 8, "head_dim": 128, "page_size": 16}, "points": rows,
+                   "fit": fit}, fh, indent=1)
 
 
 if __name__ == "__main__":

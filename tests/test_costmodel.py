@@ -135,3 +135,20 @@ def test_cad_feasibility_condition():
     assert not cm.cad_feasible(h100, 4, h100, 30e9)                    # 6.0 ms < 9.0 ms
     faster_rest = cm.with_measured_bandwidth(h100, 8e12)
     assert cm.cad_feasible(h100, 4, faster_rest, 30e9)                 # more bandwidth on the GEMM side helps
+
+
+def test_affine_latency_fit_recovers_floor_and_bandwidth():
+    """T = t0 + D / beta through exact points gives t0 and beta back; noise moves them little; bad inputs raise."""
+    t0, beta = 15e-6, 7.1e12
+    sizes = [4e6, 68e6, 270e6, 1.07e9, 4.3e9, 17e9]
+    exact = [(d, t0 + d / beta) for d in sizes]
+    f0, fb = cm.fit_affine_latency(exact)
+    assert abs(f0 - t0) < 1e-12 and abs(fb / beta - 1) < 1e-9
+    noisy = [(d, t * (1 + 0.01 * (-1) ** i)) for i, (d, t) in enumerate(exact)]
+    n0, nb = cm.fit_affine_latency(noisy)
+    assert abs(nb / beta - 1) < 0.03 and abs(n0 - t0) < 10e-6
+    assert cm.attention_latency_affine(64, 2560 * 4096, t0, beta) == pytest.approx(t0 + 64 * 2560 * 4096 / beta)
+    assert cm.attention_latency_affine(64, 2560 * 4096, 0.0, beta) == pytest.approx(cm.attention_latency(64, 2560 * 4096, beta))
+    for bad in ([(1e6, 1e-5)], [(1e6, 1e-5), (1e6, 2e-5)], [(1e6, 2e-5), (2e6, 1e-5)]):
+        with pytest.raises(ValueError):
+            cm.fit_affine_latency(bad)
