@@ -535,14 +535,18 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
                       "frac_of_value": round(world * e_bytes / (e_ms * 1e-3) / 1e9 / value, 4)}
     if want_e2e and world == 1 and not stack and R >= 2:
         # The same host-buffer steps with two microbatches in flight (the paper keeps mu microbatches resident
-        # on a stage so that transfers hide behind compute): even steps belong to microbatch A (stage handle
-        # `st`, stream A), odd steps to B (a second handle with its own workspace and staged tables, stream
-        # B), over disjoint layer pools.  Every step still copies its inputs in and its output out; the host waits
-        # for a microbatch's previous step (and reads its result) before it reuses that microbatch's buffers.
+        # on a stage so that transfers hide behind compute): even steps belong to microbatch A, odd steps to B,
+        # each with a stage handle of its own (workspace, staged tables) created with OPW_FLAG_COPY_STREAMS, over
+        # disjoint layer pools.  Both enqueue their kernels on ONE compute stream; each handle's copies run on its own
+        # streams beside the other microbatch's kernels.  Every step still copies its inputs in and its output out;
+        # the host waits for a microbatch's previous result (opw_attn_stage_wait_host_output) before it reuses that
+        # microbatch's buffers.
         Re = R - R % 2                                        # an even number of pools: half for each microbatch
-        st2 = binding.Stage(pools=inp.pools, layer_window=wl_r.layer_window, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D,
-                            max_batch=B, max_pages_per_seq=inp.max_pages_per_seq, **tune)
-        packs2 = [[(st, st2)[l & 1].packed_host_buffers(B) for l in range(R)] for _ in range(2)]
+        flags2 = tune.get("flags", 0) | binding.OPW_FLAG_COPY_STREAMS
+        tune2 = dict(tune, flags=flags2)
+        mb_stages = [binding.Stage(pools=inp.pools, layer_window=wl_r.layer_window, num_q_heads=Hq, num_kv_heads=Hkv,
+                                   head_dim=D, max_batch=B, max_pages_per_seq=inp.max_pages_per_seq, **tune2) for _ in range(2)]
+        packs2 = [[mb_stages[l & 1].packed_host_buffers(B) for l in range(R)] for _ in range(2)]
         for i in range(2):
             for l in range(R):
                 _, pq, pk, pv, _ = packs2[i][l]
@@ -550,23 +554,24 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
                 pk.copy_(inp.k_new[i, l].cpu())
                 pv.copy_(inp.v_new[i, l].cpu())
         houts = [torch.empty(B, Hq, D, dtype=torch.bfloat16).pin_memory() for _ in range(2)]
-        streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+        compute = torch.cuda.Stream()
         # This loop has its own step numbering: step s2 visits pool s2 % Re at round r0 + s2 // Re, r0 the first round
         # no pool has been appended at yet; an even pool belongs to microbatch A, an odd one to B.
         r0 = (base + warm + e2e_steps + R - 1) // R
         admitted.clear()                                      # rounds were skipped: both handles take their tables afresh
+        wait_out = binding.lib().opw_attn_stage_wait_host_output
 
         def host_step_mb(s2):
             l, t = s2 % Re, r0 + s2 // Re
             mb = l & 1
-            streams[mb].synchronize()                         # this microbatch's previous result is on the host now
-            with torch.cuda.stream(streams[mb]):
+            stage = mb_stages[mb]
+            wait_out(stage.handle)                            # this microbatch's previous result is on the host now
+            with torch.cuda.stream(compute):
                 pack = packs2[(s2 >> 1) & 1][l]
                 write_positions(pack[4], t)
-                stage = (st, st2)[mb]
                 tab = send_table(stage, l, t)
                 rc = step_host(*args_of(stage, pack, l), None if tab is None else tab.data_ptr(), houts[mb].data_ptr(), None,
-                               streams[mb].cuda_stream)
+                               compute.cuda_stream)
                 if rc != binding.OPW_OK:
                     raise binding.OpwError(rc, "opw_decode_step_host")
             return inp.kv_bytes(l, t)
@@ -582,15 +587,19 @@ def run_ours(name, steps, warmup, rotate, tune, want_e2e=True, want_cpu=False, w
             w0 = time.perf_counter()
             for s2 in range(warm2, warm2 + n2):
                 mb_bytes += host_step_mb(s2)
+            for stg in mb_stages:
+                stg.wait_host_output()
             torch.cuda.synchronize()
             mb_ms = (time.perf_counter() - w0) * 1e3
-            assert st.poll_error() == binding.OPW_OK and st2.poll_error() == binding.OPW_OK
+            assert all(stg.poll_error() == binding.OPW_OK for stg in mb_stages)
             v2 = mb_bytes / (mb_ms * 1e-3) / 1e9
             res["e2e_two_microbatches"] = {"value": round(v2, 1), "unit": "GB/s", "steps": n2,
                                            "ms_per_step": round(mb_ms / n2, 5), "timing": "wall clock, device synchronised at both ends",
+                                           "streams": "one compute stream for both microbatches; each stage's copies on its own streams (OPW_FLAG_COPY_STREAMS)",
                                            "h2d_bytes_per_step": int(round(packed + delta_bytes[0] / n2)), "d2h_bytes_per_step": int(d2h),
                                            "frac_of_value": round(v2 / value, 4)}
-        st2.close()
+        for stg in mb_stages:
+            stg.close()
     if want_submit:
         # The same steps through a plan: one native call (one CUDA graph launch) per pass over
         # the stage's layers, metadata advanced on the device.

@@ -57,6 +57,7 @@ typedef enum {
 
 #define OPW_FLAG_NONE 0u
 #define OPW_FLAG_NO_PDL 1u /* launch the kernels without programmatic stream serialisation (see opw_decode_attention) */
+#define OPW_FLAG_COPY_STREAMS 2u /* opw_decode_step_host copies on the stage's own streams (see there) */
 
 typedef struct {
   uint32_t struct_size;           /* sizeof(opw_attn_stage_config_t); checked at create */
@@ -195,6 +196,17 @@ opw_status_t opw_decode_step(opw_attn_stage_t *stage, int32_t layer, int32_t bat
  * pinned for the copies to be asynchronous; they must stay valid and unmodified until
  * the stream has passed the step.  page_table_host == NULL reuses the table staged by
  * the previous call for this layer's slot (tables rarely change between steps).
+ *
+ * With OPW_FLAG_COPY_STREAMS (Section 4: a stage keeps several microbatches resident so that
+ * transfers hide behind compute; Section 6.2: overlapping communication) the stage owns two
+ * streams and three events of its own (created at opw_attn_stage_create; no device memory): the
+ * copies in run on the first, the kernels on the caller's stream once the copies have landed, the
+ * copies out on the second once the kernels are done.  The caller's stream then carries kernels
+ * only: when two stages (two microbatches) take turns on ONE compute stream, the kernels of one
+ * follow the kernels of the other directly and every copy runs beside the other stage's kernels.
+ * Synchronising the caller's stream no longer covers the copy out: call
+ * opw_attn_stage_wait_host_output before reading out_host / lse_host and before the stage's next
+ * opw_decode_step_host.  Not for use under stream capture.
  */
 /*
  * Tensor packing for opw_decode_step_host (Section 6.2, low-overhead communication: many short
@@ -211,6 +223,10 @@ opw_status_t opw_decode_step_host(opw_attn_stage_t *stage, int32_t layer, int32_
                                   const void *k_new_host, const void *v_new_host, const int32_t *positions_host,
                                   const int32_t *page_table_host, void *out_host, float *lse_host,
                                   void *cuda_stream);
+
+/* Blocks the host until the copy out of the stage's latest opw_decode_step_host has finished (a stage created
+ * with OPW_FLAG_COPY_STREAMS; otherwise returns at once: the caller synchronises its own stream). */
+opw_status_t opw_attn_stage_wait_host_output(opw_attn_stage_t *stage);
 
 /*
  * Page-table delta from HOST memory (Section 6, first paragraph: only token, position and KV-cache

@@ -21,6 +21,7 @@ HEADERS = [os.path.join(_HERE, "csrc", "opw_kernels.cuh"), os.path.join(_HERE, "
            os.path.join(_ROOT, "include", "opw_linear_attn.h"), os.path.join(_ROOT, "include", "opw_afd.h")]
 
 OPW_FLAG_NO_PDL = 1
+OPW_FLAG_COPY_STREAMS = 2
 OPW_OK, OPW_ERR_INVALID_ARG, OPW_ERR_UNSUPPORTED, OPW_ERR_CAPACITY, OPW_ERR_CUDA, OPW_ERR_BAD_PAGE, OPW_ERR_TIMEOUT = range(7)
 
 EXPORTS = [
@@ -30,7 +31,7 @@ EXPORTS = [
     "opw_decode_attention_noalloc", "opw_attn_plan_create", "opw_attn_plan_submit", "opw_attn_plan_destroy",
     "opw_decode_step", "opw_attn_stage_host_layout", "opw_attn_stage_probe_timeout",
     "opw_linear_attn_decode_step", "opw_linear_attn_state_bytes", "opw_attn_plan_create_mixed",
-    "opw_attn_stage_page_table_delta_host",
+    "opw_attn_stage_page_table_delta_host", "opw_attn_stage_wait_host_output",
     "opw_attn_stage_shape", "opw_afd_module_workspace_bytes", "opw_afd_module_create", "opw_afd_module_step",
     "opw_afd_module_intermediates", "opw_afd_module_destroy", "opw_afd_module_poll_error",
     "opw_afd_module_launch_count", "opw_afd_module_set_trace", "opw_hbm_read_probe",
@@ -156,6 +157,8 @@ def lib() -> ctypes.CDLL:
     L.opw_attn_stage_host_layout.argtypes = [vp] + [ctypes.POINTER(ctypes.c_size_t)] * 5
     L.opw_decode_step_host.restype = ctypes.c_int
     L.opw_decode_step_host.argtypes = [vp, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]
+    L.opw_attn_stage_wait_host_output.restype = ctypes.c_int
+    L.opw_attn_stage_wait_host_output.argtypes = [vp]
     L.opw_attn_stage_page_table_delta_host.restype = ctypes.c_int
     L.opw_attn_stage_page_table_delta_host.argtypes = [vp, i32, vp, i32, vp]
     L.opw_linear_attn_decode_step.restype = ctypes.c_int
@@ -522,6 +525,9 @@ class Stage:
         opw_decode_step_host(self.handle, layer, positions.shape[0], q.data_ptr(), k_new.data_ptr(), v_new.data_ptr(),
                              positions.data_ptr(), None if page_table is None else page_table.data_ptr(),
                              out.data_ptr(), None if lse is None else lse.data_ptr(), self._stream())
+
+    def wait_host_output(self):
+        _check(lib().opw_attn_stage_wait_host_output(self.handle), "opw_attn_stage_wait_host_output")
 
     def page_table_delta_host(self, layer, triples):
         """triples: int32 host tensor [n, 3] of (batch row, logical page, physical page), pinned for an asynchronous copy."""

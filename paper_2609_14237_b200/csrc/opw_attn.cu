@@ -156,6 +156,9 @@ struct opw_attn_stage {
   int64_t launches;
   unsigned char* ws;
   uint64_t* trace;
+  // OPW_FLAG_COPY_STREAMS: the host-buffer step's copies run on streams of their own
+  cudaStream_t s_in, s_out;
+  cudaEvent_t e_in, e_k, e_out;
 };
 
 extern "C" {
@@ -194,7 +197,7 @@ size_t opw_attn_stage_workspace_bytes(const opw_attn_stage_config_t* cfg) {
 opw_status_t opw_attn_stage_create(const opw_attn_stage_config_t* cfg, opw_attn_stage_t** out) {
   if (!cfg || !out) return OPW_ERR_INVALID_ARG;
   if (cfg->struct_size != sizeof(opw_attn_stage_config_t) || cfg->reserved != 0) return OPW_ERR_INVALID_ARG;
-  if (cfg->flags & ~(uint32_t)OPW_FLAG_NO_PDL) return OPW_ERR_INVALID_ARG;
+  if (cfg->flags & ~(uint32_t)(OPW_FLAG_NO_PDL | OPW_FLAG_COPY_STREAMS)) return OPW_ERR_INVALID_ARG;
   if (!shape_ok(cfg) || cfg->device < 0) return OPW_ERR_INVALID_ARG;
   if (!cfg->layer_window || !cfg->layer_num_pages || !cfg->layer_kv_pool || !cfg->workspace) return OPW_ERR_INVALID_ARG;
   if (cfg->head_dim != 64 && cfg->head_dim != 128 && cfg->head_dim != 256) return OPW_ERR_UNSUPPORTED;
@@ -271,12 +274,39 @@ opw_status_t opw_attn_stage_create(const opw_attn_stage_config_t* cfg, opw_attn_
   st->launches = 0;
   st->trace = nullptr;
   st->ws = static_cast<unsigned char*>(cfg->workspace);
+  st->s_in = st->s_out = nullptr;
+  st->e_in = st->e_k = st->e_out = nullptr;
+  if (cfg->flags & OPW_FLAG_COPY_STREAMS) {
+    bool ok = cudaStreamCreateWithFlags(&st->s_in, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&st->s_out, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&st->e_in, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&st->e_k, cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&st->e_out, cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+      (void)cudaGetLastError();
+      opw_attn_stage_destroy(st);
+      return OPW_ERR_CUDA;
+    }
+  }
   *out = st;
   return OPW_OK;
 }
 
 opw_status_t opw_attn_stage_destroy(opw_attn_stage_t* st) {
+  if (!st) return OPW_OK;
+  if (st->e_in) cudaEventDestroy(st->e_in);
+  if (st->e_k) cudaEventDestroy(st->e_k);
+  if (st->e_out) cudaEventDestroy(st->e_out);
+  if (st->s_in) cudaStreamDestroy(st->s_in);
+  if (st->s_out) cudaStreamDestroy(st->s_out);
   delete st;
+  return OPW_OK;
+}
+
+opw_status_t opw_attn_stage_wait_host_output(opw_attn_stage_t* st) {
+  if (!st) return OPW_ERR_INVALID_ARG;
+  if (!st->e_out) return OPW_OK;                 // without copy streams the caller synchronises its own stream
+  if (cudaEventSynchronize(st->e_out) != cudaSuccess) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
   return OPW_OK;
 }
 
@@ -523,7 +553,13 @@ opw_status_t opw_decode_step_host(opw_attn_stage_t* st, int32_t layer, int32_t b
   const size_t table_elems = (size_t)st->cfg.max_batch * st->cfg.max_pages_per_seq;
   int32_t* d_table = reinterpret_cast<int32_t*>(ws + st->lay.st_table) + (size_t)layer * table_elems;
 
+  // With OPW_FLAG_COPY_STREAMS the copies in run on the stage's own stream, the kernels on the caller's, the
+  // copies out on a third, chained by events: a second stage's kernels on the same stream then follow this
+  // stage's kernels directly, and both stages' copies hide behind them.
+  const bool split_streams = st->s_in != nullptr;
+  cudaStream_t sin = split_streams ? st->s_in : stream, sout = split_streams ? st->s_out : stream;
   bool ok = true;
+  if (split_streams) ok &= cudaStreamWaitEvent(sin, st->e_k, 0) == cudaSuccess;   // the staged inputs of the previous step are no longer read
   // Tensor packing: if the caller laid q, k_new, v_new and positions out in one host buffer at the
   // offsets of opw_attn_stage_host_layout, they travel as a single copy.
   const unsigned char* hq = static_cast<const unsigned char*>(q_host);
@@ -531,21 +567,31 @@ opw_status_t opw_decode_step_host(opw_attn_stage_t* st, int32_t layer, int32_t b
                       static_cast<const unsigned char*>(v_new_host) == hq + (st->lay.st_v - st->lay.st_q) &&
                       reinterpret_cast<const unsigned char*>(positions_host) == hq + (st->lay.st_pos - st->lay.st_q);
   if (packed) {
-    ok &= cudaMemcpyAsync(d_q, q_host, (st->lay.st_pos - st->lay.st_q) + B * 4, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d_q, q_host, (st->lay.st_pos - st->lay.st_q) + B * 4, cudaMemcpyHostToDevice, sin) == cudaSuccess;
   } else {
-    ok &= cudaMemcpyAsync(d_q, q_host, B * Hq * D * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
-    ok &= cudaMemcpyAsync(d_k, k_new_host, B * Hkv * D * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
-    ok &= cudaMemcpyAsync(d_v, v_new_host, B * Hkv * D * 2, cudaMemcpyHostToDevice, stream) == cudaSuccess;
-    ok &= cudaMemcpyAsync(d_pos, positions_host, B * 4, cudaMemcpyHostToDevice, stream) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d_q, q_host, B * Hq * D * 2, cudaMemcpyHostToDevice, sin) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d_k, k_new_host, B * Hkv * D * 2, cudaMemcpyHostToDevice, sin) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d_v, v_new_host, B * Hkv * D * 2, cudaMemcpyHostToDevice, sin) == cudaSuccess;
+    ok &= cudaMemcpyAsync(d_pos, positions_host, B * 4, cudaMemcpyHostToDevice, sin) == cudaSuccess;
   }
   if (page_table_host)
     ok &= cudaMemcpyAsync(d_table, page_table_host, B * st->cfg.max_pages_per_seq * 4, cudaMemcpyHostToDevice,
-                          stream) == cudaSuccess;
+                          sin) == cudaSuccess;
+  if (split_streams) {
+    ok &= cudaEventRecord(st->e_in, sin) == cudaSuccess;
+    ok &= cudaStreamWaitEvent(stream, st->e_in, 0) == cudaSuccess;
+    ok &= cudaStreamWaitEvent(stream, st->e_out, 0) == cudaSuccess;                 // the staged output of the previous step has left
+  }
   if (!ok) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
   rc = opw_decode_step(st, layer, batch, d_q, d_k, d_v, d_pos, d_table, d_out, lse_host ? d_lse : nullptr, cuda_stream);
   if (rc != OPW_OK) return rc;
-  ok &= cudaMemcpyAsync(out_host, d_out, B * Hq * D * 2, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
-  if (lse_host) ok &= cudaMemcpyAsync(lse_host, d_lse, B * Hq * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+  if (split_streams) {
+    ok &= cudaEventRecord(st->e_k, stream) == cudaSuccess;
+    ok &= cudaStreamWaitEvent(sout, st->e_k, 0) == cudaSuccess;
+  }
+  ok &= cudaMemcpyAsync(out_host, d_out, B * Hq * D * 2, cudaMemcpyDeviceToHost, sout) == cudaSuccess;
+  if (lse_host) ok &= cudaMemcpyAsync(lse_host, d_lse, B * Hq * 4, cudaMemcpyDeviceToHost, sout) == cudaSuccess;
+  if (split_streams) ok &= cudaEventRecord(st->e_out, sout) == cudaSuccess;
   if (!ok) { (void)cudaGetLastError(); return OPW_ERR_CUDA; }
   return OPW_OK;
 }

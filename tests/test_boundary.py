@@ -100,7 +100,7 @@ def test_workspace_bytes_needs_a_valid_shape():
     (dict(softmax_scale=-1.0), B.OPW_ERR_INVALID_ARG),
     (dict(head_dim=128, tune_warps=8, tune_stages=4), B.OPW_ERR_CAPACITY),
     (dict(max_batch=0), B.OPW_ERR_INVALID_ARG),
-    (dict(flags=2), B.OPW_ERR_INVALID_ARG),                      # only OPW_FLAG_NO_PDL is defined
+    (dict(flags=4), B.OPW_ERR_INVALID_ARG),                      # only OPW_FLAG_NO_PDL and OPW_FLAG_COPY_STREAMS are defined
 ])
 def test_create_rejects_bad_configs_before_touching_cuda(over, want):
     cfg, keep = good_cfg(**over)

@@ -469,6 +469,48 @@ def test_host_buffer_step_matches_the_device_step():
     st.close()
 
 
+def test_two_stages_with_copy_streams_take_turns_on_one_compute_stream():
+    """Two microbatches, a stage handle each (OPW_FLAG_COPY_STREAMS), both enqueuing on one compute stream: copies in
+    and out run on the stages' own streams.  Twelve steps without waiting for anything but each stage's previous
+    output; pools and every output against the oracle."""
+    steps = 12
+    wl = synth.Workload("cs", 6, 32, 8, 128, [0, 64], "uniform_1024_4096", 85)
+    inp = synth.make_inputs(wl, device="cpu", growth=steps, steps=steps, lengths=np.array([5, 200, 1023, 64, 15, 3000], np.int32))
+    pools = [p.cuda() for p in inp.pools]
+    refs = [oracle.as_u16(p).copy() for p in inp.pools]
+    stages = [B.Stage(pools=pools, layer_window=wl.layer_window, num_q_heads=32, num_kv_heads=8, head_dim=128, max_batch=6,
+                      max_pages_per_seq=inp.max_pages_per_seq, flags=B.OPW_FLAG_COPY_STREAMS) for _ in range(2)]
+    compute = torch.cuda.Stream()
+    packs = [[stages[l].packed_host_buffers(6) for _ in range(2)] for l in range(2)]     # [layer = microbatch][double buffer]
+    outs = torch.empty(steps, 2, 6, 32, 128, dtype=torch.bfloat16).pin_memory()
+    lses = torch.empty(steps, 2, 6, 32, dtype=torch.float32).pin_memory()
+    tabs = [t.pin_memory() for t in inp.page_tables]
+    for step in range(steps):
+        for layer in range(2):                               # microbatch `layer` owns layer `layer` and stage `layer`
+            st = stages[layer]
+            st.wait_host_output()
+            _, q, k, v, pos = packs[layer][step & 1]
+            q.copy_(inp.q[step, layer]); k.copy_(inp.k_new[step, layer]); v.copy_(inp.v_new[step, layer])
+            pos.copy_(torch.from_numpy(inp.positions(step)))
+            with torch.cuda.stream(compute):
+                st.decode_step_host(layer, q, k, v, pos, tabs[layer] if step == 0 else None, outs[step, layer], lses[step, layer])
+    for st in stages:
+        st.wait_host_output()
+    torch.cuda.synchronize()
+    assert all(st.poll_error() == B.OPW_OK for st in stages)
+    for step in range(steps):
+        for layer in range(2):
+            assert oracle.kv_append(refs[layer], 8, 128, P, inp.k_new[step, layer], inp.v_new[step, layer],
+                                    inp.positions(step), inp.page_tables[layer]) == 0
+            ref, ref_lse, _ = oracle.decode_attention(refs[layer], 32, 8, 128, P, inp.q[step, layer], inp.kv_lens(step),
+                                                      inp.page_tables[layer], window=wl.layer_window[layer])
+            check_close(out_to_f64(outs[step, layer]), ref, lses[step, layer].numpy().astype(np.float64), ref_lse)
+    for layer in range(2):
+        assert (pools[layer].cpu().view(torch.int16).numpy().view(np.uint16) == refs[layer]).all()
+    for st in stages:
+        st.close()
+
+
 def test_host_steps_with_page_table_deltas_equal_steps_with_the_table_resent_in_full():
     """Forty decode steps from host buffers, twice: once re-sending the whole page table every step, once sending it
     in full at the first step only (with the pages of later steps still unmapped) and from then on just the
