@@ -117,6 +117,7 @@ struct opw_afd_module {
   size_t off_qkv, off_q, off_k, off_v, off_out, off_gemm, off_partials, off_tickets, off_angles, off_status;
   // tensor-core path
   bool tc_qkv, tc_o, pdl, coop_ok;
+  int max_clusters[opw_afd::kMaxSplit + 1];   // [ks]: thread-block clusters of (1, ks, 1) of the GEMM kernel the device holds at once
   int sms;
   TensorMapEncodeFn encode;
   CUtensorMap map_wqkv, map_wo;
@@ -207,14 +208,21 @@ bool encode_map(TensorMapEncodeFn fn, CUtensorMap* map, const void* base, uint64
 // `coop`: a cooperative launch -- the whole grid is resident at once or the launch is refused.
 template <typename... KArgs, typename... Args>
 cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, bool pdl, bool coop,
-                       Args&&... args) {
+                       int cluster_y, Args&&... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
   cfg.dynamicSmemBytes = smem;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[2];
+  cudaLaunchAttribute attr[3];
   int n = 0;
+  if (cluster_y > 1) {                          // thread-block clusters of (1, cluster_y, 1)
+    attr[n].id = cudaLaunchAttributeClusterDimension;
+    attr[n].val.clusterDim.x = 1;
+    attr[n].val.clusterDim.y = (unsigned)cluster_y;
+    attr[n].val.clusterDim.z = 1;
+    ++n;
+  }
   if (pdl) {
     attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[n].val.programmaticStreamSerializationAllowed = 1;
@@ -242,12 +250,25 @@ opw_status_t run_tc_gemm(opw_afd_module* m, const CUtensorMap& map_w, const void
   // kernel launched just before) for large ones and wherever the table would leave the ring too small.
   // The epilogue reuses the ring: one tile of sums for all columns, or two tiles for a chunk of columns.
   p.ksplit = ksplit_of(n_out, k, batch, m->sms < kSmsBound ? m->sms : kSmsBound);
+  // The K-split CTAs of a weight tile exchange their partial tiles inside a thread-block cluster when the device
+  // can hold every cluster of the launch at once (a cluster needs its SMs in one GPC, so fewer CTAs fit than
+  // there are SMs: 45 clusters of three on a B200 with 148 SMs, 33 of four, 74 of two); a narrower split that
+  // fits is preferred to a wider one that does not.
+  p.cluster = 0;
+  if (p.group == 1 && p.ksplit > 1) {
+    for (int ks = p.ksplit; ks >= 2; --ks)
+      if (tiles_of(n_out) * batch_tiles_of(batch) <= m->max_clusters[ks]) {
+        p.ksplit = ks;
+        p.cluster = 1;
+        break;
+      }
+  }
   const int ctas = tiles_of(n_out) * p.ksplit * batch_tiles_of(batch);
   // The shared back end pays at large batches, where publishing and reducing the partial tiles is bandwidth work
   // that a third of the CTAs would otherwise do alone (batch 256: 31 -> 27 us for the QKV projection); at small
   // batches the back end is a latency chain either way, and a cooperative launch cannot start under the previous
   // kernel's tail, which costs more than the sharing gives (batch 64: 149 -> 157 us per module step).
-  p.coop = (m->coop_ok && ctas <= m->sms && (p.ksplit > 1 || p.group > 1) && batch > kCoopMinBatch) ? 1 : 0;
+  p.coop = (!p.cluster && m->coop_ok && ctas <= m->sms && (p.ksplit > 1 || p.group > 1) && batch > kCoopMinBatch) ? 1 : 0;
   const int chunk_cols = batch < opw_afd::kChunkCols ? batch : opw_afd::kChunkCols;
   const int members = p.ksplit * p.group;
   // cooperative back end: the CTA's own tile, plus (two-tile heads) its slice of the other tile's sums
@@ -280,7 +301,7 @@ opw_status_t run_tc_gemm(opw_afd_module* m, const CUtensorMap& map_w, const void
   // trace region 0: output projection, region 1: QKV projection
   p.trace = m->trace ? m->trace + (size_t)mode * opw_afd::kTraceMaxCtas * opw_afd::kTraceWords : nullptr;
   if (angles_global) {
-    if (launch_pdl(opw_afd::rope_table_kernel, dim3(batch), dim3(128), 0, stream, m->pdl, false, positions,
+    if (launch_pdl(opw_afd::rope_table_kernel, dim3(batch), dim3(128), 0, stream, m->pdl, false, 0, positions,
                    reinterpret_cast<float2*>(m->ws + m->off_angles), (int)m->D, m->log_theta) != cudaSuccess) {
       (void)cudaGetLastError();
       return OPW_ERR_CUDA;
@@ -291,7 +312,7 @@ opw_status_t run_tc_gemm(opw_afd_module* m, const CUtensorMap& map_w, const void
   if (!encode_map(m->encode, &map_x, x, (uint64_t)batch, (uint64_t)k, (uint32_t)p.nb)) return OPW_ERR_CUDA;
   const dim3 grid(tiles_of(n_out), p.ksplit, batch_tiles_of(batch));
   if (launch_pdl(opw_afd::skinny_gemm_kernel, grid, dim3(opw_afd::kGemmThreads), 1024 + (size_t)stages * stage_bytes + angle_bytes,
-                 stream, m->pdl, p.coop != 0, map_w, map_x, p) != cudaSuccess) {
+                 stream, m->pdl, p.coop != 0, p.cluster ? p.ksplit : 0, map_w, map_x, p) != cudaSuccess) {
     (void)cudaGetLastError();
     return OPW_ERR_CUDA;
   }
@@ -356,6 +377,21 @@ opw_status_t opw_afd_module_create(opw_attn_stage_t* stage, int32_t layer, int32
     m->coop_ok = coop != 0;
     ok = ok && cudaFuncSetAttribute(opw_afd::skinny_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)kGemmSmemBudget) == cudaSuccess;
+    for (int ks = 0; ks <= opw_afd::kMaxSplit; ++ks) m->max_clusters[ks] = 0;
+    for (int ks = 2; ok && ks <= opw_afd::kMaxSplit; ++ks) {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(1, ks, 1);
+      cfg.blockDim = dim3(opw_afd::kGemmThreads);
+      cfg.dynamicSmemBytes = kGemmSmemBudget;      // the most a launch asks for
+      cudaLaunchAttribute at;
+      at.id = cudaLaunchAttributeClusterDimension;
+      at.val.clusterDim.x = 1; at.val.clusterDim.y = (unsigned)ks; at.val.clusterDim.z = 1;
+      cfg.attrs = &at;
+      cfg.numAttrs = 1;
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, opw_afd::skinny_gemm_kernel, &cfg) != cudaSuccess) { (void)cudaGetLastError(); n = 0; }
+      m->max_clusters[ks] = n;
+    }
     const int n_qkv = (Hq + 2 * Hkv) * D, n_attn = Hq * D;
     ok = ok && encode_map(m->encode, &m->map_wqkv, w_qkv, (uint64_t)n_qkv, (uint64_t)hidden, opw_afd::kTileM);
     ok = ok && encode_map(m->encode, &m->map_wo, w_o, (uint64_t)hidden, (uint64_t)n_attn, opw_afd::kTileM);

@@ -13,13 +13,18 @@
 // four column groups) -- the epilogue is a chain of L2 round trips, so it wants many threads.
 //
 // With N/128 tiles alone a 6144 x 4096 projection would occupy 48 of 148 SMs, too few to pull
-// the weights at HBM speed, so K is also split over `ksplit` CTAs per tile; each writes its fp32
-// partial tile to a workspace.  When the whole grid fits the device (a cooperative launch guarantees
-// that every CTA is resident) the CTAs of a tile meet at a counter and each of them reduces and
-// finishes its own slice of the batch columns -- the back end would otherwise sit on a third of the
-// SMs while the others idle; with more CTAs than SMs nobody may wait, and the last CTA of a tile to
-// arrive (an atomic ticket) reduces and finishes all of it.  Either way the partial tiles are added
-// in split order: deterministic.
+// the weights at HBM speed, so K is also split over `ksplit` CTAs per tile, and the partial tiles
+// have to meet.  Three back ends, chosen by the host:
+//   * cluster: the ksplit CTAs of a tile are one thread-block cluster (1, ksplit, 1).  They are resident
+//     together by construction, meet at the cluster's hardware barrier, and each adds up and finishes its own
+//     slice of the batch columns, reading the other members' tiles from their shared memory.  Used whenever
+//     the device holds all clusters of the launch at once (a cluster needs its SMs in one GPC).
+//   * cooperative: the whole grid is resident (cooperative launch); the CTAs of a tile meet at a counter in
+//     global memory and share the back end the same way, the partial tiles passing through the workspace.
+//     Used for heads that span two weight tiles (D = 256) at large batches.
+//   * last CTA: with no residency guarantee nobody may wait; every CTA writes its partial tile to the
+//     workspace and the last one of a tile to arrive (an atomic ticket) reduces and finishes all of it.
+// In all three the partial tiles are added in split order: deterministic.
 //
 // Epilogues: plain (bf16 C[b, n]) and rotary (the QKV projection of the attention module: pairs
 // (d, d + D/2) of the q and k heads are rotated, still as fp32 accumulators, by angles that the
@@ -57,6 +62,8 @@ struct GemmParams {
   int nb;                 // MMA N of a full batch tile: min(batch, 256) rounded up to a multiple of 16
   int group;              // weight tiles that share a ticket and an epilogue: 1, or 2 (rotary at D = 256)
   int coop;               // the launch is cooperative (every CTA resident): the CTAs of a ticket group share the back end
+  int cluster;            // the ksplit CTAs of a weight tile form a thread-block cluster (1, ksplit, 1): they exchange their
+                          // partial tiles through distributed shared memory (group == 1 only)
   const float2* angles_g; // mode 1: [batch, D/2] (cos, sin) in global memory, or null: computed here in shared memory
   int stages;
   int ksplit;
@@ -154,6 +161,27 @@ __device__ __forceinline__ void g_tmem_ld16(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// Thread-block cluster: the shared-memory address of the same variable in the CTA of rank `rank`, loads from
+// it, and the cluster's hardware barrier (split in two halves; it does not spin, every CTA of a cluster is
+// resident with the others).
+__device__ __forceinline__ uint32_t g_mapa(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ float4 g_ld_cluster_f4(uint32_t addr) {
+  float4 v;
+  asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ uint32_t g_ld_cluster_u32(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.shared::cluster.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void g_cluster_arrive() { asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory"); }
+__device__ __forceinline__ void g_cluster_wait() { asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory"); }
+
 // Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes, stored as TMA's
 // 128-byte swizzle leaves them: 8-row groups 1024 bytes apart (stride byte offset), leading
 // byte offset unused (1), descriptor version 1, layout type 2 = 128-byte swizzle.  Addresses and
@@ -237,6 +265,7 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
   __shared__ uint32_t tmem_slot;
   __shared__ volatile int s_fail;
   __shared__ int s_last;
+  __shared__ volatile uint32_t s_flags[kMaxSplit];           // written by the other CTAs of a cluster: their accumulators are good
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int tile = blockIdx.x, split = blockIdx.y;
@@ -436,6 +465,73 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     const float4* part = reinterpret_cast<const float4*>(p.partials + (size_t)pt * p.ksplit * split_floats) + (size_t)cb * kTileM / 4;
     gemm_reduce_partials(part, reinterpret_cast<float4*>(dst), (ce - cb) * kTileM / 4, p.ksplit, own ? split : -1, split_floats / 4);
   };
+
+  if (p.cluster) {
+    // ---- hand-off inside a thread-block cluster: the ksplit CTAs of this weight tile run at the same time on
+    // SMs of one GPC (a cluster is resident as a whole), meet at the cluster's hardware barrier instead of
+    // counting arrivals in global memory, and read each other's shared memory.  Member r takes a slice of the
+    // batch columns, adds that slice of all members' tiles in split order and finishes it.  Every CTA passes
+    // both barriers whatever happened to it (its waits are bounded), so no member is left waiting; a member that
+    // failed makes all skip the epilogue.
+    // Measured alternatives: members sending their accumulators into the owner's shared memory with remote
+    // stores, and members exchanging the slices through the workspace in L2 with only the barrier taken from the
+    // cluster, were both slower (the cluster's network moves some 20 GB/s per SM either way; a write to L2 and a
+    // read back are two round trips where this is one). ----
+    const int ks = p.ksplit;
+    if (tid == 0) s_flags[0] = good ? 1u : 0u;
+    g_cluster_arrive();
+    g_cluster_wait();
+    g_stamp(p, cta, 4);
+    const int cb = (int)((int64_t)batch_here * split / ks), ce = (int)((int64_t)batch_here * (split + 1) / ks);
+    float* mine = stage_f + (size_t)cb * kTileM;
+    // The members' flags and the values are requested together: one round trip through the cluster's network,
+    // not one per member.  The sums are formed whatever the flags say (a failed member's tile is just numbers);
+    // only the epilogue depends on them.
+    uint32_t flag[kMaxSplit];
+    const uint32_t flag_local = g_smem_u32(const_cast<uint32_t*>(&s_flags[0]));
+#pragma unroll
+    for (int sp = 0; sp < kMaxSplit; ++sp) flag[sp] = sp < ks ? g_ld_cluster_u32(g_mapa(flag_local, (uint32_t)sp)) : 1u;
+    {
+      const int n4 = (ce - cb) * kTileM / 4;
+      float4* dst = reinterpret_cast<float4*>(mine);
+      const uint32_t local = g_smem_u32(dst);
+      uint32_t remote[kMaxSplit];
+#pragma unroll
+      for (int sp = 0; sp < kMaxSplit; ++sp) remote[sp] = sp < ks ? g_mapa(local, (uint32_t)sp) : 0u;
+      constexpr int R = 2;
+      for (int ib = tid; ib < n4; ib += R * kGemmThreads) {
+        float4 v[R][kMaxSplit];
+#pragma unroll
+        for (int r = 0; r < R; ++r)
+#pragma unroll
+          for (int sp = 0; sp < kMaxSplit; ++sp) {
+            const int i = ib + r * kGemmThreads;
+            if (i < n4 && sp < ks && sp != split) v[r][sp] = g_ld_cluster_f4(remote[sp] + 16u * (uint32_t)i);
+          }
+#pragma unroll
+        for (int r = 0; r < R; ++r) {
+          const int i = ib + r * kGemmThreads;
+          if (i >= n4) break;
+          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+          for (int sp = 0; sp < kMaxSplit; ++sp)
+            if (sp < ks) {
+              const float4 t = sp == split ? dst[i] : v[r][sp];
+              acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+            }
+          dst[i] = acc;
+        }
+      }
+    }
+    const bool all_good = (flag[0] & flag[1] & flag[2] & flag[3]) != 0;
+    __syncthreads();
+    g_cluster_arrive();                         // this CTA no longer reads the others' shared memory
+    g_stamp(p, cta, 5);
+    if (all_good && ce > cb) epilogue(tile, mine, mine, cb, ce);
+    g_cluster_wait();                           // and leaves only when nobody reads its own any more
+    g_stamp(p, cta, 6);
+    return;
+  }
 
   if (!shared_epilogue) {                     // one CTA holds the whole sum of its tile
     if (good) epilogue(tile, stage_f, stage_f, 0, batch_here);
