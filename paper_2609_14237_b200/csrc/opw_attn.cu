@@ -31,7 +31,7 @@ struct Shape {
 };
 
 struct Layout {          // byte offsets into the caller's workspace
-  size_t status, cum[2], partials[2], comb_scratch, row_count, st_q, st_k, st_v, st_pos, st_out, st_lse, st_delta, st_table, total;
+  size_t status, cum[2], partials[2], split_list[2], comb_scratch, row_count, st_q, st_k, st_v, st_pos, st_out, st_lse, st_delta, st_table, total;
 };
 
 bool shape_ok(const opw_attn_stage_config_t* c) {
@@ -68,6 +68,7 @@ Layout carve(const opw_attn_stage_config_t* c, const Shape& s, int sms) {
   for (int i = 0; i < 2; ++i) {        // two sets: a plan may run a step's combine beside the next attention
     L.cum[i] = off;      off += align_up((B + 2) * 4, 256);
     L.partials[i] = off; off += align_up(workers * 2 * opw::kSegPerShare * G * (D + 2) * 4, 256);
+    L.split_list[i] = off; off += align_up(B * Hkv * 4, 256);   // rows left as partials, in launches with very many rows
   }
   L.comb_scratch = off; off += align_up((size_t)kCombineScratchSlots * G * (D + 2) * 4, 256);
   L.row_count = off; off += align_up(B * Hkv * 4, 256);
@@ -387,6 +388,11 @@ static opw_status_t validate_step(opw_attn_stage_t* st, const StepArgs& a) {
 }
 
 // The split-KV kernel of one step, using workspace set `ws_set` (0 or 1).
+// Launches with this many (sequence, kv head) rows or more have the attention kernel list the rows it leaves
+// as partials and the combine walk that list instead of running a block per row (see combine_kernel).
+constexpr int kRowListMin = 4096;
+static inline bool use_row_list(const opw_attn_stage_t* st, int batch) { return batch * st->cfg.num_kv_heads >= kRowListMin; }
+
 static opw_status_t launch_attention(opw_attn_stage_t* st, const StepArgs& a, int ws_set, cudaStream_t stream) {
   const int D = st->cfg.head_dim, Hq = st->cfg.num_q_heads, Hkv = st->cfg.num_kv_heads, G = Hq / Hkv;
   opw::AttnParams p;
@@ -404,6 +410,8 @@ static opw_status_t launch_attention(opw_attn_stage_t* st, const StepArgs& a, in
   p.cum = reinterpret_cast<int32_t*>(st->ws + st->lay.cum[ws_set]);
   p.status = reinterpret_cast<uint32_t*>(st->ws + st->lay.status);
   p.ticket = reinterpret_cast<int32_t*>(st->ws + st->lay.status + 16 + 16 * ws_set);
+  p.split_list = use_row_list(st, a.batch) ? reinterpret_cast<int32_t*>(st->ws + st->lay.split_list[ws_set]) : nullptr;
+  p.split_count = reinterpret_cast<int32_t*>(st->ws + st->lay.status + 64 + 32 * ws_set);
   p.trace = st->trace;
   p.num_pages = st->num_pages[a.layer];
   p.batch = a.batch;
@@ -456,6 +464,9 @@ static opw_status_t launch_combine(opw_attn_stage_t* st, const StepArgs& a, int 
   c.num_workers = st->grid * st->shape.warps;
   c.scratch = reinterpret_cast<float*>(st->ws + st->lay.comb_scratch);
   c.row_count = reinterpret_cast<int32_t*>(st->ws + st->lay.row_count);
+  const bool listed = use_row_list(st, a.batch);
+  c.split_list = listed ? reinterpret_cast<const int32_t*>(st->ws + st->lay.split_list[ws_set]) : nullptr;
+  c.split_count = reinterpret_cast<int32_t*>(st->ws + st->lay.status + 64 + 32 * ws_set);
   // Few rows can have very many partials each (long contexts at small batch): split each row's
   // merge over several blocks so that about one block per SM is busy (two per SM measured slower:
   // the hand-off between a row's blocks costs more than the extra parallelism gives).
@@ -465,7 +476,8 @@ static opw_status_t launch_combine(opw_attn_stage_t* st, const StepArgs& a, int 
   if (splits > kCombineScratchSlots / rows) splits = kCombineScratchSlots / rows;
   if (splits < 1) splits = 1;
   const bool pdl = (st->cfg.flags & OPW_FLAG_NO_PDL) == 0 && !side_stream;
-  const dim3 grid(rows, splits);
+  const int list_blocks = st->sms * (small ? 4 : 2);
+  const dim3 grid(listed ? (rows < list_blocks ? rows : list_blocks) : rows, listed ? 1 : splits);
   cudaError_t e;
 #define OPW_LAUNCH_COMBINE(DIM)                                                                                            \
   e = small ? launch(opw::combine_kernel<opw::kCombineThreadsSmall, DIM>, grid, dim3(opw::kCombineThreadsSmall), 0, stream, \

@@ -52,6 +52,8 @@ struct AttnParams {
   int32_t* cum;          // [batch+1] pages before sequence b (written by block 0)
   uint32_t* status;
   int32_t* ticket;       // dynamic-chunk counter, zero at launch (the combine kernel re-zeroes it)
+  int32_t* split_list;   // or null.  Many-row launches: the rows left as partials, each listed once, by the worker
+  int32_t* split_count;  // whose segment holds the row's first unit; [0] their number (zero at launch; the combine re-zeroes it)
   uint64_t* trace;       // optional [num_workers][4]: {smid | units<<32, t_begin, t_first_tile, t_end} in ns
   int64_t num_pages;
   int32_t batch, Hq, Hkv, G;
@@ -808,6 +810,7 @@ __global__ void __maxnreg__(D > 128 ? 255 : 200) attn_splitkv_kernel(AttnParams 
         }
       } else {
         // partial: unnormalised o, running max and sum, into this worker's slot
+        if (p.split_list != nullptr && seg_from_first && lane == 0) p.split_list[atomicAdd(p.split_count, 1)] = row;
         const int64_t pslot = slot_base + (seg_on_first_row ? 0 : 1);
         float* pb = p.partials + pslot * (int64_t)(p.G * (D + 2));
         if (qrow < p.G) {
@@ -864,6 +867,8 @@ struct CombineParams {
   const int32_t* positions;
   float* scratch;             // [rows * splits][G*(D+2)] intermediates (used when gridDim.y > 1)
   int32_t* row_count;         // [rows] arrival counters, zero between launches
+  const int32_t* split_list;  // or null.  List mode (many rows, most of them complete): the rows to merge, as the attention
+  int32_t* split_count;       // kernel listed them; [0] their number, [1] blocks that have read it (both zero between launches)
   __nv_bfloat16* out;
   float* lse;
   int32_t batch, Hq, Hkv, G, D;
@@ -925,11 +930,11 @@ __device__ __forceinline__ void combine_accumulate(float* acc, const float* part
 // nothing waits) merges those `splits` intermediates and writes the output.
 // kD: the head dimension as a compile-time constant (0: read it from the parameters); the kernel is
 // bound by integer arithmetic more than by memory, and divisions by D are a good part of it.
-template <int kCT, int kD = 0>
-__global__ void __launch_bounds__(kCT, kCT == 128 ? 5 : 2) combine_kernel(CombineParams p) {
-  pdl_launch_dependents();
-  const int row = blockIdx.x;
-  const int splits = gridDim.y, split = blockIdx.y;
+// One row (and split).  `listed`: list mode -- the dependency wait is behind the caller, the row is known to be
+// split, and the prefix sums are read from memory.
+template <int kCT, int kD>
+__device__ __forceinline__ void combine_row(const CombineParams& p, const int row, const int split, const int splits,
+                                            const bool listed) {
   const int b = row / p.Hkv, g = row - b * p.Hkv;
   const int D = kD ? kD : p.D, G = p.G;
   const int GD = G * D;
@@ -963,7 +968,7 @@ __global__ void __launch_bounds__(kCT, kCT == 128 ? 5 : 2) combine_kernel(Combin
   // first batch of candidates -- so that under programmatic dependent launch all of it runs beneath the
   // attention kernel's tail and only the loads of the partials are left for afterwards.  Larger batches
   // read the prefix sums the attention kernel stored, after the wait.
-  const bool early = p.batch <= kCombineScanBatch;
+  const bool early = !listed && p.batch <= kCombineScanBatch;
   int32_t cum_b = 0, cum_all = 0, cnt = 0;
   int64_t U = 0, ustart = 0, uend = 0, wf = 0, wl = 0, ncand = 0;
   ShareMath sm;
@@ -1060,8 +1065,10 @@ __global__ void __launch_bounds__(kCT, kCT == 128 ? 5 : 2) combine_kernel(Combin
     prepare();
   }
 
-  pdl_wait();                                  // partials and complete rows are final now
-  if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *p.ticket = 0;
+  if (!listed) {
+    pdl_wait();                                // partials and complete rows are final now
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) *p.ticket = 0;
+  }
   __nv_bfloat16* ob = p.out + ((int64_t)b * p.Hq + (int64_t)g * G) * D;
   float* lse_row = p.lse ? p.lse + (int64_t)b * p.Hq + g * G : nullptr;
   if (n <= 0) {   // inactive slot: zeros, lse = -inf
@@ -1169,6 +1176,42 @@ __global__ void __launch_bounds__(kCT, kCT == 128 ? 5 : 2) combine_kernel(Combin
       ob[e] = __float2bfloat16_rn(Lh > 0.f ? acc[j] / Lh : 0.f);
       if (lse_row && e == h * D) lse_row[h] = Lh > 0.f ? (run_M[h] + log2f(Lh)) * 0.6931471805599453f : -INFINITY;
     }
+  }
+}
+
+
+// grid = (rows, splits), or in list mode (p.split_list set; splits == 1) any number of blocks: a launch with very
+// many rows has most of them complete (a row can only be split at one of the launch's segment boundaries, a few
+// thousand), and a block per row just to find that out costs more than the merges.  There the attention kernel
+// lists the rows it left as partials, and the blocks of this kernel walk that list; inactive rows, which no
+// worker sees, are found and zeroed here.
+template <int kCT, int kD = 0>
+__global__ void __launch_bounds__(kCT, kCT == 128 ? 5 : 2) combine_kernel(CombineParams p) {
+  pdl_launch_dependents();
+  if (p.split_list == nullptr) {
+    combine_row<kCT, kD>(p, blockIdx.x, blockIdx.y, gridDim.y, false);
+    return;
+  }
+  __shared__ int32_t n_listed;
+  pdl_wait();                                  // the list, the partials and the complete rows are final now
+  if (threadIdx.x == 0) {
+    n_listed = __ldcg(p.split_count);
+    if (blockIdx.x == 0) *p.ticket = 0;
+    // the last block to have read the count puts both counters back to zero for the next launch
+    if (atomicAdd(p.split_count + 1, 1) == (int32_t)gridDim.x - 1) { p.split_count[0] = 0; p.split_count[1] = 0; }
+  }
+  __syncthreads();
+  const int D = kD ? kD : p.D;
+  for (int b = blockIdx.x; b < p.batch; b += gridDim.x) {     // inactive slots: zeros, lse = -inf
+    if (visible_keys(p.kv_lens, p.positions, b) > 0) continue;
+    __nv_bfloat16* ob = p.out + (int64_t)b * p.Hq * D;
+    for (int e = threadIdx.x; e < p.Hq * D; e += kCT) ob[e] = __float2bfloat16(0.f);
+    if (p.lse) for (int h = threadIdx.x; h < p.Hq; h += kCT) p.lse[(int64_t)b * p.Hq + h] = -INFINITY;
+  }
+  const int n = n_listed;
+  for (int i = blockIdx.x; i < n; i += gridDim.x) {
+    combine_row<kCT, kD>(p, __ldcg(p.split_list + i), 0, 1, true);
+    __syncthreads();                           // the next row reuses the shared-memory state
   }
 }
 

@@ -135,6 +135,8 @@ extern "C" opw_status_t opw_decode_attention_noalloc(int32_t num_q_heads, int32_
   p.cum = reinterpret_cast<int32_t*>(ws + kStatusBytes);
   p.status = reinterpret_cast<uint32_t*>(ws);
   p.ticket = reinterpret_cast<int32_t*>(ws + 16);
+  p.split_list = nullptr;
+  p.split_count = nullptr;
   p.trace = nullptr;
   p.num_pages = num_pages;
   p.batch = batch;
@@ -177,6 +179,8 @@ extern "C" opw_status_t opw_decode_attention_noalloc(int32_t num_q_heads, int32_
   c.max_pages = max_pages_per_seq;
   c.window = window;
   c.num_workers = d->sms * kWarps;
+  c.split_list = nullptr;
+  c.split_count = nullptr;
   opw_na::combine_kernel<opw_na::kCombineThreads><<<batch * num_kv_heads, opw_na::kCombineThreads, 0, stream>>>(c);
   if (cudaGetLastError() != cudaSuccess) return OPW_ERR_CUDA;
   return OPW_OK;

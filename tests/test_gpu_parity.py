@@ -670,6 +670,35 @@ def test_overlapped_plan_with_an_empty_item_between_live_ones(flags):
     st.close()
 
 
+@pytest.mark.parametrize("flags", [0, B.OPW_PLAN_OVERLAP | B.OPW_PLAN_GRAPH])
+def test_plan_of_fused_steps_with_very_many_rows(flags):
+    """512 sequences x 8 kv heads = 4096 rows: list mode in every item of a plan (with the overlap flag the
+    combine of one item runs beside the next item's attention, each on its own list)."""
+    wl = synth.Workload("pl", 512, 16, 8, 64, [0, 40, 0], "uniform_1_200", 84)
+    inp = synth.make_inputs(wl, device="cpu", growth=1, steps=1)
+    pools = [p.cuda() for p in inp.pools]
+    refs = [oracle.as_u16(p).copy() for p in inp.pools]
+    st = B.Stage(pools=pools, layer_window=wl.layer_window, num_q_heads=16, num_kv_heads=8, head_dim=64,
+                 max_batch=512, max_pages_per_seq=inp.max_pages_per_seq)
+    dq, dk, dv = inp.q.cuda(), inp.k_new.cuda(), inp.v_new.cuda()
+    pos = dev(inp.positions(0))
+    tabs = [t.cuda() for t in inp.page_tables]
+    outs = [torch.full((512, 16, 64), float("nan"), dtype=torch.bfloat16, device="cuda") for _ in range(3)]
+    items = [dict(layer=l, batch=512, q=dq[0, l].data_ptr(), k_new=dk[0, l].data_ptr(), v_new=dv[0, l].data_ptr(),
+                  positions=pos.data_ptr(), page_table=tabs[l].data_ptr(), out=outs[l].data_ptr()) for l in range(3)]
+    plan = B.opw_attn_plan_create(st.handle, items, flags)
+    B.opw_attn_plan_submit(plan, torch.cuda.current_stream().cuda_stream)
+    assert st.poll_error() == B.OPW_OK
+    for l in range(3):
+        assert oracle.kv_append(refs[l], 8, 64, P, inp.k_new[0, l], inp.v_new[0, l], inp.positions(0), inp.page_tables[l]) == 0
+        ref, _, _ = oracle.decode_attention(refs[l], 16, 8, 64, P, inp.q[0, l], inp.kv_lens(0), inp.page_tables[l],
+                                            window=wl.layer_window[l])
+        check_close(out_to_f64(outs[l]), ref, max_abs=2.0 ** -8 * float(np.abs(ref).max()) + 1e-3)
+        assert (pools[l].cpu().view(torch.int16).numpy().view(np.uint16) == refs[l]).all()
+    B.opw_attn_plan_destroy(plan)
+    st.close()
+
+
 def test_overlapped_plan_needs_distinct_outputs_for_consecutive_items():
     pool = torch.zeros(4 * 2 * 2 * 16 * 64, dtype=torch.bfloat16, device="cuda")
     st = B.Stage(pools=[pool], layer_window=[0], num_q_heads=8, num_kv_heads=2, head_dim=64, max_batch=2, max_pages_per_seq=2)
@@ -775,6 +804,36 @@ def test_many_short_sequences_fill_the_static_batch():
     # where half a bf16 ulp is already 1.6e-2.  The absolute bound is stated for the benchmark
     # configurations; here the bound relative to the value (2^-8 |ref|, in check_close) is the binding one.
     check_close(out_to_f64(out), ref, lse, ref_lse, max_abs=2.0 ** -8 * float(np.abs(ref).max()) + 1e-3)
+
+
+@pytest.mark.parametrize("flags", [0, B.OPW_FLAG_NO_PDL])
+@pytest.mark.parametrize("window", [0, 48])
+def test_very_many_rows_list_mode_split_rows_complete_rows_and_inactive_slots(flags, window):
+    """batch x kv heads >= 4096: the attention kernel lists the rows it leaves as partials and the combine walks
+    that list; complete rows are final as the attention kernel wrote them, inactive slots are zeroed by the
+    combine.  Lengths 0..300 give all three kinds; two launches in a row check that the list's counters return
+    to zero."""
+    rng = np.random.default_rng(163)
+    Hq, Hkv, D = 16, 8, 64
+    lens = rng.integers(0, 301, size=640).astype(np.int32)
+    lens[rng.integers(0, 640, size=40)] = 0
+    lens = lens.tolist()
+    pool_np, tab, q_bits, _, _ = make_case(rng, [max(n, 1) for n in lens], Hq, Hkv, D)
+    ref, ref_lse, rc = oracle.decode_attention(pool_np, Hq, Hkv, D, P, q_bits, lens, tab, window=window)
+    assert rc == 0
+    pool = dev(pool_np, torch.bfloat16)
+    st = B.Stage(pools=[pool], layer_window=[window], num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, max_batch=len(lens),
+                 max_pages_per_seq=tab.shape[1], flags=flags)
+    q, kv, tb = dev(q_bits, torch.bfloat16), dev(np.asarray(lens, np.int32)), dev(tab.astype(np.int32))
+    for _ in range(2):
+        out = torch.full((len(lens), Hq, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+        lse = torch.full((len(lens), Hq), float("nan"), dtype=torch.float32, device="cuda")
+        st.decode_attention(0, q, kv, tb, out, lse)
+        assert st.poll_error() == B.OPW_OK
+        # short rows: the bound relative to the value is the binding one (see the test of many short sequences)
+        check_close(out_to_f64(out), ref, lse.cpu().numpy().astype(np.float64), ref_lse,
+                    max_abs=2.0 ** -8 * float(np.abs(ref).max()) + 1e-3)
+    st.close()
 
 
 def test_head_dim_256_long_rows_full_and_windowed():
