@@ -11,8 +11,10 @@
  *     y = out W_o^T
  * The two projections run on a hand-written tcgen05 kernel made for decode shapes: the weight
  * rows fill the tensor core's M dimension and TMEM lanes, the few batch rows its N dimension,
- * TMA streams the weights once, K is split over CTAs so that every SM pulls weights; batches of
- * more than 256 rows are walked in tiles of 256.  Only with OPW_AFD_LIBRARY_GEMM, kept as a
+ * TMA streams the weights once, K is split over CTAs so that every SM pulls weights (the K-splits of
+ * a weight tile run as one thread-block cluster and add up their tiles through each other's shared
+ * memory where the device can hold all clusters at once); batches of more than 256 rows are walked in
+ * tiles of 256.  Only with OPW_AFD_LIBRARY_GEMM, kept as a
  * comparison arm, are they cuBLASLt calls followed by a separate rotary kernel instead.
  * It exists to measure the contrast the paper's analysis rests on (Section 3.1: memory-bound
  * attention against GEMM-dominated projections) on the same device, and to let a caller move
