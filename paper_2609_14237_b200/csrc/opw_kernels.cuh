@@ -129,6 +129,7 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
 // Programmatic dependent launch: a kernel launched with the stream-serialization attribute may
 // start while its predecessor in the stream still runs; it must not touch anything the
 // predecessor (or, transitively, earlier kernels) produces before pdl_wait() returns.
+__device__ __forceinline__ void prefetch_l1(const void* p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
@@ -590,6 +591,11 @@ __global__ void __maxnreg__(D > 128 ? 255 : 200) attn_splitkv_kernel(AttnParams 
     nx = describe(n0 + lane, n1);
     next_known = true;
     next_issued = 0;
+    if (n0 < n1) {                            // the next segment starts with a row switch: its queries, its new key and value
+      const int64_t nrow = __shfl_sync(0xffffffffu, nx.row, 0);
+      if (lane * 64 < p.G * D) prefetch_l1(p.q + nrow * p.G * D + lane * 64);
+      if (p.k_new != nullptr && (lane & 15) * 64 < D) prefetch_l1((lane < 16 ? p.k_new : p.v_new) + nrow * D + (lane & 15) * 64);
+    }
   };
   for (u = u0; u < u1; ++u) {
     if (u - wbase == 32) {                    // slide the descriptor windows
@@ -625,6 +631,14 @@ __global__ void __maxnreg__(D > 128 ? 255 : 200) attn_splitkv_kernel(AttnParams 
       for (int nt = 0; nt < NT; ++nt) o[nt][0] = o[nt][1] = o[nt][2] = o[nt][3] = 0.f;
       m_lo = m_hi = -1e30f;
       l_lo = l_hi = 0.f;
+      // Rows follow each other in memory (q: [row][G][D], k_new / v_new: [row][D]) and, mostly, in this
+      // worker's units: ask L1 for the next row's queries and its new key and value now, so that the next row
+      // switch and that row's last unit do not each wait for an L2 round trip.
+      if (row + 1 < p.batch * p.Hkv) {
+        if (lane * 64 < p.G * D) prefetch_l1(p.q + (int64_t)(row + 1) * p.G * D + lane * 64);
+        if (p.k_new != nullptr && (lane & 15) * 64 < D)
+          prefetch_l1((lane < 16 ? p.k_new : p.v_new) + (int64_t)(row + 1) * D + (lane & 15) * 64);
+      }
     }
 
     // fused append: this unit is the page that receives the step's new key/value row
