@@ -27,7 +27,7 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 
-def measure_point(batch, seq_len, window, Hq=32, Hkv=8, D=128, submits=30):
+def measure_point(batch, seq_len, window, Hq=32, Hkv=8, D=128, submits=30, rounds=3):
     import torch
 
     from paper_2609_14237_b200 import binding, synth
@@ -37,7 +37,7 @@ def measure_point(batch, seq_len, window, Hq=32, Hkv=8, D=128, submits=30):
     per_layer = batch * visible * kvb
     layers = int(min(16, max(2, -(-(1 << 30) // max(per_layer, 1)))))
     wl = synth.Workload("profile", batch, Hq, Hkv, D, [window] * layers, f"const_{seq_len}", 4242)
-    inp = synth.make_inputs(wl, device="cuda", growth=submits + 8, steps=1)
+    inp = synth.make_inputs(wl, device="cuda", growth=rounds * submits + 8, steps=1)
     st = binding.Stage(pools=inp.pools, layer_window=wl.layer_window, num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D,
                        max_batch=batch, max_pages_per_seq=inp.max_pages_per_seq)
     pos = torch.from_numpy(inp.positions(0)).cuda()
@@ -50,21 +50,28 @@ def measure_point(batch, seq_len, window, Hq=32, Hkv=8, D=128, submits=30):
     for _ in range(3):
         binding.opw_attn_plan_submit(plan, stream.cuda_stream)
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(submits):
-        binding.opw_attn_plan_submit(plan, stream.cuda_stream)
-    e1.record(stream)
-    torch.cuda.synchronize()
+    # the fastest of `rounds` timed rounds: a point measured right after a much larger one (its pools just
+    # freed, the clocks still settling) can read several per cent slow in a single round
+    times = []
+    for _ in range(rounds):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(submits):
+            binding.opw_attn_plan_submit(plan, stream.cuda_stream)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1) * 1e3 / (submits * layers))
     assert st.poll_error() == binding.OPW_OK
-    t_us = e0.elapsed_time(e1) * 1e3 / (submits * layers)
-    tokens = sum(min(seq_len + 4 + i, window) if window else seq_len + 4 + i for i in range(submits)) / submits
+    t_us = min(times)
+    first = 4 + submits * times.index(t_us)                # tokens appended before the fastest round began
+    tokens = sum(min(seq_len + first + i, window) if window else seq_len + first + i for i in range(submits)) / submits
     nbytes = batch * tokens * kvb
     binding.opw_attn_plan_destroy(plan)
     st.close()
     del inp
     torch.cuda.empty_cache()
     return {"batch": batch, "seq_len": seq_len, "window": window, "layers": layers, "t_us": round(t_us, 2),
+            "t_us_median": round(float(np.median(times)), 2),
             "kv_bytes": int(nbytes), "beta_eff_gbs": round(nbytes / (t_us * 1e-6) / 1e9, 1)}
 
 
