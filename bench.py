@@ -753,7 +753,8 @@ def run_afd_module(steps, name="c2_llama8b", hidden=4096, layers=4, batch=None):
                                 max_batch=Bn, max_pages_per_seq=inp.max_pages_per_seq, flags=binding.OPW_FLAG_NO_PDL)
     res = {}
     for label, st, flags in (("tcgen05", stage, 0), ("library", stage, binding.OPW_AFD_LIBRARY_GEMM),
-                             ("tcgen05_no_pdl", stage_plain, binding.OPW_AFD_NO_PDL)):
+                             ("tcgen05_no_pdl", stage_plain, binding.OPW_AFD_NO_PDL),
+                             ("tcgen05_no_cluster", stage, binding.OPW_AFD_NO_CLUSTER)):
         mods = [binding.AfdModule(st, l, w_qkv[l], w_o[l], 10000.0, flags) for l in range(layers)]
         res[label] = timed(lambda l, pos: mods[l].step(x, pos, inp.page_tables[l], y))
         assert all(m.poll_error() == 0 for m in mods) and st.poll_error() == 0
@@ -786,6 +787,7 @@ def run_afd_module(steps, name="c2_llama8b", hidden=4096, layers=4, batch=None):
     return {"value": round(Bn / (res["tcgen05"] * 1e-3), 1), "unit": "sequence-steps/s per layer (whole attention module)",
             "ms_per_step": round(res["tcgen05"], 5), "ms_per_step_library_gemm": round(res["library"], 5),
             "ms_per_step_without_programmatic_dependent_launch": round(res["tcgen05_no_pdl"], 5),
+            "ms_per_step_without_clusters": round(res["tcgen05_no_cluster"], 5),
             "ms_per_step_plan": round(res["plan"], 5),
             "ms_per_step_core_attention_alone": round(res["attention"], 5),
             "projection_weight_bytes_per_step": weight_bytes, "kv_bytes_per_step": int(inp.kv_bytes(0, 0)),

@@ -44,6 +44,9 @@ typedef struct opw_afd_module opw_afd_module_t;
 #define OPW_AFD_NO_PDL 2u       /* launch the tensor-core projections without programmatic dependent launch (by
                                    default their set-up and first weight tiles overlap the tail of the previous
                                    kernel in the stream, as the stage's own kernels do) */
+#define OPW_AFD_NO_CLUSTER 4u   /* never run the K-splits of a weight tile as a thread-block cluster: their partial tiles
+                                   always meet in the workspace (the path taken anyway where the clusters of a launch do
+                                   not all fit the device, and for heads that span two weight tiles) */
 
 /* Scratch bytes of one module: qkv, q, k_new, v_new and attention-output buffers for
  * max_batch rows, split-K partial tiles, the table of rotation angles, 32 MiB of workspace for

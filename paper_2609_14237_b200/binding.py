@@ -99,7 +99,7 @@ class PlanOp(ctypes.Structure):
 
 OPW_OP_ATTENTION, OPW_OP_LINEAR, OPW_OP_AFD_MODULE = 0, 1, 2
 OPW_PLAN_GRAPH, OPW_PLAN_ADVANCE, OPW_PLAN_OVERLAP = 1, 2, 4
-OPW_AFD_LIBRARY_GEMM, OPW_AFD_NO_PDL = 1, 2
+OPW_AFD_LIBRARY_GEMM, OPW_AFD_NO_PDL, OPW_AFD_NO_CLUSTER = 1, 2, 4
 
 
 def build(force: bool = False, verbose: bool = False) -> str:

@@ -116,7 +116,7 @@ struct opw_afd_module {
   unsigned char* ws;
   size_t off_qkv, off_q, off_k, off_v, off_out, off_gemm, off_partials, off_tickets, off_angles, off_status;
   // tensor-core path
-  bool tc_qkv, tc_o, pdl, coop_ok;
+  bool tc_qkv, tc_o, pdl, coop_ok, no_cluster;
   int max_clusters[opw_afd::kMaxSplit + 1];   // [ks]: thread-block clusters of (1, ks, 1) of the GEMM kernel the device holds at once
   int sms;
   TensorMapEncodeFn encode;
@@ -255,7 +255,7 @@ opw_status_t run_tc_gemm(opw_afd_module* m, const CUtensorMap& map_w, const void
   // there are SMs: 45 clusters of three on a B200 with 148 SMs, 33 of four, 74 of two); a narrower split that
   // fits is preferred to a wider one that does not.
   p.cluster = 0;
-  if (p.group == 1 && p.ksplit > 1) {
+  if (p.group == 1 && p.ksplit > 1 && !m->no_cluster) {
     for (int ks = p.ksplit; ks >= 2; --ks)
       if (tiles_of(n_out) * batch_tiles_of(batch) <= m->max_clusters[ks]) {
         p.ksplit = ks;
@@ -333,7 +333,7 @@ opw_status_t opw_afd_module_create(opw_attn_stage_t* stage, int32_t layer, int32
                                    const void* w_o, float rope_theta, uint32_t flags, void* workspace,
                                    size_t workspace_bytes, opw_afd_module_t** out) {
   if (!stage || !w_qkv || !w_o || !workspace || !out) return OPW_ERR_INVALID_ARG;
-  if (hidden < 8 || hidden % 8 != 0 || !(rope_theta > 0.f) || (flags & ~(OPW_AFD_LIBRARY_GEMM | OPW_AFD_NO_PDL))) return OPW_ERR_INVALID_ARG;
+  if (hidden < 8 || hidden % 8 != 0 || !(rope_theta > 0.f) || (flags & ~(OPW_AFD_LIBRARY_GEMM | OPW_AFD_NO_PDL | OPW_AFD_NO_CLUSTER))) return OPW_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255) || (reinterpret_cast<uintptr_t>(w_qkv) & 15) ||
       (reinterpret_cast<uintptr_t>(w_o) & 15))
     return OPW_ERR_INVALID_ARG;
@@ -362,6 +362,7 @@ opw_status_t opw_afd_module_create(opw_attn_stage_t* stage, int32_t layer, int32
   m->tc_qkv = !library;
   m->tc_o = !library;
   m->pdl = (flags & OPW_AFD_NO_PDL) == 0;
+  m->no_cluster = (flags & OPW_AFD_NO_CLUSTER) != 0;
   bool ok = true;
   if (m->tc_qkv || m->tc_o) {
     void* fn = nullptr;

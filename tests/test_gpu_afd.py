@@ -170,6 +170,15 @@ def test_module_without_programmatic_dependent_launch():
     run_module(17, [40, 900, 33, 2047], 16, 4, 128, 1024, steps=3, flags=B.OPW_AFD_NO_PDL)
 
 
+@pytest.mark.parametrize("Hq,Hkv,D,hidden,n", [(8, 2, 64, 256, 5), (16, 2, 128, 512, 40), (32, 8, 128, 4096, 8), (4, 2, 64, 256, 200)])
+def test_module_with_the_partial_tiles_meeting_in_the_workspace(Hq, Hkv, D, hidden, n):
+    """The K-splits of a weight tile run as a thread-block cluster wherever all clusters of a launch fit the
+    device (every other test at these shapes); this is the hand-off through the workspace that larger launches
+    and two-tile heads fall back to: last CTA of a tile up to 128 rows, the cooperative back end above."""
+    rng = np.random.default_rng(50 + n)
+    run_module(51 + n, list(rng.integers(1, 300, n)), Hq, Hkv, D, hidden, steps=2, inactive=(1,), flags=B.OPW_AFD_NO_CLUSTER)
+
+
 @BOTH
 def test_llama8b_layer_shape_and_a_batch_that_changes_between_steps(flags):
     run_module(21, [17, 900, 33, 2047, 512, 64, 5, 1200], 32, 8, 128, 4096, steps=3, batches=[8, 3, 8], flags=flags)
@@ -243,7 +252,7 @@ def test_create_and_step_validate_arguments():
     base = (ws.data_ptr() + 255) // 256 * 256
     for kw, status in ((dict(layer=1), B.OPW_ERR_INVALID_ARG), (dict(hidden=12), B.OPW_ERR_INVALID_ARG),
                        (dict(rope_theta=0.0), B.OPW_ERR_INVALID_ARG), (dict(workspace=base + 8), B.OPW_ERR_INVALID_ARG),
-                       (dict(flags=4), B.OPW_ERR_INVALID_ARG),
+                       (dict(flags=8), B.OPW_ERR_INVALID_ARG),
                        (dict(workspace_bytes=nbytes - 1), B.OPW_ERR_CAPACITY)):
         args = dict(stage=stage.handle, layer=0, hidden=256, w_qkv=w_qkv.data_ptr(), w_o=w_o.data_ptr(),
                     rope_theta=1e4, workspace=base, workspace_bytes=nbytes)
