@@ -387,12 +387,14 @@ static opw_status_t validate_step(opw_attn_stage_t* st, const StepArgs& a) {
   return OPW_OK;
 }
 
-// The split-KV kernel of one step, using workspace set `ws_set` (0 or 1).
 // Launches with this many (sequence, kv head) rows or more have the attention kernel list the rows it leaves
-// as partials and the combine walk that list instead of running a block per row (see combine_kernel).
+// as partials and the combine walk that list instead of running a block per row (see combine_kernel).  Measured
+// on both sides of the threshold: 2048 rows of about 200 pages each (most rows split) 517 us per step with a
+// block per row, 532 us with the list; 8192 rows of about 10 pages 161 against 149 us.
 constexpr int kRowListMin = 4096;
 static inline bool use_row_list(const opw_attn_stage_t* st, int batch) { return batch * st->cfg.num_kv_heads >= kRowListMin; }
 
+// The split-KV kernel of one step, using workspace set `ws_set` (0 or 1).
 static opw_status_t launch_attention(opw_attn_stage_t* st, const StepArgs& a, int ws_set, cudaStream_t stream) {
   const int D = st->cfg.head_dim, Hq = st->cfg.num_q_heads, Hkv = st->cfg.num_kv_heads, G = Hq / Hkv;
   opw::AttnParams p;
