@@ -117,7 +117,7 @@ struct opw_afd_module {
   size_t off_qkv, off_q, off_k, off_v, off_out, off_gemm, off_partials, off_tickets, off_angles, off_status;
   // tensor-core path
   bool tc_qkv, tc_o, pdl, coop_ok, no_cluster;
-  int max_clusters[opw_afd::kMaxSplit + 1];   // [ks]: thread-block clusters of (1, ks, 1) of the GEMM kernel the device holds at once
+  int max_clusters[2 * opw_afd::kMaxSplit + 1];   // [n]: thread-block clusters of n CTAs of the GEMM kernel the device holds at once
   int sms;
   TensorMapEncodeFn encode;
   CUtensorMap map_wqkv, map_wo;
@@ -208,7 +208,7 @@ bool encode_map(TensorMapEncodeFn fn, CUtensorMap* map, const void* base, uint64
 // `coop`: a cooperative launch -- the whole grid is resident at once or the launch is refused.
 template <typename... KArgs, typename... Args>
 cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, bool pdl, bool coop,
-                       int cluster_y, Args&&... args) {
+                       int cluster_x, int cluster_y, Args&&... args) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
   cfg.blockDim = block;
@@ -216,9 +216,9 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
   cfg.stream = stream;
   cudaLaunchAttribute attr[3];
   int n = 0;
-  if (cluster_y > 1) {                          // thread-block clusters of (1, cluster_y, 1)
+  if (cluster_x * cluster_y > 1) {              // thread-block clusters of (cluster_x, cluster_y, 1)
     attr[n].id = cudaLaunchAttributeClusterDimension;
-    attr[n].val.clusterDim.x = 1;
+    attr[n].val.clusterDim.x = (unsigned)cluster_x;
     attr[n].val.clusterDim.y = (unsigned)cluster_y;
     attr[n].val.clusterDim.z = 1;
     ++n;
@@ -255,9 +255,9 @@ opw_status_t run_tc_gemm(opw_afd_module* m, const CUtensorMap& map_w, const void
   // there are SMs: 45 clusters of three on a B200 with 148 SMs, 33 of four, 74 of two); a narrower split that
   // fits is preferred to a wider one that does not.
   p.cluster = 0;
-  if (p.group == 1 && p.ksplit > 1 && !m->no_cluster) {
-    for (int ks = p.ksplit; ks >= 2; --ks)
-      if (tiles_of(n_out) * batch_tiles_of(batch) <= m->max_clusters[ks]) {
+  if (p.ksplit * p.group > 1 && !m->no_cluster && tiles_of(n_out) % p.group == 0) {
+    for (int ks = p.ksplit; ks * p.group >= 2; --ks)
+      if (tiles_of(n_out) / p.group * batch_tiles_of(batch) <= m->max_clusters[ks * p.group]) {
         p.ksplit = ks;
         p.cluster = 1;
         break;
@@ -276,7 +276,7 @@ opw_status_t run_tc_gemm(opw_afd_module* m, const CUtensorMap& map_w, const void
                           opw_afd::kTileM * sizeof(float);
   const size_t epi_last = p.group == 1 ? (size_t)p.nb * opw_afd::kTileM * sizeof(float)
                                        : ((size_t)opw_afd::kChunkCols + chunk_cols) * opw_afd::kTileM * sizeof(float);
-  const size_t epi_bytes = p.coop ? epi_coop : epi_last;
+  const size_t epi_bytes = (p.coop || (p.cluster && p.group == 2)) ? epi_coop : epi_last;
   bool angles_global = mode == 1 && batch > kSmemAngleBatch;
   size_t angle_bytes = 0;
   int stages = 0;
@@ -301,7 +301,7 @@ opw_status_t run_tc_gemm(opw_afd_module* m, const CUtensorMap& map_w, const void
   // trace region 0: output projection, region 1: QKV projection
   p.trace = m->trace ? m->trace + (size_t)mode * opw_afd::kTraceMaxCtas * opw_afd::kTraceWords : nullptr;
   if (angles_global) {
-    if (launch_pdl(opw_afd::rope_table_kernel, dim3(batch), dim3(128), 0, stream, m->pdl, false, 0, positions,
+    if (launch_pdl(opw_afd::rope_table_kernel, dim3(batch), dim3(128), 0, stream, m->pdl, false, 1, 1, positions,
                    reinterpret_cast<float2*>(m->ws + m->off_angles), (int)m->D, m->log_theta) != cudaSuccess) {
       (void)cudaGetLastError();
       return OPW_ERR_CUDA;
@@ -312,7 +312,7 @@ opw_status_t run_tc_gemm(opw_afd_module* m, const CUtensorMap& map_w, const void
   if (!encode_map(m->encode, &map_x, x, (uint64_t)batch, (uint64_t)k, (uint32_t)p.nb)) return OPW_ERR_CUDA;
   const dim3 grid(tiles_of(n_out), p.ksplit, batch_tiles_of(batch));
   if (launch_pdl(opw_afd::skinny_gemm_kernel, grid, dim3(opw_afd::kGemmThreads), 1024 + (size_t)stages * stage_bytes + angle_bytes,
-                 stream, m->pdl, p.coop != 0, p.cluster ? p.ksplit : 0, map_w, map_x, p) != cudaSuccess) {
+                 stream, m->pdl, p.coop != 0, p.cluster ? p.group : 1, p.cluster ? p.ksplit : 1, map_w, map_x, p) != cudaSuccess) {
     (void)cudaGetLastError();
     return OPW_ERR_CUDA;
   }
@@ -378,8 +378,8 @@ opw_status_t opw_afd_module_create(opw_attn_stage_t* stage, int32_t layer, int32
     m->coop_ok = coop != 0;
     ok = ok && cudaFuncSetAttribute(opw_afd::skinny_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                     (int)kGemmSmemBudget) == cudaSuccess;
-    for (int ks = 0; ks <= opw_afd::kMaxSplit; ++ks) m->max_clusters[ks] = 0;
-    for (int ks = 2; ok && ks <= opw_afd::kMaxSplit; ++ks) {
+    for (int ks = 0; ks <= 2 * opw_afd::kMaxSplit; ++ks) m->max_clusters[ks] = 0;
+    for (int ks = 2; ok && ks <= 2 * opw_afd::kMaxSplit; ++ks) {
       cudaLaunchConfig_t cfg = {};
       cfg.gridDim = dim3(1, ks, 1);
       cfg.blockDim = dim3(opw_afd::kGemmThreads);

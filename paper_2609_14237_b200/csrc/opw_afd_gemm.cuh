@@ -15,13 +15,14 @@
 // With N/128 tiles alone a 6144 x 4096 projection would occupy 48 of 148 SMs, too few to pull
 // the weights at HBM speed, so K is also split over `ksplit` CTAs per tile, and the partial tiles
 // have to meet.  Three back ends, chosen by the host:
-//   * cluster: the ksplit CTAs of a tile are one thread-block cluster (1, ksplit, 1).  They are resident
-//     together by construction, meet at the cluster's hardware barrier, and each adds up and finishes its own
-//     slice of the batch columns, reading the other members' tiles from their shared memory.  Used whenever
-//     the device holds all clusters of the launch at once (a cluster needs its SMs in one GPC).
+//   * cluster: the ksplit CTAs of a tile -- or, where a head spans two weight tiles (D = 256), the 2 * ksplit
+//     CTAs of both -- are one thread-block cluster (1 or 2, ksplit, 1).  They are resident together by
+//     construction, meet at the cluster's hardware barrier, and each adds up and finishes its own slice of the
+//     batch columns, reading the other members' tiles from their shared memory.  Used whenever the device
+//     holds all clusters of the launch at once (a cluster needs its SMs in one GPC).
 //   * cooperative: the whole grid is resident (cooperative launch); the CTAs of a tile meet at a counter in
 //     global memory and share the back end the same way, the partial tiles passing through the workspace.
-//     Used for heads that span two weight tiles (D = 256) at large batches.
+//     Used at large batches where the clusters do not fit.
 //   * last CTA: with no residency guarantee nobody may wait; every CTA writes its partial tile to the
 //     workspace and the last one of a tile to arrive (an atomic ticket) reduces and finishes all of it.
 // In all three the partial tiles are added in split order: deterministic.
@@ -62,8 +63,8 @@ struct GemmParams {
   int nb;                 // MMA N of a full batch tile: min(batch, 256) rounded up to a multiple of 16
   int group;              // weight tiles that share a ticket and an epilogue: 1, or 2 (rotary at D = 256)
   int coop;               // the launch is cooperative (every CTA resident): the CTAs of a ticket group share the back end
-  int cluster;            // the ksplit CTAs of a weight tile form a thread-block cluster (1, ksplit, 1): they exchange their
-                          // partial tiles through distributed shared memory (group == 1 only)
+  int cluster;            // the ksplit * group CTAs of a ticket group form a thread-block cluster (group, ksplit, 1): they
+                          // exchange their partial tiles through distributed shared memory
   const float2* angles_g; // mode 1: [batch, D/2] (cos, sin) in global memory, or null: computed here in shared memory
   int stages;
   int ksplit;
@@ -477,57 +478,81 @@ skinny_gemm_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_const
     // stores, and members exchanging the slices through the workspace in L2 with only the barrier taken from the
     // cluster, were both slower (the cluster's network moves some 20 GB/s per SM either way; a write to L2 and a
     // read back are two round trips where this is one). ----
-    const int ks = p.ksplit;
-    if (tid == 0) s_flags[0] = good ? 1u : 0u;
+    // A head that spans two weight tiles (group = 2) makes the cluster (2, ksplit, 1): the 2 * ksplit CTAs of both
+    // tiles, each owning a slice of the columns for which it sums both tiles (its own in place, the other into a
+    // second buffer) and rotates each against the other.
+    const int ks = p.ksplit, members = ks * p.group;
+    const int tl = p.group == 2 ? (tile & 1) : 0;                         // this CTA's tile inside the group
+    const int rank = tl * ks + split;                                     // which slice it owns
+    auto cta_of = [&](int tl_, int sp_) -> uint32_t { return p.group == 2 ? (uint32_t)(tl_ + 2 * sp_) : (uint32_t)sp_; };
+    uint32_t my_cta;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(my_cta));
+    if (tid == 0) s_flags[0] = (good && my_cta == cta_of(tl, split)) ? 1u : 0u;   // (a rank order other than x-major: treated as a failure)
     g_cluster_arrive();
     g_cluster_wait();
     g_stamp(p, cta, 4);
-    const int cb = (int)((int64_t)batch_here * split / ks), ce = (int)((int64_t)batch_here * (split + 1) / ks);
+    const int cb = (int)((int64_t)batch_here * rank / members), ce = (int)((int64_t)batch_here * (rank + 1) / members);
     float* mine = stage_f + (size_t)cb * kTileM;
+    float* other = stage_f + split_floats;                                // the head's other tile, this slice (group = 2)
     // The members' flags and the values are requested together: one round trip through the cluster's network,
     // not one per member.  The sums are formed whatever the flags say (a failed member's tile is just numbers);
     // only the epilogue depends on them.
-    uint32_t flag[kMaxSplit];
+    uint32_t flags_and = 1u;
     const uint32_t flag_local = g_smem_u32(const_cast<uint32_t*>(&s_flags[0]));
-#pragma unroll
-    for (int sp = 0; sp < kMaxSplit; ++sp) flag[sp] = sp < ks ? g_ld_cluster_u32(g_mapa(flag_local, (uint32_t)sp)) : 1u;
     {
+      uint32_t flag[2 * kMaxSplit];
+#pragma unroll
+      for (int m = 0; m < 2 * kMaxSplit; ++m) flag[m] = m < members ? g_ld_cluster_u32(g_mapa(flag_local, (uint32_t)m)) : 1u;
+      // dst[i] = sum over the splits of tile `tls` of their values at the slice, in split order; `own`: this CTA's
+      // own partial is one of them and is read from `src_local` (which may be dst itself)
       const int n4 = (ce - cb) * kTileM / 4;
-      float4* dst = reinterpret_cast<float4*>(mine);
-      const uint32_t local = g_smem_u32(dst);
-      uint32_t remote[kMaxSplit];
+      const uint32_t slice_local = g_smem_u32(mine);
+      auto pull_sum = [&](float4* dst, int tls, bool own) {
+        uint32_t remote[kMaxSplit];
 #pragma unroll
-      for (int sp = 0; sp < kMaxSplit; ++sp) remote[sp] = sp < ks ? g_mapa(local, (uint32_t)sp) : 0u;
-      constexpr int R = 2;
-      for (int ib = tid; ib < n4; ib += R * kGemmThreads) {
-        float4 v[R][kMaxSplit];
+        for (int sp = 0; sp < kMaxSplit; ++sp) remote[sp] = sp < ks ? g_mapa(slice_local, cta_of(tls, sp)) : 0u;
+        constexpr int R = 2;
+        for (int ib = tid; ib < n4; ib += R * kGemmThreads) {
+          float4 v[R][kMaxSplit];
 #pragma unroll
-        for (int r = 0; r < R; ++r)
+          for (int r = 0; r < R; ++r)
 #pragma unroll
-          for (int sp = 0; sp < kMaxSplit; ++sp) {
-            const int i = ib + r * kGemmThreads;
-            if (i < n4 && sp < ks && sp != split) v[r][sp] = g_ld_cluster_f4(remote[sp] + 16u * (uint32_t)i);
-          }
-#pragma unroll
-        for (int r = 0; r < R; ++r) {
-          const int i = ib + r * kGemmThreads;
-          if (i >= n4) break;
-          float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-#pragma unroll
-          for (int sp = 0; sp < kMaxSplit; ++sp)
-            if (sp < ks) {
-              const float4 t = sp == split ? dst[i] : v[r][sp];
-              acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+            for (int sp = 0; sp < kMaxSplit; ++sp) {
+              const int i = ib + r * kGemmThreads;
+              if (i < n4 && sp < ks && !(own && sp == split)) v[r][sp] = g_ld_cluster_f4(remote[sp] + 16u * (uint32_t)i);
             }
-          dst[i] = acc;
+#pragma unroll
+          for (int r = 0; r < R; ++r) {
+            const int i = ib + r * kGemmThreads;
+            if (i >= n4) break;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int sp = 0; sp < kMaxSplit; ++sp)
+              if (sp < ks) {
+                const float4 t = (own && sp == split) ? reinterpret_cast<const float4*>(mine)[i] : v[r][sp];
+                acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+              }
+            dst[i] = acc;
+          }
         }
-      }
+      };
+      pull_sum(reinterpret_cast<float4*>(mine), tl, true);
+      if (p.group == 2) pull_sum(reinterpret_cast<float4*>(other), tl ^ 1, false);
+#pragma unroll
+      for (int m = 0; m < 2 * kMaxSplit; ++m) flags_and &= flag[m];
     }
-    const bool all_good = (flag[0] & flag[1] & flag[2] & flag[3]) != 0;
+    const bool all_good = flags_and != 0;
     __syncthreads();
     g_cluster_arrive();                         // this CTA no longer reads the others' shared memory
     g_stamp(p, cta, 5);
-    if (all_good && ce > cb) epilogue(tile, mine, mine, cb, ce);
+    if (all_good && ce > cb) {
+      if (p.group == 1) {
+        epilogue(tile, mine, mine, cb, ce);
+      } else {
+        epilogue(tile, mine, other, cb, ce);
+        epilogue(tile ^ 1, other, mine, cb, ce);
+      }
+    }
     g_cluster_wait();                           // and leaves only when nobody reads its own any more
     g_stamp(p, cta, 6);
     return;

@@ -237,6 +237,33 @@ def test_the_two_projection_paths_agree():
     assert np.abs(outs[0][3] - outs[1][3]).max() <= 2.0 ** -5 * rms
 
 
+@pytest.mark.parametrize("Hq,Hkv,D,hidden,n", [(4, 2, 256, 512, 70), (8, 2, 128, 1024, 33), (4, 2, 256, 256, 200)])
+def test_cluster_and_workspace_hand_offs_give_the_same_bits(Hq, Hkv, D, hidden, n):
+    """Where both hand-offs cut K the same way, the partial tiles are added in the same (split) order: q, k, v and
+    y come out bit for bit the same whether the K-splits met in a thread-block cluster or in the workspace."""
+    outs = []
+    for flags in (0, B.OPW_AFD_NO_CLUSTER):
+        rng = np.random.default_rng(77)
+        lens = [int(v) for v in rng.integers(1, 90, n)]
+        pool_np, tab, _, _, _ = make_case(rng, [v + 1 for v in lens], Hq, Hkv, D)
+        w1 = to_dev_bf16(oracle.f32_to_bf16_bits((rng.standard_normal(((Hq + 2 * Hkv) * D, hidden)) / hidden ** 0.5).astype(np.float32)))
+        w2 = to_dev_bf16(oracle.f32_to_bf16_bits((rng.standard_normal((hidden, Hq * D)) / (Hq * D) ** 0.5).astype(np.float32)))
+        x = to_dev_bf16(oracle.f32_to_bf16_bits(rng.standard_normal((n, hidden)).astype(np.float32)))
+        stage = B.Stage(pools=[to_dev_bf16(pool_np)], layer_window=[0], num_q_heads=Hq, num_kv_heads=Hkv, head_dim=D, max_batch=n,
+                        max_pages_per_seq=tab.shape[1])
+        mod = B.AfdModule(stage, 0, w1, w2, THETA, flags)
+        y = torch.empty(n, hidden, dtype=torch.bfloat16, device="cuda")
+        mod.step(x, torch.tensor(lens, dtype=torch.int32, device="cuda"), torch.from_numpy(tab).cuda(), y)
+        torch.cuda.synchronize()
+        assert mod.poll_error() == B.OPW_OK and stage.poll_error() == B.OPW_OK
+        outs.append([t.clone().view(torch.int16) for t in mod.intermediates(n)[:3]] + [y.view(torch.int16)])
+        mod.close()
+        stage.close()
+    # (these launches have so few weight tiles that their clusters fit any B200 without narrowing the K-split)
+    for a, b_ in zip(outs[0], outs[1]):
+        assert torch.equal(a, b_)
+
+
 def test_create_and_step_validate_arguments():
     pool = torch.zeros(4 * 2 * 2 * P * 64, dtype=torch.bfloat16, device="cuda")
     stage = B.Stage(pools=[pool], layer_window=[0], num_q_heads=8, num_kv_heads=2, head_dim=64, max_batch=2,
